@@ -1,0 +1,296 @@
+/*
+ * ARL^2 hybrid attention layer -- CPU float64 oracle.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the
+ * layer computes, written from the paper's equations.  It shares no code with the
+ * CUDA library and must never be reached from the product path: only the tests,
+ * the smoke check and the bench's CPU-baseline leg may build or call it.
+ *
+ * Everything is double precision, plain loops, no blocking, no fusion.  The only
+ * parallelism is an OpenMP loop over independent (stream, head, row) units, used
+ * when the file is built with -fopenmp for the timed CPU baseline.
+ *
+ * Layouts (all host pointers, row-major, contiguous):
+ *   q, k, v, out   [B, L, H, D]   token-major, the shape of x*W reshaped to heads
+ *   g              [B, L, H]      combine-gate logits x*W_g (Eq. 6)
+ *   S              [B, H, D, D]   recurrent state, row = key dim, column = value dim
+ *   w_phi_*        [H, D, D]      per-head feature map, applied as row-vector * W
+ *                                 (index [h][in][out]); NULL = identity
+ *   rope_cos/sin   [L, D/2]       rotation tables; NULL = no rotation
+ *   a              [B, H]         decay-gate logits, alpha = sigmoid(a)
+ *   beta_logit     [B, L, H]      learning-rate logits (delta rules only)
+ *
+ * Readings of the paper where it is silent (each is an interface choice, listed
+ * again in the design notes):
+ *   - RoPE rotates adjacent pairs (2m, 2m+1) by the angle whose cos/sin the caller
+ *     supplies per token: (x0, x1) -> (x0 c - x1 s, x0 s + x1 c).      [parity unpinned]
+ *   - L2Norm(x) = x / sqrt(sum_d x_d^2 + eps), over the head dimension.  [eps: parity unpinned]
+ *   - phi is a bias-free linear map per head (a grouped 1x1 convolution).
+ *   - softmax scale is 1/sqrt(D) as in Eq. 1 unless the caller passes another.
+ *   - gates are the logistic sigmoid of the supplied logits.
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static double sigmoid(double x) { return 1.0 / (1.0 + exp(-x)); }
+
+int arl2_oracle_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* RoPE of one head vector x[D] at token position `pos` (Eq. 2, Eq. 3), in place. */
+static void rope(double *x, int D, const double *cos_t, const double *sin_t, int pos)
+{
+    if (!cos_t || !sin_t) return;
+    for (int m = 0; m < D / 2; ++m) {
+        double c = cos_t[(size_t)pos * (D / 2) + m];
+        double s = sin_t[(size_t)pos * (D / 2) + m];
+        double x0 = x[2 * m], x1 = x[2 * m + 1];
+        x[2 * m]     = x0 * c - x1 * s;
+        x[2 * m + 1] = x0 * s + x1 * c;
+    }
+}
+
+/* y = x * W_h  (row vector times the head's D x D map); W == NULL is the identity. */
+static void phi(const double *x, const double *W, int h, int D, double *y)
+{
+    if (!W) { memcpy(y, x, sizeof(double) * D); return; }
+    const double *Wh = W + (size_t)h * D * D;
+    for (int o = 0; o < D; ++o) {
+        double acc = 0.0;
+        for (int i = 0; i < D; ++i) acc += x[i] * Wh[(size_t)i * D + o];
+        y[o] = acc;
+    }
+}
+
+static void l2norm(double *x, int D, double eps)
+{
+    double ss = 0.0;
+    for (int d = 0; d < D; ++d) ss += x[d] * x[d];
+    double r = 1.0 / sqrt(ss + eps);
+    for (int d = 0; d < D; ++d) x[d] *= r;
+}
+
+/*
+ * Feature maps of Eq. 3 for one tensor x [B, L, H, D]:
+ *   mode 0: y = L2Norm(RoPE(phi(x)))   (Q' and K')
+ *   mode 1: y = phi(x)                 (V')
+ */
+void arl2_oracle_feature(int B, int H, int L, int D, const double *x, const double *W,
+                         const double *rope_cos, const double *rope_sin, double eps,
+                         int mode, double *y)
+{
+    for (int b = 0; b < B; ++b)
+        for (int l = 0; l < L; ++l)
+            for (int h = 0; h < H; ++h) {
+                size_t off = (((size_t)b * L + l) * H + h) * D;
+                phi(x + off, W, h, D, y + off);
+                if (mode == 0) {
+                    rope(y + off, D, rope_cos, rope_sin, l);
+                    l2norm(y + off, D, eps);
+                }
+            }
+}
+
+/*
+ * One output row of the layer: token i of head h of stream b.
+ *   O_intra = softmax_j(<RoPE(Q_i), RoPE(K_j)> * scale) V_j   over all L tokens (Eq. 2)
+ *   Q'_i    = L2Norm(RoPE(phi_q(Q_i)))                          (Eq. 3)
+ *   O_inter = Q'_i S                                            (Eq. 5 / Eq. 8)
+ *   O_i     = O_intra + sigmoid(g_i) * O_inter                  (Eq. 6-7, Algorithm 1)
+ * S is read, never written (clean-pass-only update, Sec. 3.3).
+ * scratch: at least L + 3*D doubles.
+ */
+static void step_row(int b, int h, int i, int H, int L, int D,
+                     const double *q, const double *k, const double *v, const double *g,
+                     const double *S, const double *wq,
+                     const double *rope_cos, const double *rope_sin,
+                     double scale, double eps, double *o, double *scratch)
+{
+    double *p = scratch;          /* L  */
+    double *qr = p + L;           /* D  */
+    double *kr = qr + D;          /* D  */
+    double *qf = kr + D;          /* D  */
+    size_t qoff = (((size_t)b * L + i) * H + h) * D;
+
+    memcpy(qr, q + qoff, sizeof(double) * D);
+    rope(qr, D, rope_cos, rope_sin, i);
+
+    /* scores over the whole block: bidirectional, no mask */
+    double mx = -INFINITY;
+    for (int j = 0; j < L; ++j) {
+        size_t koff = (((size_t)b * L + j) * H + h) * D;
+        memcpy(kr, k + koff, sizeof(double) * D);
+        rope(kr, D, rope_cos, rope_sin, j);
+        double s = 0.0;
+        for (int d = 0; d < D; ++d) s += qr[d] * kr[d];
+        p[j] = s * scale;
+        if (p[j] > mx) mx = p[j];
+    }
+    double den = 0.0;
+    for (int j = 0; j < L; ++j) { p[j] = exp(p[j] - mx); den += p[j]; }
+
+    for (int d = 0; d < D; ++d) o[d] = 0.0;
+    for (int j = 0; j < L; ++j) {
+        size_t voff = (((size_t)b * L + j) * H + h) * D;
+        double w = p[j] / den;
+        for (int d = 0; d < D; ++d) o[d] += w * v[voff + d];
+    }
+
+    /* inter branch: every token reads the same pre-update state */
+    phi(q + qoff, wq, h, D, qf);
+    rope(qf, D, rope_cos, rope_sin, i);
+    l2norm(qf, D, eps);
+    const double *Sh = S + ((size_t)b * H + h) * D * D;
+    double gate = sigmoid(g[((size_t)b * L + i) * H + h]);
+    for (int e = 0; e < D; ++e) {
+        double acc = 0.0;
+        for (int d = 0; d < D; ++d) acc += qf[d] * Sh[(size_t)d * D + e];
+        o[e] += gate * acc;
+    }
+}
+
+/* Full denoise-step output, every (b, h, i). */
+void arl2_oracle_step(int B, int H, int L, int D,
+                      const double *q, const double *k, const double *v, const double *g,
+                      const double *S, const double *wq,
+                      const double *rope_cos, const double *rope_sin,
+                      double scale, double eps, double *out)
+{
+    long total = (long)B * H * L;
+#pragma omp parallel
+    {
+        double *scratch = (double *)malloc(sizeof(double) * ((size_t)L + 3 * (size_t)D));
+#pragma omp for schedule(dynamic, 16)
+        for (long t = 0; t < total; ++t) {
+            int i = (int)(t % L);
+            int h = (int)((t / L) % H);
+            int b = (int)(t / ((long)L * H));
+            step_row(b, h, i, H, L, D, q, k, v, g, S, wq, rope_cos, rope_sin, scale, eps,
+                     out + (((size_t)b * L + i) * H + h) * D, scratch);
+        }
+        free(scratch);
+    }
+}
+
+/*
+ * Sampled denoise-step output: n (b, h, i) triples; out_rows is [n, D].
+ * Used where the full L x L work per head is too slow to compare in full.
+ */
+void arl2_oracle_step_rows(int B, int H, int L, int D,
+                           const double *q, const double *k, const double *v, const double *g,
+                           const double *S, const double *wq,
+                           const double *rope_cos, const double *rope_sin,
+                           double scale, double eps,
+                           int n, const int *bs, const int *hs, const int *is, double *out_rows)
+{
+    (void)B;
+#pragma omp parallel
+    {
+        double *scratch = (double *)malloc(sizeof(double) * ((size_t)L + 3 * (size_t)D));
+#pragma omp for schedule(dynamic, 4)
+        for (int t = 0; t < n; ++t)
+            step_row(bs[t], hs[t], is[t], H, L, D, q, k, v, g, S, wq, rope_cos, rope_sin,
+                     scale, eps, out_rows + (size_t)t * D, scratch);
+        free(scratch);
+    }
+}
+
+/*
+ * State commit for one (b, h), run once per block from the clean pass's K, V
+ * (Algorithm 1, clean-pass branch).  K' = L2Norm(RoPE(phi_k(K))), V' = phi_v(V).
+ *
+ *   rule 0  gated linear:  S <- alpha S + sum_j K'_j^T V'_j
+ *           (Eq. 4 with the correction term dropped and beta = 1; one decay per
+ *            head per block)
+ *   rule 1  Eq. 4 as printed, frame level:
+ *           S <- alpha S + K'^T diag(beta) (V' - K' S_old),  beta_j = sigmoid(beta_logit)
+ *   rule 2  Eq. 4 applied token by token in order j = 0..L-1, the decay alpha
+ *           applied once before the first token:
+ *           S <- alpha S;  for j: S <- S + beta_j K'_j^T (V'_j - K'_j S)
+ */
+static void commit_head(int b, int h, int H, int L, int D,
+                        const double *kc, const double *vc, double alpha,
+                        const double *beta_logit, const double *wk, const double *wv,
+                        const double *rope_cos, const double *rope_sin, double eps,
+                        int rule, double *S)
+{
+    double *Sh = S + ((size_t)b * H + h) * D * D;
+    double *kf = (double *)malloc(sizeof(double) * D);
+    double *vf = (double *)malloc(sizeof(double) * D);
+    double *pred = (double *)malloc(sizeof(double) * D);
+    double *dS = (double *)calloc((size_t)D * D, sizeof(double));
+    double *Sold = NULL;
+    if (rule == 1) {
+        Sold = (double *)malloc(sizeof(double) * D * D);
+        memcpy(Sold, Sh, sizeof(double) * D * D);
+    }
+    if (rule == 2)
+        for (size_t t = 0; t < (size_t)D * D; ++t) Sh[t] *= alpha;
+
+    for (int j = 0; j < L; ++j) {
+        size_t off = (((size_t)b * L + j) * H + h) * D;
+        phi(kc + off, wk, h, D, kf);
+        rope(kf, D, rope_cos, rope_sin, j);
+        l2norm(kf, D, eps);
+        phi(vc + off, wv, h, D, vf);
+        double beta = 1.0;
+        if (rule != 0 && beta_logit) beta = sigmoid(beta_logit[((size_t)b * L + j) * H + h]);
+        if (rule == 0) {
+            for (int d = 0; d < D; ++d)
+                for (int e = 0; e < D; ++e) dS[(size_t)d * D + e] += kf[d] * vf[e];
+        } else {
+            const double *Sref = (rule == 1) ? Sold : Sh;
+            for (int e = 0; e < D; ++e) {
+                double acc = 0.0;
+                for (int d = 0; d < D; ++d) acc += kf[d] * Sref[(size_t)d * D + e];
+                pred[e] = acc;
+            }
+            double *dst = (rule == 1) ? dS : Sh;
+            for (int d = 0; d < D; ++d)
+                for (int e = 0; e < D; ++e)
+                    dst[(size_t)d * D + e] += beta * kf[d] * (vf[e] - pred[e]);
+        }
+    }
+    if (rule == 0 || rule == 1)
+        for (size_t t = 0; t < (size_t)D * D; ++t) Sh[t] = alpha * Sh[t] + dS[t];
+
+    free(Sold); free(dS); free(pred); free(vf); free(kf);
+}
+
+/* heads: optional list of n_heads (b, h) pairs to commit; NULL = all of them. */
+void arl2_oracle_commit(int B, int H, int L, int D,
+                        const double *kc, const double *vc, const double *a,
+                        const double *beta_logit, const double *wk, const double *wv,
+                        const double *rope_cos, const double *rope_sin, double eps,
+                        int rule, int n_heads, const int *bs, const int *hs, double *S)
+{
+    int total = bs ? n_heads : B * H;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int t = 0; t < total; ++t) {
+        int b = bs ? bs[t] : t / H;
+        int h = bs ? hs[t] : t % H;
+        double alpha = sigmoid(a[(size_t)b * H + h]);
+        commit_head(b, h, H, L, D, kc, vc, alpha, beta_logit, wk, wv, rope_cos, rope_sin, eps,
+                    rule, S);
+    }
+}
+
+/* S <- 0 for stream `stream` (or all streams when stream < 0): Algorithm 1, first line. */
+void arl2_oracle_reset(int B, int H, int D, int stream, double *S)
+{
+    size_t per = (size_t)H * D * D;
+    if (stream < 0) memset(S, 0, sizeof(double) * per * B);
+    else memset(S + per * stream, 0, sizeof(double) * per);
+}

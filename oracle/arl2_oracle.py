@@ -1,0 +1,153 @@
+"""ctypes front end of the CPU float64 oracle (``arl2_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+bench's CPU-baseline leg.  Nothing on the product path imports this module, and
+this module imports nothing from the CUDA package.
+
+Every function takes numpy arrays or torch CPU tensors of any float dtype, widens
+them to float64 (so the oracle sees exactly the bf16 / fp32 values the GPU saw) and
+returns float64 numpy arrays.  Shapes follow the C file's header comment.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "arl2_oracle.c")
+_BUILD = os.path.join(_HERE, "_build")
+_SO = os.path.join(_BUILD, "libarl2_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O2 -fopenmp); returns the path of the library."""
+    with _lock:
+        stale = (not os.path.exists(_SO)) or os.path.getmtime(_SO) < os.path.getmtime(_SRC)
+        if force or stale:
+            os.makedirs(_BUILD, exist_ok=True)
+            tmp = _SO + ".%d.tmp" % os.getpid()
+            subprocess.check_call(
+                ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-Wall", "-o", tmp, _SRC, "-lm"]
+            )
+            os.replace(tmp, _SO)
+    return _SO
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        lib.arl2_oracle_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def threads() -> int:
+    """Number of OpenMP threads the oracle will use."""
+    return int(_load().arl2_oracle_threads())
+
+
+def _f64(x):
+    """Widen to a contiguous float64 numpy array (None stays None)."""
+    if x is None:
+        return None
+    if hasattr(x, "detach"):  # torch tensor
+        x = x.detach().cpu().double().numpy()
+    return np.ascontiguousarray(x, dtype=np.float64)
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _ip(a):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def feature(x, W, rope_cos, rope_sin, eps: float, mode: int):
+    """Eq. 3: mode 0 = L2Norm(RoPE(phi(x))), mode 1 = phi(x).  x is [B, L, H, D]."""
+    x, W, rope_cos, rope_sin = _f64(x), _f64(W), _f64(rope_cos), _f64(rope_sin)
+    B, L, H, D = x.shape
+    y = np.empty_like(x)
+    _load().arl2_oracle_feature(
+        B, H, L, D, _p(x), _p(W), _p(rope_cos), _p(rope_sin), ctypes.c_double(eps), mode, _p(y)
+    )
+    return y
+
+
+def step(q, k, v, g, S, wq=None, rope_cos=None, rope_sin=None, scale=None, eps=1e-6):
+    """One denoise-step call of the layer: returns O [B, L, H, D]; S is only read."""
+    q, k, v, g, S = _f64(q), _f64(k), _f64(v), _f64(g), _f64(S)
+    wq, rope_cos, rope_sin = _f64(wq), _f64(rope_cos), _f64(rope_sin)
+    B, L, H, D = q.shape
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    out = np.empty_like(q)
+    _load().arl2_oracle_step(
+        B, H, L, D, _p(q), _p(k), _p(v), _p(g), _p(S), _p(wq), _p(rope_cos), _p(rope_sin),
+        ctypes.c_double(scale), ctypes.c_double(eps), _p(out),
+    )
+    return out
+
+
+def step_rows(q, k, v, g, S, rows, wq=None, rope_cos=None, rope_sin=None, scale=None,
+              eps=1e-6):
+    """Outputs of the sampled (b, h, i) triples in ``rows`` ([n, 3] ints): returns [n, D]."""
+    q, k, v, g, S = _f64(q), _f64(k), _f64(v), _f64(g), _f64(S)
+    wq, rope_cos, rope_sin = _f64(wq), _f64(rope_cos), _f64(rope_sin)
+    B, L, H, D = q.shape
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    rows = np.asarray(rows, dtype=np.int32).reshape(-1, 3)
+    bs = np.ascontiguousarray(rows[:, 0])
+    hs = np.ascontiguousarray(rows[:, 1])
+    is_ = np.ascontiguousarray(rows[:, 2])
+    assert (bs >= 0).all() and (bs < B).all() and (hs >= 0).all() and (hs < H).all()
+    assert (is_ >= 0).all() and (is_ < L).all()
+    out = np.empty((rows.shape[0], D), dtype=np.float64)
+    _load().arl2_oracle_step_rows(
+        B, H, L, D, _p(q), _p(k), _p(v), _p(g), _p(S), _p(wq), _p(rope_cos), _p(rope_sin),
+        ctypes.c_double(scale), ctypes.c_double(eps), rows.shape[0], _ip(bs), _ip(hs), _ip(is_),
+        _p(out),
+    )
+    return out
+
+
+def commit(kc, vc, a, S, wk=None, wv=None, rope_cos=None, rope_sin=None, eps=1e-6, rule=0,
+           beta_logit=None, heads=None):
+    """State commit, once per block.  Returns the new S (the argument is not modified).
+
+    ``heads``: optional [n, 2] list of (b, h) pairs; other heads are left as they were.
+    """
+    kc, vc, a = _f64(kc), _f64(vc), _f64(a)
+    wk, wv, rope_cos, rope_sin = _f64(wk), _f64(wv), _f64(rope_cos), _f64(rope_sin)
+    beta_logit = _f64(beta_logit)
+    S = _f64(S).copy()
+    B, L, H, D = kc.shape
+    assert S.shape == (B, H, D, D) and a.shape == (B, H)
+    if heads is None:
+        n, bs, hs = 0, None, None
+    else:
+        heads = np.asarray(heads, dtype=np.int32).reshape(-1, 2)
+        n = heads.shape[0]
+        bs = np.ascontiguousarray(heads[:, 0])
+        hs = np.ascontiguousarray(heads[:, 1])
+    _load().arl2_oracle_commit(
+        B, H, L, D, _p(kc), _p(vc), _p(a), _p(beta_logit), _p(wk), _p(wv), _p(rope_cos),
+        _p(rope_sin), ctypes.c_double(eps), rule, n, _p(bs), _p(hs), _p(S),
+    )
+    return S
+
+
+def reset(S, stream: int = -1):
+    """S <- 0 for one stream or all (stream < 0).  Returns a new array."""
+    S = _f64(S).copy()
+    B, H, D, _ = S.shape
+    _load().arl2_oracle_reset(B, H, D, stream, _p(S))
+    return S

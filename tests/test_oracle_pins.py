@@ -1,0 +1,397 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+None of these tests touches the CUDA path.  Each pin is chosen so that a plausible
+mistake in the oracle (a dropped term, a wrong sign or index, a transposed operand)
+fails at least one of them: brute force with independent code on tiny inputs, closed
+forms, invariants, and special cases that reduce to a library routine.
+"""
+import cmath
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2605_16579_b200 import workload
+
+RNG = np.random.default_rng(20260516)
+
+
+def rnd(*shape, scale=1.0):
+    return RNG.standard_normal(shape) * scale
+
+
+def rope_np(x, cos, sin):
+    """Adjacent pairs rotated as a complex product, via torch's complex view (library)."""
+    t = torch.from_numpy(np.ascontiguousarray(x)).double()
+    B, L, H, D = t.shape
+    z = torch.view_as_complex(t.reshape(B, L, H, D // 2, 2).contiguous())
+    rot = torch.complex(torch.from_numpy(cos).double(), torch.from_numpy(sin).double())
+    z = z * rot.view(1, L, 1, D // 2)
+    return torch.view_as_real(z).reshape(B, L, H, D).numpy()
+
+
+def tables(L, D):
+    """Exact float64 cos/sin of 1-D positions (so that cos^2 + sin^2 = 1 to rounding)."""
+    ang = np.arange(L)[:, None] * (10000.0 ** (-2.0 * np.arange(D // 2) / D))[None, :]
+    return np.cos(ang), np.sin(ang)
+
+
+# ----------------------------------------------------------------------------------------
+# A1: intra-block softmax (Eq. 2)
+# ----------------------------------------------------------------------------------------
+
+def brute_force_layer(q, k, v, g, S, wq, cos, sin, scale, eps):
+    """Pure-Python restatement with independent structure: complex numbers for the
+    rotation, naive exp(s)/sum exp(s) without max subtraction, list arithmetic."""
+    B, L, H, D = q.shape
+    out = np.zeros_like(q)
+
+    def rot(vec, pos):
+        res = []
+        for m in range(D // 2):
+            z = complex(vec[2 * m], vec[2 * m + 1]) * complex(cos[pos][m], sin[pos][m])
+            res += [z.real, z.imag]
+        return res
+
+    for b in range(B):
+        for h in range(H):
+            kr = [rot(list(k[b, j, h]), j) for j in range(L)]
+            for i in range(L):
+                qr = rot(list(q[b, i, h]), i)
+                e = [math.exp(scale * sum(x * y for x, y in zip(qr, kr[j]))) for j in range(L)]
+                z = sum(e)
+                o = [sum(e[j] / z * v[b, j, h, d] for j in range(L)) for d in range(D)]
+                u = [sum(q[b, i, h, a] * wq[h, a, c] for a in range(D)) for c in range(D)]
+                u = rot(u, i)
+                n = math.sqrt(sum(x * x for x in u) + eps)
+                u = [x / n for x in u]
+                gate = 1.0 / (1.0 + math.exp(-g[b, i, h]))
+                for c in range(D):
+                    o[c] += gate * sum(u[a] * S[b, h, a, c] for a in range(D))
+                out[b, i, h] = o
+    return out
+
+
+@pytest.mark.parametrize("L,D", [(1, 2), (5, 4), (8, 4)])
+def test_step_brute_force_tiny(oracle, L, D):
+    B, H = 2, 2
+    q, k, v = rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H, D)
+    g, S, wq = rnd(B, L, H), rnd(B, H, D, D), rnd(H, D, D)
+    ang = rnd(L, D // 2)
+    cos, sin = np.cos(ang), np.sin(ang)
+    ref = brute_force_layer(q, k, v, g, S, wq, cos, sin, 0.37, 1e-6)
+    got = oracle.step(q, k, v, g, S, wq, cos, sin, scale=0.37, eps=1e-6)
+    np.testing.assert_allclose(got, ref, rtol=1e-11, atol=1e-12)
+
+
+def test_softmax_matches_library_attention(oracle):
+    """S = 0, no rotation: the layer is textbook attention (first block, Algorithm 1)."""
+    B, L, H, D = 2, 37, 3, 16
+    q, k, v, g = rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H)
+    S = np.zeros((B, H, D, D))
+    got = oracle.step(q, k, v, g, S, rnd(H, D, D))
+    tq, tk, tv = (torch.from_numpy(x).permute(0, 2, 1, 3) for x in (q, k, v))
+    ref = torch.softmax(tq @ tk.transpose(-1, -2) / math.sqrt(D), dim=-1) @ tv
+    np.testing.assert_allclose(got, ref.permute(0, 2, 1, 3).numpy(), rtol=1e-11, atol=1e-13)
+
+
+def test_softmax_with_rope_matches_library(oracle):
+    B, L, H, D = 1, 29, 2, 8
+    q, k, v, g = rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H)
+    cos, sin = tables(L, D)
+    got = oracle.step(q, k, v, g, np.zeros((B, H, D, D)), None, cos, sin)
+    tq, tk = (torch.from_numpy(rope_np(x, cos, sin)).permute(0, 2, 1, 3) for x in (q, k))
+    tv = torch.from_numpy(v).permute(0, 2, 1, 3)
+    ref = torch.softmax(tq @ tk.transpose(-1, -2) / math.sqrt(D), dim=-1) @ tv
+    np.testing.assert_allclose(got, ref.permute(0, 2, 1, 3).numpy(), rtol=1e-11, atol=1e-13)
+
+
+def test_zero_query_gives_column_mean(oracle):
+    B, L, H, D = 1, 23, 2, 8
+    k, v = rnd(B, L, H, D), rnd(B, L, H, D)
+    cos, sin = tables(L, D)
+    got = oracle.step(np.zeros((B, L, H, D)), k, v, rnd(B, L, H), np.zeros((B, H, D, D)),
+                      None, cos, sin, eps=1e-6)
+    ref = np.broadcast_to(v.mean(axis=1, keepdims=True), v.shape)
+    np.testing.assert_allclose(got, ref, rtol=1e-12, atol=1e-13)
+
+
+def test_key_shift_invariance(oracle):
+    B, L, H, D = 1, 19, 2, 8
+    q, k, v, g = rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H)
+    S = np.zeros((B, H, D, D))
+    c = rnd(1, 1, H, D)
+    a = oracle.step(q, k, v, g, S)
+    b = oracle.step(q, k + c, v, g, S)
+    np.testing.assert_allclose(a, b, rtol=1e-10, atol=1e-12)
+
+
+def test_large_scores_do_not_overflow(oracle):
+    """Max subtraction: scores of +-800 would overflow a naive exp."""
+    B, L, H, D = 1, 6, 1, 4
+    q = rnd(B, L, H, D) * 40
+    k = rnd(B, L, H, D) * 40
+    v = rnd(B, L, H, D)
+    out = oracle.step(q, k, v, rnd(B, L, H), np.zeros((B, H, D, D)), scale=1.0)
+    assert np.isfinite(out).all()
+    assert (out.min(axis=1) >= v.min(axis=1) - 1e-12).all()
+    assert (out.max(axis=1) <= v.max(axis=1) + 1e-12).all()
+
+
+# ----------------------------------------------------------------------------------------
+# A2: feature maps (Eq. 3)
+# ----------------------------------------------------------------------------------------
+
+def test_feature_map_against_library_ops(oracle):
+    B, L, H, D = 2, 11, 3, 8
+    x, W = rnd(B, L, H, D), rnd(H, D, D)
+    cos, sin = tables(L, D)
+    got = oracle.feature(x, W, cos, sin, 1e-6, 0)
+    u = torch.einsum("blhi,hio->blho", torch.from_numpy(x), torch.from_numpy(W)).numpy()
+    u = rope_np(u, cos, sin)
+    ref = u / np.sqrt((u * u).sum(-1, keepdims=True) + 1e-6)
+    np.testing.assert_allclose(got, ref, rtol=1e-12, atol=1e-14)
+    got_v = oracle.feature(x, W, cos, sin, 1e-6, 1)
+    ref_v = torch.einsum("blhi,hio->blho", torch.from_numpy(x), torch.from_numpy(W)).numpy()
+    np.testing.assert_allclose(got_v, ref_v, rtol=1e-12, atol=1e-14)
+
+
+def test_feature_unit_norm_and_commutation(oracle):
+    B, L, H, D = 1, 13, 2, 16
+    x, W = rnd(B, L, H, D), rnd(H, D, D)
+    cos, sin = tables(L, D)
+    y = oracle.feature(x, W, cos, sin, 0.0, 0)
+    np.testing.assert_allclose((y * y).sum(-1), 1.0, rtol=1e-12)
+    # rotation preserves the norm, so normalising before or after it is the same
+    y_nr = oracle.feature(x, W, None, None, 0.0, 0)
+    np.testing.assert_allclose(rope_np(y_nr, cos, sin), y, rtol=1e-12, atol=1e-14)
+    # identity map, no rotation: Q' = Q / |Q|
+    y_id = oracle.feature(x, None, None, None, 0.0, 0)
+    np.testing.assert_allclose(y_id, x / np.linalg.norm(x, axis=-1, keepdims=True), rtol=1e-12)
+    # identity tables (angle 0) are a no-op
+    y_0 = oracle.feature(x, W, np.ones((L, D // 2)), np.zeros((L, D // 2)), 0.0, 0)
+    np.testing.assert_allclose(y_0, y_nr, rtol=1e-13)
+
+
+def test_rope_quarter_turn(oracle):
+    """A rotation by 90 degrees sends (x0, x1) to (-x1, x0): fixes the sign convention."""
+    B, L, H, D = 1, 2, 1, 4
+    x = rnd(B, L, H, D)
+    y = oracle.feature(x, None, np.zeros((L, 2)), np.ones((L, 2)), 0.0, 0)
+    n = np.linalg.norm(x, axis=-1, keepdims=True)
+    ref = np.stack([-x[..., 1], x[..., 0], -x[..., 3], x[..., 2]], axis=-1) / n
+    np.testing.assert_allclose(y, ref, rtol=1e-13)
+
+
+# ----------------------------------------------------------------------------------------
+# A3 / A4: frame-level readout and the gated combination (Eq. 5-8)
+# ----------------------------------------------------------------------------------------
+
+def test_zero_values_isolate_inter_branch(oracle):
+    B, L, H, D = 2, 9, 2, 8
+    q, k, g, S, wq = rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H), rnd(B, H, D, D), rnd(H, D, D)
+    cos, sin = tables(L, D)
+    got = oracle.step(q, k, np.zeros((B, L, H, D)), g, S, wq, cos, sin)
+    qf = oracle.feature(q, wq, cos, sin, 1e-6, 0)
+    ref = torch.einsum("blhd,bhde->blhe", torch.from_numpy(qf), torch.from_numpy(S)).numpy()
+    ref = ref / (1.0 + np.exp(-g))[..., None]
+    np.testing.assert_allclose(got, ref, rtol=1e-11, atol=1e-13)
+    # positive rescaling of Q leaves Q' (eps = 0) and hence the readout unchanged
+    a = oracle.step(q, k, np.zeros((B, L, H, D)), g, S, wq, cos, sin, eps=0.0)
+    b = oracle.step(3.7 * q, k, np.zeros((B, L, H, D)), g, S, wq, cos, sin, eps=0.0)
+    np.testing.assert_allclose(a, b, rtol=1e-11, atol=1e-13)
+
+
+def test_closed_gate_and_linearity_in_state(oracle):
+    B, L, H, D = 1, 10, 2, 8
+    q, k, v, g = rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H)
+    S1, S2, wq = rnd(B, H, D, D), rnd(B, H, D, D), rnd(H, D, D)
+    zero = np.zeros_like(S1)
+    intra = oracle.step(q, k, v, g, zero, wq)
+    shut = oracle.step(q, k, v, np.full_like(g, -800.0), S1, wq)
+    np.testing.assert_allclose(shut, intra, rtol=1e-13, atol=1e-15)
+    o1 = oracle.step(q, k, v, g, S1, wq) - intra
+    o2 = oracle.step(q, k, v, g, S2, wq) - intra
+    o12 = oracle.step(q, k, v, g, 2.0 * S1 - 0.5 * S2, wq) - intra
+    np.testing.assert_allclose(o12, 2.0 * o1 - 0.5 * o2, rtol=1e-9, atol=1e-12)
+
+
+def test_token_order_equivariance(oracle):
+    """All tokens read the same pre-update state (Eq. 8): permuting the block's tokens
+    permutes the outputs and leaves the committed state unchanged."""
+    B, L, H, D = 2, 21, 2, 8
+    q, k, v, g = rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H)
+    S, a = rnd(B, H, D, D), rnd(B, H)
+    wq, wk, wv = rnd(H, D, D), rnd(H, D, D), rnd(H, D, D)
+    cos, sin = tables(L, D)
+    perm = RNG.permutation(L)
+    o = oracle.step(q, k, v, g, S, wq, cos, sin)
+    op = oracle.step(q[:, perm], k[:, perm], v[:, perm], g[:, perm], S, wq, cos[perm], sin[perm])
+    np.testing.assert_allclose(op, o[:, perm], rtol=1e-10, atol=1e-12)
+    s = oracle.commit(k, v, a, S, wk, wv, cos, sin)
+    sp = oracle.commit(k[:, perm], v[:, perm], a, S, wk, wv, cos[perm], sin[perm])
+    np.testing.assert_allclose(sp, s, rtol=1e-12, atol=1e-12)
+
+
+def test_step_never_writes_state(oracle):
+    B, L, H, D = 1, 12, 2, 8
+    S = rnd(B, H, D, D)
+    keep = S.copy()
+    for n in range(7):
+        oracle.step(rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H), S,
+                    rnd(H, D, D))
+        assert S.tobytes() == keep.tobytes()
+
+
+# ----------------------------------------------------------------------------------------
+# A6 / A7: commit and reset
+# ----------------------------------------------------------------------------------------
+
+def test_commit_against_library_ops(oracle):
+    B, L, H, D = 2, 17, 3, 8
+    kc, vc, a, S = rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, H), rnd(B, H, D, D)
+    wk, wv = rnd(H, D, D), rnd(H, D, D)
+    cos, sin = tables(L, D)
+    got = oracle.commit(kc, vc, a, S, wk, wv, cos, sin)
+    kf = torch.from_numpy(oracle.feature(kc, wk, cos, sin, 1e-6, 0))
+    vf = torch.from_numpy(oracle.feature(vc, wv, cos, sin, 1e-6, 1))
+    alpha = 1.0 / (1.0 + np.exp(-a))
+    ref = alpha[..., None, None] * S + torch.einsum("blhd,blhe->bhde", kf, vf).numpy()
+    np.testing.assert_allclose(got, ref, rtol=1e-11, atol=1e-13)
+    # subset of heads: the others stay as they were
+    part = oracle.commit(kc, vc, a, S, wk, wv, cos, sin, heads=[(1, 2), (0, 0)])
+    np.testing.assert_allclose(part[1, 2], ref[1, 2], rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(part[0, 0], ref[0, 0], rtol=1e-11, atol=1e-13)
+    assert part[0, 1].tobytes() == S[0, 1].tobytes()
+
+
+def test_commit_closed_form_over_blocks(oracle):
+    """S_T = (prod alpha) S_0 + sum_t (prod_{s>t} alpha_s) K'_t^T V'_t."""
+    B, L, H, D, T = 1, 9, 2, 8, 6
+    wk, wv = rnd(H, D, D), rnd(H, D, D)
+    cos, sin = tables(L, D)
+    S0 = rnd(B, H, D, D)
+    ks, vs, as_ = [rnd(B, L, H, D) for _ in range(T)], [rnd(B, L, H, D) for _ in range(T)], \
+        [rnd(B, H) + 2.0 for _ in range(T)]
+    S = S0
+    for t in range(T):
+        S = oracle.commit(ks[t], vs[t], as_[t], S, wk, wv, cos, sin)
+    alphas = [1.0 / (1.0 + np.exp(-x)) for x in as_]
+    ref = np.prod(alphas, axis=0)[..., None, None] * S0
+    for t in range(T):
+        kf = torch.from_numpy(oracle.feature(ks[t], wk, cos, sin, 1e-6, 0))
+        vf = torch.from_numpy(oracle.feature(vs[t], wv, cos, sin, 1e-6, 1))
+        w = np.ones((B, H))
+        for s in range(t + 1, T):
+            w = w * alphas[s]
+        ref = ref + w[..., None, None] * torch.einsum("blhd,blhe->bhde", kf, vf).numpy()
+    np.testing.assert_allclose(S, ref, rtol=1e-11, atol=1e-12)
+
+
+def orthonormal_keys(B, L, H, D):
+    k = np.empty((B, L, H, D))
+    for b in range(B):
+        for h in range(H):
+            qmat, _ = np.linalg.qr(rnd(D, D))
+            k[b, :, h, :] = qmat[:, :L].T
+    return k
+
+
+@pytest.mark.parametrize("rule", [0, 1, 2])
+def test_associative_memory(oracle, rule):
+    """alpha = 1, orthonormal keys, empty state: reading with key j returns value j."""
+    B, L, H, D = 1, 6, 2, 8
+    k, v = orthonormal_keys(B, L, H, D), rnd(B, L, H, D)
+    a = np.full((B, H), 800.0)                  # sigmoid -> exactly 1
+    beta = np.full((B, L, H), 800.0)
+    S = oracle.commit(k, v, a, np.zeros((B, H, D, D)), eps=0.0, rule=rule, beta_logit=beta)
+    out = oracle.step(k, k, np.zeros_like(v), np.full((B, L, H), 800.0), S, eps=0.0)
+    np.testing.assert_allclose(out, v, rtol=1e-10, atol=1e-12)
+
+
+def test_delta_rules_overwrite_and_coincide(oracle):
+    """Eq. 4 with orthonormal keys and alpha = beta = 1 replaces what the state held for
+    those keys (K' S_new = V'), and the frame-level and token-sequential forms agree."""
+    B, L, H, D = 1, 5, 2, 8
+    k, v = orthonormal_keys(B, L, H, D), rnd(B, L, H, D)
+    S0 = rnd(B, H, D, D)
+    one, beta = np.full((B, H), 800.0), np.full((B, L, H), 800.0)
+    s1 = oracle.commit(k, v, one, S0, eps=0.0, rule=1, beta_logit=beta)
+    s2 = oracle.commit(k, v, one, S0, eps=0.0, rule=2, beta_logit=beta)
+    np.testing.assert_allclose(s1, s2, rtol=1e-10, atol=1e-12)
+    read = torch.einsum("blhd,bhde->blhe", torch.from_numpy(k), torch.from_numpy(s1)).numpy()
+    np.testing.assert_allclose(read, v, rtol=1e-10, atol=1e-12)
+    # with an empty state and beta = 1 the correction term vanishes at frame level
+    a = rnd(B, H)
+    kk, vv = rnd(B, L, H, D), rnd(B, L, H, D)
+    r0 = oracle.commit(kk, vv, a, np.zeros_like(S0), rule=0)
+    r1 = oracle.commit(kk, vv, a, np.zeros_like(S0), rule=1, beta_logit=beta)
+    np.testing.assert_allclose(r0, r1, rtol=1e-12, atol=1e-14)
+    # frame-level Eq. 4 against library ops, general keys, decay and learning rates
+    a, bl = rnd(B, H), rnd(B, L, H)
+    got = oracle.commit(kk, vv, a, S0, rule=1, beta_logit=bl)
+    kf = torch.from_numpy(oracle.feature(kk, None, None, None, 1e-6, 0))
+    tv, tS = torch.from_numpy(vv), torch.from_numpy(S0)
+    resid = tv - torch.einsum("blhd,bhde->blhe", kf, tS)
+    resid = resid * torch.from_numpy(1.0 / (1.0 + np.exp(-bl)))[..., None]
+    ref = torch.from_numpy(1.0 / (1.0 + np.exp(-a)))[..., None, None] * tS \
+        + torch.einsum("blhd,blhe->bhde", kf, resid)
+    np.testing.assert_allclose(got, ref.numpy(), rtol=1e-11, atol=1e-13)
+
+
+def test_state_norm_stays_bounded(oracle):
+    """Unit-norm keys and alpha <= alpha_max < 1: |S_T|_F <= max_t |K'^T V'|_F / (1 - alpha_max)."""
+    B, L, H, D, T = 1, 12, 2, 8, 60
+    S = np.zeros((B, H, D, D))
+    amax = 1.0 / (1.0 + math.exp(-2.5))
+    bound = 0.0
+    norms = []
+    for t in range(T):
+        k, v = rnd(B, L, H, D), rnd(B, L, H, D)
+        a = np.minimum(rnd(B, H) * 0.5 + 2.0, 2.5)
+        delta = oracle.commit(k, v, np.full((B, H), -800.0), np.zeros_like(S))
+        bound = max(bound, np.sqrt((delta ** 2).sum(axis=(-1, -2))).max())
+        S = oracle.commit(k, v, a, S)
+        norms.append(np.sqrt((S ** 2).sum(axis=(-1, -2))).max())
+    assert max(norms) <= bound / (1.0 - amax)
+    assert max(norms[T // 2:]) < 1.5 * max(norms[: T // 2])   # flat, not growing with T
+
+
+def test_reset(oracle):
+    S = rnd(3, 2, 4, 4)
+    r = oracle.reset(S, 1)
+    assert (r[1] == 0).all() and r[0].tobytes() == S[0].tobytes() and r[2].tobytes() == S[2].tobytes()
+    assert (oracle.reset(S) == 0).all()
+
+
+def test_step_rows_matches_full_step(oracle):
+    cfg = workload.custom(B=2, H=3, D=8, L=40)
+    q, k, v, g = workload.step_inputs(cfg, 0, 0)
+    S, wq = rnd(2, 3, 8, 8), rnd(3, 8, 8)
+    cos, sin = tables(40, 8)
+    full = oracle.step(q, k, v, g, S, wq, cos, sin)
+    rows = [(0, 0, 0), (1, 2, 39), (0, 1, 17), (1, 0, 5)]
+    got = oracle.step_rows(q, k, v, g, S, rows, wq, cos, sin)
+    for r, (b, h, i) in enumerate(rows):
+        assert got[r].tobytes() == full[b, i, h].tobytes()
+
+
+def test_golden_fixture_regression(oracle):
+    """The stored tiny case (written by tests/golden/make_golden.py from the oracle alone)."""
+    import json
+    import os
+
+    with open(os.path.join(os.path.dirname(__file__), "golden", "tiny_layer.json")) as f:
+        doc = json.load(f)
+    A = lambda key: np.array(doc[key], dtype=np.float64)  # noqa: E731
+    cos, sin = np.cos(A("angle")), np.sin(A("angle"))
+    out = oracle.step(A("q"), A("k"), A("v"), A("g"), A("S0"), A("wq"), cos, sin, eps=doc["eps"])
+    S1 = oracle.commit(A("kc"), A("vc"), A("a"), A("S0"), A("wk"), A("wv"), cos, sin,
+                       eps=doc["eps"])
+    np.testing.assert_allclose(out, A("out"), rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(S1, A("S1"), rtol=1e-13, atol=1e-15)
+    # and the same case through the independent pure-Python restatement
+    ref = brute_force_layer(A("q"), A("k"), A("v"), A("g"), A("S0"), A("wq"), cos, sin,
+                            1.0 / math.sqrt(doc["D"]), doc["eps"])
+    np.testing.assert_allclose(A("out"), ref, rtol=1e-11, atol=1e-13)
