@@ -1,0 +1,396 @@
+"""Benchmark of the ARL^2 hybrid attention layer on B200.
+
+A bench "step" is one autoregressive block of the layer's whole hot path: `n_steps` denoise
+passes (intra-block softmax + state readout + gated combine, the state only read) followed by
+one state commit.  The metric is tokens per second through the denoise passes, with the commit
+time included:  value = N_gpus * B * L * n_steps / t_block.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload long] [--impl reference]
+
+N > 1 is launched by torchrun, one rank per GPU.  The layer shards by (stream, head) with no
+exchange inside it, so ranks are independent replicas ("weak" scaling); torch.distributed is
+used only for the barrier and the max-over-ranks of the device time.
+
+`--impl reference` times the CPU float64 checker (as it stands) on the host cores, on bounded
+samples of the same workload, and prints the same JSON line with "impl": "reference".
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "hybrid-attn layer tokens/s per denoise step"
+UNIT = "tokens/s"
+RING = 3  # pre-generated step-input sets the timed loop rotates through
+
+
+def peaks():
+    """Measured roofline denominators of this machine's B200s, else the stated fallback."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+            "source": "fallback"}
+
+
+def workload_text(cfg):
+    return (f"{cfg.name}: B={cfg.B} H={cfg.H} D={cfg.D} L={cfg.L} {cfg.dtype}, "
+            f"{cfg.steps} denoise steps + 1 commit per block")
+
+
+def step_flops(cfg):
+    """Algorithmic tensor flops of one denoise pass: QK^T, PV, Q W_phi_q, Q' S."""
+    return cfg.B * cfg.H * (4.0 * cfg.L * cfg.L * cfg.D + 4.0 * cfg.L * cfg.D * cfg.D)
+
+
+def step_bytes(cfg):
+    """Algorithmic HBM bytes of one denoise pass: Q, K, V in, O out, gate logits, S and W_phi_q."""
+    e = cfg.elem_bytes
+    return cfg.B * cfg.H * (4.0 * cfg.L * cfg.D * e + 4.0 * cfg.L + cfg.D * cfg.D * (4 + e))
+
+
+class ClockSampler:
+    """nvidia-smi in the background during the timed region (read-only queries)."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc, self.index = None, index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "50", "-i", str(self.index)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, power, reasons = [], [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for n, val in zip(names, parts[3:7]):
+                if val.lower() == "active":
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "samples": len(sm),
+                "power_w_max": max(power), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------
+# CPU checker timings (the "reference arm" of this tier and the cpu_baseline leg)
+# ------------------------------------------------------------------------------------------
+
+class CpuSample:
+    """Times the CPU float64 checker on a bounded sample of one block of `cfg`."""
+
+    def __init__(self, cfg):
+        import numpy as np
+
+        from oracle import arl2_oracle
+        from paper_2605_16579_b200 import workload
+
+        self.np, self.o, self.cfg = np, arl2_oracle, cfg
+        self.threads = arl2_oracle.threads()
+        f64 = lambda t: None if t is None else t.double().numpy()  # noqa: E731
+        q, k, v, g = workload.step_inputs(cfg, 0, 0)
+        kc, vc, a = workload.commit_inputs(cfg, 0)
+        self.q, self.k, self.v, self.g = f64(q), f64(k), f64(v), f64(g)
+        self.kc, self.vc, self.a = f64(kc), f64(vc), f64(a)
+        wq, wk, wv = workload.feature_weights(cfg)
+        cos, sin = workload.rope_tables(cfg.L, cfg.D)
+        self.wq, self.wk, self.wv, self.cos, self.sin = f64(wq), f64(wk), f64(wv), f64(cos), f64(sin)
+        rng = np.random.default_rng(1)
+        self.S = rng.standard_normal((cfg.B, cfg.H, cfg.D, cfg.D)) * 0.1
+        self.rng = rng
+
+    def time_rows(self, n):
+        cfg, np = self.cfg, self.np
+        rows = np.stack([self.rng.integers(0, cfg.B, n), self.rng.integers(0, cfg.H, n),
+                         self.rng.integers(0, cfg.L, n)], axis=1)
+        t0 = time.perf_counter()
+        self.o.step_rows(self.q, self.k, self.v, self.g, self.S, rows, self.wq, self.cos, self.sin)
+        return time.perf_counter() - t0
+
+    def time_heads(self, n):
+        cfg = self.cfg
+        heads = [((i // cfg.H) % cfg.B, i % cfg.H) for i in range(n)]
+        t0 = time.perf_counter()
+        self.o.commit(self.kc, self.vc, self.a, self.S, self.wk, self.wv, self.cos, self.sin,
+                      heads=heads)
+        return time.perf_counter() - t0
+
+    def block_seconds(self, n_rows, t_rows, n_heads, t_heads):
+        """Extrapolate one block (n_steps denoise passes + commit) from the sample rates."""
+        cfg = self.cfg
+        rows_per_step = cfg.B * cfg.L * cfg.H
+        return cfg.steps * rows_per_step * (t_rows / n_rows) + cfg.B * cfg.H * (t_heads / n_heads)
+
+
+def run_reference(args):
+    from paper_2605_16579_b200 import workload
+
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = workload.CONFIGS[args.workload]
+    s = CpuSample(cfg)
+    target = min(1.0, 150.0 / max(args.steps + args.warmup, 1))  # seconds of CPU work per step
+    t = s.time_rows(s.threads)  # calibration
+    n_rows = max(s.threads, int(s.threads * (0.8 * target) / max(t, 1e-6)))
+    n_heads = 1 if s.time_heads(1) > 0.2 * target else min(s.threads, cfg.B * cfg.H)
+    for _ in range(args.warmup):
+        s.time_rows(n_rows)
+    per_step, est = [], []
+    for _ in range(args.steps):
+        tr = s.time_rows(n_rows)
+        th = s.time_heads(n_heads)
+        per_step.append(tr + th)
+        est.append(s.block_seconds(n_rows, tr, n_heads, th))
+    block_s = statistics.mean(est)
+    value = cfg.B * cfg.L * cfg.steps / block_s
+    sample = (f"per step: {n_rows} random output rows (b,h,i) of one denoise pass + commit of "
+              f"{n_heads} head(s), extrapolated to {cfg.steps} passes over B*L*H = "
+              f"{cfg.B * cfg.L * cfg.H} rows and {cfg.B * cfg.H} heads")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * statistics.mean(per_step), "extrapolated_block_ms": 1e3 * block_s,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": workload_text(cfg)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": s.threads, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------
+# the CUDA arm
+# ------------------------------------------------------------------------------------------
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2605_16579_b200 import arl2, workload
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the layer has no CPU path")
+    arl2.load(build_if_missing=True)
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg = workload.CONFIGS[args.workload]
+    layer = arl2.Layer(cfg.B, cfg.H, cfg.L, cfg.D, cfg.dtype, device=dev)
+    wq, wk, wv = (w.to(dev) for w in workload.feature_weights(cfg))
+    cos, sin = (t.to(dev) for t in workload.rope_tables(cfg.L, cfg.D))
+    layer.set_params(wq, wk, wv, cos, sin)
+
+    host_sets = [workload.step_inputs(cfg, 0, s + 10 * rank) for s in range(RING)]
+    host_commit = workload.commit_inputs(cfg, rank)
+    dev_sets = [tuple(t.to(dev) for t in hs) for hs in host_sets]
+    dev_commit = tuple(t.to(dev) for t in host_commit)
+    out = torch.empty(cfg.B, cfg.L, cfg.H, cfg.D, dtype=cfg.torch_dtype, device=dev)
+    set_bytes = sum(t.numel() * t.element_size() for t in host_sets[0])
+
+    step_events = []
+
+    def block(i, timed):
+        for s in range(cfg.steps):
+            q, k, v, g = dev_sets[(i * cfg.steps + s) % RING]
+            if timed:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                layer.set_profile_events(e0, e1)
+                step_events.append((e0, e1))
+            layer.denoise_step(q, k, v, g, out=out)
+        layer.commit(*dev_commit)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        block(i, False)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = layer.launch_count
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for i in range(args.steps):
+        block(i, True)
+    t1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    launches = layer.launch_count - launches0
+    ms_total = t0.elapsed_time(t1)
+    kern_ms = [a.elapsed_time(b) for a, b in step_events]
+    layer.sync_status()
+
+    # end to end through the same entry points with HOST buffers: every pass copies its inputs
+    # from pinned host memory and its output back inside the timed region
+    e2e_blocks = max(1, min(args.steps, 5))
+    pin_sets = [tuple(t.pin_memory() for t in hs) for hs in host_sets]
+    pin_commit = tuple(t.pin_memory() for t in host_commit)
+    pin_out = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+    stage = tuple(torch.empty_like(t) for t in dev_sets[0])
+    stage_c = tuple(torch.empty_like(t) for t in dev_commit)
+
+    def block_host(i):
+        for s in range(cfg.steps):
+            for d, h in zip(stage, pin_sets[(i * cfg.steps + s) % RING]):
+                d.copy_(h, non_blocking=True)
+            layer.denoise_step(*stage, out=out)
+            pin_out.copy_(out, non_blocking=True)
+        for d, h in zip(stage_c, pin_commit):
+            d.copy_(h, non_blocking=True)
+        layer.commit(*stage_c)
+
+    block_host(0)
+    barrier()
+    h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    h0.record()
+    for i in range(e2e_blocks):
+        block_host(i)
+    h1.record()
+    barrier()
+    ms_e2e = h0.elapsed_time(h1)
+    commit_bytes = sum(t.numel() * t.element_size() for t in host_commit)
+    h2d = cfg.steps * set_bytes + commit_bytes
+    d2h = cfg.steps * out.numel() * out.element_size()
+
+    if world > 1:
+        t = torch.tensor([ms_total, ms_e2e, statistics.mean(kern_ms)], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, ms_e2e, kern_mean = (float(x) for x in t.tolist())
+    else:
+        kern_mean = statistics.mean(kern_ms)
+
+    if rank == 0:
+        pk = peaks()
+        tokens_per_block = world * cfg.B * cfg.L * cfg.steps
+        ms_block = ms_total / args.steps
+        value = tokens_per_block / (ms_block * 1e-3)
+        timed_seconds = ms_total * 1e-3
+        # a kernel timed inside a seconds-long loop runs under the power cap: sustained figure
+        use_sustained = timed_seconds > 1.0
+        peak = pk["bf16_tflops_sustained"] if use_sustained else pk["bf16_tflops"]
+        achieved = step_flops(cfg) / (kern_mean * 1e-3) / 1e12
+        traffic = None
+        tpath = os.path.join(ROOT, "profiles", "step_kernel_traffic.json")
+        if os.path.exists(tpath):
+            with open(tpath) as f:
+                rec = json.load(f)
+            if rec.get("step_kernel") == layer.step_kernel:
+                # DRAM bytes of the captured (smaller) case scaled by the (stream, head) count
+                traffic = rec["dram_bytes_per_head"] * cfg.B * cfg.H
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_block, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
+            "data": "synthetic",
+            "config": {
+                "workload": workload_text(cfg),
+                "step_definition": "one AR block = n_steps denoise passes + 1 state commit",
+                "l2": f"inputs larger than L2: ring of {RING} input sets of {set_bytes >> 20} MiB",
+                "parallelism": "replicas" if world > 1 else "single GPU",
+                "step_kernel": layer.step_kernel,
+            },
+            "denoise_pass": {"kernel_ms_mean": kern_mean, "kernel_ms_median": statistics.median(kern_ms),
+                             "tokens_per_s": cfg.B * cfg.L / (kern_mean * 1e-3)},
+            "roofline": {
+                "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "traffic": traffic,
+                "peak_kind": ("sustained" if use_sustained else "burst") + " bf16, " + pk["source"],
+                "frac_of_burst": achieved / pk["bf16_tflops"],
+                "algorithmic_flops_per_launch": step_flops(cfg),
+                "algorithmic_bytes_per_launch": step_bytes(cfg),
+                "hbm_frac": step_bytes(cfg) / (kern_mean * 1e-3) / 1e9 / pk["hbm_gbs"],
+            },
+            "e2e": {"value": world * cfg.B * cfg.L * cfg.steps * e2e_blocks / (ms_e2e * 1e-3),
+                    "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "blocks_timed": e2e_blocks},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            s = CpuSample(cfg)
+            t = s.time_rows(s.threads)
+            n_rows = max(s.threads, int(s.threads * 12.0 / max(t, 1e-6)))
+            tr = s.time_rows(n_rows)
+            n_heads = min(s.threads, cfg.B * cfg.H)
+            th = s.time_heads(n_heads)
+            block_s = s.block_seconds(n_rows, tr, n_heads, th)
+            line["cpu_baseline"] = {
+                "value": cfg.B * cfg.L * cfg.steps / block_s, "unit": UNIT, "cores": s.threads,
+                "kind": "oracle",
+                "sample": (f"{n_rows} random output rows of one denoise pass ({tr:.1f} s) and the "
+                           f"commit of {n_heads} heads ({th:.1f} s), extrapolated to one block"),
+            }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="long", choices=["tiny", "small", "chunked", "batched", "long"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,172 @@
+/*
+ * arl2.h -- C ABI of the ARL^2 hybrid attention layer for NVIDIA B200 (sm_100a).
+ *
+ * The layer is the attention core that an autoregressive video-diffusion model runs at
+ * every denoising step of every block (paper Sec. 3.2-3.3, Algorithm 1):
+ *
+ *   O_intra = Softmax(RoPE(Q), RoPE(K), V)          over the block's L tokens   (Eq. 2)
+ *   Q'      = L2Norm(RoPE(phi_q(Q)))                                            (Eq. 3)
+ *   O_inter = Q' S                                   same pre-update S for all   (Eq. 5, 8)
+ *   O       = O_intra + sigmoid(g) (.) O_inter       headwise gate               (Eq. 6-7)
+ *   S      <- sigmoid(a) S + K'^T V'                 once per block, clean pass  (Eq. 4, Sec. 3.3)
+ *
+ * Conventions shared by every call
+ *   - All `d_*` pointers are DEVICE pointers owned by the caller; the library never
+ *     allocates or frees device memory and keeps only the pointers it is given
+ *     (state, workspace, parameters) until arl2_destroy.
+ *   - Tensors are contiguous.  Q, K, V, O: [B, L, H, D] (token-major).  State S:
+ *     [B, H, D, D] fp32, row = key dimension, column = value dimension.  Combine-gate
+ *     logits g: [B, L, H] fp32.  Decay logits a: [B, H] fp32.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls are
+ *     asynchronous on it; ordering between calls is stream order.
+ *   - Every function returns an arl2_status (0 = ok, negative = error).  Argument errors
+ *     are found on the host before any launch and leave S untouched.  Nothing aborts,
+ *     traps or throws.  arl2_last_error() gives a thread-local message for the last error.
+ *   - A context is not thread-safe; distinct contexts are independent.
+ */
+#ifndef ARL2_H
+#define ARL2_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct arl2_ctx arl2_ctx; /* opaque, host memory owned by the library */
+
+typedef enum {
+    ARL2_OK = 0,
+    ARL2_ERR_INVALID_ARG = -1, /* NULL pointer, bad size, bad struct_size ...              */
+    ARL2_ERR_UNSUPPORTED = -2, /* shape / dtype combination with no kernel                  */
+    ARL2_ERR_CUDA = -3,        /* a CUDA runtime or driver call failed                      */
+    ARL2_ERR_TIMEOUT = -4,     /* a bounded wait inside a kernel expired (device status)    */
+    ARL2_ERR_WORKSPACE = -5    /* workspace too small or misaligned                         */
+} arl2_status;
+
+typedef enum {
+    ARL2_BF16 = 0, /* bf16 inputs/outputs, tensor-core contractions, fp32 accumulation      */
+    ARL2_FP32 = 1  /* fp32 inputs/outputs, fp32 FMA arithmetic end to end (the 1e-4 mode)   */
+} arl2_dtype;
+
+/* arl2_config.flags */
+#define ARL2_FLAG_FORCE_SIMT 1u /* bf16 I/O through the plain-FMA kernels (debug / A-B checks) */
+
+typedef struct {
+    uint32_t struct_size; /* sizeof(arl2_config), for versioning                            */
+    int32_t B;            /* independent streams (videos), >= 1                             */
+    int32_t H;            /* heads, >= 1                                                    */
+    int32_t L;            /* tokens per autoregressive block, >= 1, any value               */
+    int32_t D;            /* head dimension: 64 or 128                                      */
+    int32_t io_dtype;     /* arl2_dtype of Q, K, V, O and of the feature-map weights        */
+    float softmax_scale;  /* 0 -> 1/sqrt(D) (Eq. 1)                                         */
+    float l2_eps;         /* epsilon inside the root of L2Norm; 0 -> 1e-6                   */
+    int32_t commit_rule;  /* 0 = gated linear S <- alpha S + K'^T V'; others reserved       */
+    uint32_t flags;       /* ARL2_FLAG_*                                                    */
+} arl2_config;
+
+/*
+ * Bytes of device scratch a context of this shape needs (256-byte aligned base).  It
+ * holds a status word, the rotated copy of K made once per step, tensor-core operand
+ * copies of S and of the feature maps, and the partial sums of the commit reduction.
+ * Returns 0 for an invalid configuration.
+ */
+size_t arl2_workspace_bytes(const arl2_config* cfg);
+
+/*
+ * Create a context (Algorithm 1: the state lives for one video per stream).
+ *   d_state      [B, H, D, D] fp32, caller-owned; NOT cleared by this call -- call
+ *                arl2_reset, or arl2_set_state to resume from a checkpoint.
+ *   d_workspace  >= arl2_workspace_bytes(cfg) bytes, 256-byte aligned, caller-owned,
+ *                private to this context until arl2_destroy.
+ * Launches one small kernel on `stream` that clears the workspace header.
+ */
+int arl2_create(const arl2_config* cfg, void* d_state, void* d_workspace,
+                size_t workspace_bytes, void* stream, arl2_ctx** out);
+
+/*
+ * Feature maps phi_q, phi_k, phi_v (Eq. 3: per-head grouped 1x1 maps, read here as
+ * bias-free linear maps applied as row-vector times matrix) and the rotary tables.
+ *   d_wphi_*   [H, D, D] indexed [head][in][out], io_dtype; NULL = identity map.
+ *   d_rope_cos, d_rope_sin  [L, D/2] fp32: cos / sin of the angle of pair (2m, 2m+1) at
+ *              token l; both NULL = no rotation.  The same tables serve Q and K and both
+ *              branches.
+ * The pointers are kept; the buffers must stay valid and unchanged until replaced or
+ * the context is destroyed.  On the tensor-core path this call also launches a kernel
+ * that writes operand copies of the maps into the workspace.
+ */
+int arl2_set_params(arl2_ctx* ctx, const void* d_wphi_q, const void* d_wphi_k,
+                    const void* d_wphi_v, const float* d_rope_cos, const float* d_rope_sin,
+                    void* stream);
+
+/*
+ * One denoising pass of the layer (Algorithm 1, inner loop; Eq. 2, 3, 5-8):
+ *   d_out[b,i,h,:] = softmax_j(<RoPE(q_i), RoPE(k_j)> scale) v_j
+ *                    + sigmoid(g[b,i,h]) * L2Norm(RoPE(q_i Wphi_q[h])) S[b,h]
+ * READS the state, never writes it (clean-pass-only update, Sec. 3.3): S is bitwise
+ * unchanged after any number of calls.  d_q, d_k, d_v, d_out: [B, L, H, D] io_dtype;
+ * d_gate_logits: [B, L, H] fp32 (the projection x W_g of Eq. 6).  d_out must not
+ * alias an input.
+ */
+int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const void* d_v,
+                      const float* d_gate_logits, void* d_out, void* stream);
+
+/*
+ * State commit, once per block, from the clean pass's K and V (Algorithm 1, clean-pass
+ * branch; Eq. 4 in its gated-linear form):
+ *   S[b,h] <- sigmoid(a[b,h]) S[b,h] + sum_l K'_l^T V'_l,
+ *   K' = L2Norm(RoPE(k Wphi_k[h])),  V' = v Wphi_v[h].
+ * The ONLY call that changes S besides reset / set_state.  The reduction over tokens
+ * is split across thread blocks and summed in a fixed order: results are bitwise
+ * reproducible.  d_k_clean, d_v_clean: [B, L, H, D] io_dtype; d_decay_logits: [B, H] fp32.
+ */
+int arl2_commit(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
+                const float* d_decay_logits, void* stream);
+
+/* S <- 0 for stream `stream_index` (0..B-1) or all streams (-1): Algorithm 1, first line. */
+int arl2_reset(arl2_ctx* ctx, int32_t stream_index, void* stream);
+
+/*
+ * Checkpoint / resume.  `dst` / `src` hold [B, H, D, D] fp32 and may be host or device
+ * memory (cudaMemcpyDefault).  set_state also refreshes the operand copy of S.
+ */
+int arl2_get_state(arl2_ctx* ctx, float* dst, void* stream);
+int arl2_set_state(arl2_ctx* ctx, const float* src, void* stream);
+
+/*
+ * Synchronise `stream` and return the device status word: ARL2_OK, or ARL2_ERR_TIMEOUT
+ * if a bounded wait inside a kernel expired (the kernel then returned early; its output
+ * is undefined, the context stays usable).  The word is cleared by the call.
+ */
+int arl2_sync_status(arl2_ctx* ctx, void* stream);
+
+/*
+ * Measurement hook (no counterpart in the paper).  `ev_before` / `ev_after` are
+ * cudaEvent_t handles (as void*) or NULL.  While set, the NEXT arl2_denoise_step records
+ * them on its stream immediately before and after its dominant kernel (the fused
+ * attention kernel, not the K rotation pass), then forgets them.  Lets a caller time that
+ * kernel alone without a profiler.
+ */
+int arl2_set_profile_events(arl2_ctx* ctx, void* ev_before, void* ev_after);
+
+/* Number of kernel launches this context has issued so far (all entry points). */
+uint64_t arl2_launch_count(const arl2_ctx* ctx);
+
+/* Which kernel family serves arl2_denoise_step for this context: "tcgen05" or "simt". */
+const char* arl2_step_kernel_name(const arl2_ctx* ctx);
+
+/* Frees the host context only; no device buffer is touched and nothing is synchronised
+   (the caller makes sure its streams are done with the workspace before reusing it). */
+void arl2_destroy(arl2_ctx* ctx);
+
+/* Thread-local message describing the last error returned on this thread ("" if none). */
+const char* arl2_last_error(void);
+
+/* Library version string. */
+const char* arl2_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ARL2_H */

@@ -1,0 +1,238 @@
+"""ctypes binding of ``libarl2.so`` (the C ABI in ``include/arl2.h``), same names.
+
+Argument marshalling only: every step of the layer runs in the library's CUDA kernels.
+PyTorch appears here as the owner of device memory and streams -- tensors are passed as
+``data_ptr()`` and the current CUDA stream as a ``void*``.  There is no fallback: if the
+library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libarl2.so")
+
+ARL2_BF16, ARL2_FP32 = 0, 1
+ARL2_FLAG_FORCE_SIMT = 1
+
+EXPORTS = (
+    "arl2_workspace_bytes", "arl2_create", "arl2_set_params", "arl2_denoise_step", "arl2_commit",
+    "arl2_reset", "arl2_get_state", "arl2_set_state", "arl2_sync_status", "arl2_launch_count",
+    "arl2_set_profile_events",
+    "arl2_step_kernel_name", "arl2_destroy", "arl2_last_error", "arl2_version",
+)
+
+
+class Arl2Error(RuntimeError):
+    pass
+
+
+class arl2_config(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32),
+        ("B", ctypes.c_int32), ("H", ctypes.c_int32), ("L", ctypes.c_int32), ("D", ctypes.c_int32),
+        ("io_dtype", ctypes.c_int32),
+        ("softmax_scale", ctypes.c_float), ("l2_eps", ctypes.c_float),
+        ("commit_rule", ctypes.c_int32), ("flags", ctypes.c_uint32),
+    ]
+
+
+_lib = None
+
+
+def load(build_if_missing: bool = False) -> ctypes.CDLL:
+    """Load the library (once).  Raises Arl2Error when it is absent: there is no CPU path."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if build_if_missing:
+        from . import build as _build
+
+        _build.build_library()
+    if not os.path.exists(LIB_PATH):
+        raise Arl2Error(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2605_16579_b200.build` "
+            "(nvcc, sm_100a).  The layer has no CPU or PyTorch fallback."
+        )
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, cp = ctypes.c_void_p, ctypes.POINTER(arl2_config)
+    lib.arl2_workspace_bytes.restype = ctypes.c_size_t
+    lib.arl2_workspace_bytes.argtypes = [cp]
+    lib.arl2_create.restype = ctypes.c_int
+    lib.arl2_create.argtypes = [cp, vp, vp, ctypes.c_size_t, vp, ctypes.POINTER(vp)]
+    lib.arl2_set_params.restype = ctypes.c_int
+    lib.arl2_set_params.argtypes = [vp] * 7
+    lib.arl2_denoise_step.restype = ctypes.c_int
+    lib.arl2_denoise_step.argtypes = [vp] * 7
+    lib.arl2_commit.restype = ctypes.c_int
+    lib.arl2_commit.argtypes = [vp] * 5
+    lib.arl2_reset.restype = ctypes.c_int
+    lib.arl2_reset.argtypes = [vp, ctypes.c_int32, vp]
+    lib.arl2_get_state.restype = ctypes.c_int
+    lib.arl2_get_state.argtypes = [vp, vp, vp]
+    lib.arl2_set_state.restype = ctypes.c_int
+    lib.arl2_set_state.argtypes = [vp, vp, vp]
+    lib.arl2_sync_status.restype = ctypes.c_int
+    lib.arl2_sync_status.argtypes = [vp, vp]
+    lib.arl2_set_profile_events.restype = ctypes.c_int
+    lib.arl2_set_profile_events.argtypes = [vp, vp, vp]
+    lib.arl2_launch_count.restype = ctypes.c_uint64
+    lib.arl2_launch_count.argtypes = [vp]
+    lib.arl2_step_kernel_name.restype = ctypes.c_char_p
+    lib.arl2_step_kernel_name.argtypes = [vp]
+    lib.arl2_destroy.restype = None
+    lib.arl2_destroy.argtypes = [vp]
+    lib.arl2_last_error.restype = ctypes.c_char_p
+    lib.arl2_version.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def _check(status: int, what: str):
+    if status != 0:
+        msg = load().arl2_last_error().decode()
+        raise Arl2Error(f"{what} failed with status {status}: {msg}")
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def make_config(B, H, L, D, dtype, softmax_scale=0.0, l2_eps=0.0, commit_rule=0, flags=0):
+    io = {"bf16": ARL2_BF16, "fp32": ARL2_FP32, torch.bfloat16: ARL2_BF16,
+          torch.float32: ARL2_FP32}[dtype]
+    return arl2_config(ctypes.sizeof(arl2_config), B, H, L, D, io, softmax_scale, l2_eps,
+                       commit_rule, flags)
+
+
+def arl2_workspace_bytes(cfg: arl2_config) -> int:
+    n = load().arl2_workspace_bytes(ctypes.byref(cfg))
+    if n == 0:
+        raise Arl2Error("arl2_workspace_bytes: " + load().arl2_last_error().decode())
+    return n
+
+
+class Layer:
+    """One context: owns (through torch) the state and workspace buffers it hands to the library.
+
+    Methods mirror the C entry points one to one; tensors must be contiguous CUDA tensors of
+    the configured dtype.
+    """
+
+    def __init__(self, B, H, L, D, dtype="bf16", device="cuda:0", softmax_scale=0.0, l2_eps=0.0,
+                 flags=0):
+        lib = load()
+        self.cfg = make_config(B, H, L, D, dtype, softmax_scale, l2_eps, 0, flags)
+        self.B, self.H, self.L, self.D = B, H, L, D
+        self.device = torch.device(device)
+        self.dtype = torch.bfloat16 if self.cfg.io_dtype == ARL2_BF16 else torch.float32
+        self.workspace_bytes = arl2_workspace_bytes(self.cfg)
+        with torch.cuda.device(self.device):
+            self.state = torch.empty(B, H, D, D, dtype=torch.float32, device=self.device)
+            self.workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8,
+                                         device=self.device)
+            ctx = ctypes.c_void_p()
+            _check(lib.arl2_create(ctypes.byref(self.cfg), _ptr(self.state), _ptr(self.workspace),
+                                   self.workspace_bytes, _stream(), ctypes.byref(ctx)),
+                   "arl2_create")
+        self._ctx = ctx
+        self._params = None  # keeps the parameter tensors alive
+        self.reset()
+
+    # -- the C entry points ------------------------------------------------------------
+    def set_params(self, wq=None, wk=None, wv=None, rope_cos=None, rope_sin=None):
+        for w in (wq, wk, wv):
+            if w is not None:
+                self._want(w, (self.H, self.D, self.D), self.dtype, "feature map")
+        for t in (rope_cos, rope_sin):
+            if t is not None:
+                self._want(t, (self.L, self.D // 2), torch.float32, "rope table")
+        self._params = (wq, wk, wv, rope_cos, rope_sin)
+        with torch.cuda.device(self.device):
+            _check(load().arl2_set_params(self._ctx, _ptr(wq), _ptr(wk), _ptr(wv), _ptr(rope_cos),
+                                          _ptr(rope_sin), _stream()), "arl2_set_params")
+
+    def denoise_step(self, q, k, v, gate_logits, out=None):
+        shape = (self.B, self.L, self.H, self.D)
+        for t in (q, k, v):
+            self._want(t, shape, self.dtype, "q/k/v")
+        self._want(gate_logits, (self.B, self.L, self.H), torch.float32, "gate_logits")
+        if out is None:
+            out = torch.empty(shape, dtype=self.dtype, device=self.device)
+        else:
+            self._want(out, shape, self.dtype, "out")
+        with torch.cuda.device(self.device):
+            _check(load().arl2_denoise_step(self._ctx, _ptr(q), _ptr(k), _ptr(v), _ptr(gate_logits),
+                                            _ptr(out), _stream()), "arl2_denoise_step")
+        return out
+
+    def commit(self, k_clean, v_clean, decay_logits):
+        shape = (self.B, self.L, self.H, self.D)
+        self._want(k_clean, shape, self.dtype, "k_clean")
+        self._want(v_clean, shape, self.dtype, "v_clean")
+        self._want(decay_logits, (self.B, self.H), torch.float32, "decay_logits")
+        with torch.cuda.device(self.device):
+            _check(load().arl2_commit(self._ctx, _ptr(k_clean), _ptr(v_clean), _ptr(decay_logits),
+                                      _stream()), "arl2_commit")
+
+    def reset(self, stream_index: int = -1):
+        with torch.cuda.device(self.device):
+            _check(load().arl2_reset(self._ctx, stream_index, _stream()), "arl2_reset")
+
+    def get_state(self) -> torch.Tensor:
+        """Copy of S as a CPU fp32 tensor [B, H, D, D] (synchronises the stream)."""
+        dst = torch.empty(self.B, self.H, self.D, self.D, dtype=torch.float32)
+        with torch.cuda.device(self.device):
+            _check(load().arl2_get_state(self._ctx, _ptr(dst), _stream()), "arl2_get_state")
+            torch.cuda.current_stream().synchronize()
+        return dst
+
+    def set_state(self, src: torch.Tensor):
+        src = src.to(torch.float32).contiguous()
+        assert tuple(src.shape) == (self.B, self.H, self.D, self.D)
+        with torch.cuda.device(self.device):
+            _check(load().arl2_set_state(self._ctx, _ptr(src), _stream()), "arl2_set_state")
+            torch.cuda.current_stream().synchronize()
+
+    def sync_status(self):
+        with torch.cuda.device(self.device):
+            _check(load().arl2_sync_status(self._ctx, _stream()), "arl2_sync_status")
+
+    def set_profile_events(self, before: "torch.cuda.Event", after: "torch.cuda.Event"):
+        """The next denoise_step records these events around its dominant kernel."""
+        _check(load().arl2_set_profile_events(self._ctx, ctypes.c_void_p(before.cuda_event),
+                                              ctypes.c_void_p(after.cuda_event)),
+               "arl2_set_profile_events")
+
+    @property
+    def launch_count(self) -> int:
+        return int(load().arl2_launch_count(self._ctx))
+
+    @property
+    def step_kernel(self) -> str:
+        return load().arl2_step_kernel_name(self._ctx).decode()
+
+    def close(self):
+        if self._ctx is not None:
+            load().arl2_destroy(self._ctx)
+            self._ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- helpers -----------------------------------------------------------------------
+    def _want(self, t, shape, dtype, what):
+        if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous()
+                and tuple(t.shape) == tuple(shape) and t.dtype == dtype):
+            raise Arl2Error(f"{what}: expected a contiguous CUDA tensor {tuple(shape)} {dtype}, got "
+                            f"{tuple(t.shape)} {t.dtype} on {t.device}")

@@ -1,0 +1,350 @@
+// Host side of the C ABI declared in include/arl2.h: argument checks, workspace layout,
+// kernel selection and launches.  No device memory is allocated here.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "arl2_internal.h"
+
+namespace arl2 {
+
+static thread_local char g_error[512] = "";
+
+void set_error(const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_error, sizeof(g_error), fmt, ap);
+    va_end(ap);
+}
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct Layout {
+    size_t status, k_rot, partials, state_bf16, wq_op, wk_op, wv_op, total;
+    int nsplit;
+};
+
+bool valid_config(const arl2_config* c)
+{
+    if (c == nullptr) { set_error("config is NULL"); return false; }
+    if (c->struct_size != sizeof(arl2_config)) {
+        set_error("config.struct_size is %u, this library expects %zu", c->struct_size,
+                  sizeof(arl2_config));
+        return false;
+    }
+    if (c->B < 1 || c->H < 1 || c->L < 1) {
+        set_error("B, H and L must be >= 1 (got B=%d H=%d L=%d)", c->B, c->H, c->L);
+        return false;
+    }
+    if ((int64_t)c->B * c->H > 65535 * 8 || c->H > 65535 || c->B > 65535) {
+        set_error("B=%d, H=%d exceed the launch grid limits", c->B, c->H);
+        return false;
+    }
+    if (c->D != 64 && c->D != 128) { set_error("D must be 64 or 128 (got %d)", c->D); return false; }
+    if (c->io_dtype != ARL2_BF16 && c->io_dtype != ARL2_FP32) {
+        set_error("io_dtype must be ARL2_BF16 or ARL2_FP32 (got %d)", c->io_dtype);
+        return false;
+    }
+    if (c->commit_rule != 0) {
+        set_error("commit_rule %d is reserved; only 0 (gated linear) is built", c->commit_rule);
+        return false;
+    }
+    if (!(c->softmax_scale >= 0.0f) || !(c->l2_eps >= 0.0f) || isinf(c->softmax_scale) ||
+        isinf(c->l2_eps)) {
+        set_error("softmax_scale and l2_eps must be finite and >= 0");
+        return false;
+    }
+    if ((size_t)c->B * c->L * c->H * c->D >= ((size_t)1 << 40)) {
+        set_error("tensor too large");
+        return false;
+    }
+    return true;
+}
+
+Layout make_layout(const arl2_config& c)
+{
+    Layout l;
+    size_t esz = c.io_dtype == ARL2_FP32 ? 4 : 2;
+    size_t tensor = (size_t)c.B * c.L * c.H * c.D * esz;
+    size_t dd = (size_t)c.D * c.D;
+    l.nsplit = (c.L + kCommitChunk - 1) / kCommitChunk;
+    size_t off = 0;
+    l.status = off;     off += align_up(kStatusWords * sizeof(uint32_t));
+    l.k_rot = off;      off += align_up(tensor);
+    l.partials = off;   off += align_up((size_t)c.B * c.H * l.nsplit * dd * sizeof(float));
+    l.state_bf16 = off; off += align_up((size_t)c.B * c.H * dd * 2);
+    l.wq_op = off;      off += align_up((size_t)c.H * dd * 2);
+    l.wk_op = off;      off += align_up((size_t)c.H * dd * 2);
+    l.wv_op = off;      off += align_up((size_t)c.H * dd * 2);
+    l.total = off;
+    return l;
+}
+
+}  // namespace
+}  // namespace arl2
+
+using namespace arl2;
+
+struct arl2_ctx {
+    arl2_config cfg;
+    Shape shape;
+    Layout lay;
+    float* state;
+    uint8_t* ws;
+    const void *wq, *wk, *wv;
+    const float *rope_cos, *rope_sin;
+    bool use_tc;
+    uint64_t launches;
+    cudaEvent_t ev_before, ev_after;  // one-shot timing hook around the step kernel
+};
+
+namespace {
+
+inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
+
+bool check_ctx(const arl2_ctx* ctx)
+{
+    if (ctx == nullptr) { set_error("context is NULL"); return false; }
+    return true;
+}
+
+// adds the launches of a helper to the context's counter; passes errors through
+int account(arl2_ctx* ctx, int n)
+{
+    if (n < 0) return n;
+    ctx->launches += (uint64_t)n;
+    return ARL2_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* arl2_version(void) { return "arl2-b200 0.1"; }
+
+const char* arl2_last_error(void) { return g_error; }
+
+size_t arl2_workspace_bytes(const arl2_config* cfg)
+{
+    if (!valid_config(cfg)) return 0;
+    return make_layout(*cfg).total;
+}
+
+int arl2_create(const arl2_config* cfg, void* d_state, void* d_workspace, size_t workspace_bytes,
+                void* stream, arl2_ctx** out)
+{
+    if (out == nullptr) { set_error("out is NULL"); return ARL2_ERR_INVALID_ARG; }
+    *out = nullptr;
+    if (!valid_config(cfg)) return ARL2_ERR_INVALID_ARG;
+    if (d_state == nullptr || d_workspace == nullptr) {
+        set_error("d_state and d_workspace must not be NULL");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    Layout lay = make_layout(*cfg);
+    if (workspace_bytes < lay.total) {
+        set_error("workspace has %zu bytes, this configuration needs %zu", workspace_bytes, lay.total);
+        return ARL2_ERR_WORKSPACE;
+    }
+    if (reinterpret_cast<uintptr_t>(d_workspace) % kAlign != 0 ||
+        reinterpret_cast<uintptr_t>(d_state) % 16 != 0) {
+        set_error("d_workspace must be 256-byte aligned and d_state 16-byte aligned");
+        return ARL2_ERR_WORKSPACE;
+    }
+    int ndev = 0;
+    cudaError_t e = cudaGetDeviceCount(&ndev);
+    if (e != cudaSuccess || ndev == 0) {
+        set_error("no CUDA device: %s", cudaGetErrorString(e));
+        return ARL2_ERR_CUDA;
+    }
+    arl2_ctx* ctx = new (std::nothrow) arl2_ctx();
+    if (ctx == nullptr) { set_error("out of host memory"); return ARL2_ERR_INVALID_ARG; }
+    ctx->cfg = *cfg;
+    ctx->shape.B = cfg->B; ctx->shape.H = cfg->H; ctx->shape.L = cfg->L; ctx->shape.D = cfg->D;
+    float scale = cfg->softmax_scale > 0.0f ? cfg->softmax_scale : 1.0f / sqrtf((float)cfg->D);
+    ctx->shape.scale_log2 = scale * 1.4426950408889634f;
+    ctx->shape.eps = cfg->l2_eps > 0.0f ? cfg->l2_eps : 1e-6f;
+    ctx->lay = lay;
+    ctx->state = static_cast<float*>(d_state);
+    ctx->ws = static_cast<uint8_t*>(d_workspace);
+    ctx->wq = ctx->wk = ctx->wv = nullptr;
+    ctx->rope_cos = ctx->rope_sin = nullptr;
+    ctx->use_tc = false;  // the tensor-core path is selected here once it is built
+    ctx->launches = 0;
+    ctx->ev_before = ctx->ev_after = nullptr;
+    int r = account(ctx, fill_zero(ctx->ws + lay.status, kStatusWords * sizeof(uint32_t),
+                                   as_stream(stream)));
+    if (r != ARL2_OK) { delete ctx; return r; }
+    *out = ctx;
+    return ARL2_OK;
+}
+
+int arl2_set_params(arl2_ctx* ctx, const void* d_wphi_q, const void* d_wphi_k, const void* d_wphi_v,
+                    const float* d_rope_cos, const float* d_rope_sin, void* stream)
+{
+    (void)stream;
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    if ((d_rope_cos == nullptr) != (d_rope_sin == nullptr)) {
+        set_error("rope_cos and rope_sin must both be given or both be NULL");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    ctx->wq = d_wphi_q; ctx->wk = d_wphi_k; ctx->wv = d_wphi_v;
+    ctx->rope_cos = d_rope_cos; ctx->rope_sin = d_rope_sin;
+    return ARL2_OK;
+}
+
+int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const void* d_v,
+                      const float* d_gate_logits, void* d_out, void* stream)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    if (!d_q || !d_k || !d_v || !d_gate_logits || !d_out) {
+        set_error("denoise_step: q, k, v, gate_logits and out must not be NULL");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    if (d_out == d_q || d_out == d_k || d_out == d_v) {
+        set_error("denoise_step: out must not alias an input");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = as_stream(stream);
+    const void* k_rot = d_k;
+    if (ctx->rope_cos != nullptr) {
+        void* buf = ctx->ws + ctx->lay.k_rot;
+        int r = account(ctx, simt_rope_k(ctx->shape, ctx->cfg.io_dtype, d_k, ctx->rope_cos,
+                                         ctx->rope_sin, buf, st));
+        if (r != ARL2_OK) return r;
+        k_rot = buf;
+    }
+    StepArgs a;
+    a.s = ctx->shape;
+    a.q = d_q; a.k_rot = k_rot; a.v = d_v; a.gate = d_gate_logits;
+    a.state = ctx->state; a.wq = ctx->wq;
+    a.rope_cos = ctx->rope_cos; a.rope_sin = ctx->rope_sin;
+    a.out = d_out;
+    a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status);
+    cudaEvent_t e0 = ctx->ev_before, e1 = ctx->ev_after;
+    ctx->ev_before = ctx->ev_after = nullptr;
+    if (e0 != nullptr) cudaEventRecord(e0, st);
+    int r = account(ctx, simt_step(a, ctx->cfg.io_dtype, st));
+    if (e1 != nullptr) cudaEventRecord(e1, st);
+    return r;
+}
+
+int arl2_set_profile_events(arl2_ctx* ctx, void* ev_before, void* ev_after)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    ctx->ev_before = static_cast<cudaEvent_t>(ev_before);
+    ctx->ev_after = static_cast<cudaEvent_t>(ev_after);
+    return ARL2_OK;
+}
+
+int arl2_commit(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
+                const float* d_decay_logits, void* stream)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    if (!d_k_clean || !d_v_clean || !d_decay_logits) {
+        set_error("commit: k_clean, v_clean and decay_logits must not be NULL");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    CommitArgs a;
+    a.s = ctx->shape;
+    a.k = d_k_clean; a.v = d_v_clean; a.decay = d_decay_logits;
+    a.wk = ctx->wk; a.wv = ctx->wv;
+    a.rope_cos = ctx->rope_cos; a.rope_sin = ctx->rope_sin;
+    a.state = ctx->state;
+    a.partials = reinterpret_cast<float*>(ctx->ws + ctx->lay.partials);
+    a.state_bf16 = ctx->use_tc ? reinterpret_cast<__nv_bfloat16*>(ctx->ws + ctx->lay.state_bf16)
+                               : nullptr;
+    a.nsplit = ctx->lay.nsplit;
+    a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status);
+    return account(ctx, simt_commit(a, ctx->cfg.io_dtype, as_stream(stream)));
+}
+
+int arl2_reset(arl2_ctx* ctx, int32_t stream_index, void* stream)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    if (stream_index < -1 || stream_index >= ctx->cfg.B) {
+        set_error("reset: stream_index %d out of range [-1, %d)", stream_index, ctx->cfg.B);
+        return ARL2_ERR_INVALID_ARG;
+    }
+    size_t per = (size_t)ctx->cfg.H * ctx->cfg.D * ctx->cfg.D;
+    size_t first = stream_index < 0 ? 0 : (size_t)stream_index * per;
+    size_t count = stream_index < 0 ? per * ctx->cfg.B : per;
+    cudaStream_t st = as_stream(stream);
+    int r = account(ctx, fill_zero(ctx->state + first, count * sizeof(float), st));
+    if (r != ARL2_OK) return r;
+    if (ctx->use_tc) {
+        auto* sb = reinterpret_cast<__nv_bfloat16*>(ctx->ws + ctx->lay.state_bf16);
+        r = account(ctx, fill_zero(sb + first, count * 2, st));
+    }
+    return r;
+}
+
+int arl2_get_state(arl2_ctx* ctx, float* dst, void* stream)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    if (dst == nullptr) { set_error("get_state: dst is NULL"); return ARL2_ERR_INVALID_ARG; }
+    size_t bytes = (size_t)ctx->cfg.B * ctx->cfg.H * ctx->cfg.D * ctx->cfg.D * sizeof(float);
+    cudaError_t e = cudaMemcpyAsync(dst, ctx->state, bytes, cudaMemcpyDefault, as_stream(stream));
+    if (e != cudaSuccess) {
+        set_error("get_state: %s", cudaGetErrorString(e));
+        return ARL2_ERR_CUDA;
+    }
+    return ARL2_OK;
+}
+
+int arl2_set_state(arl2_ctx* ctx, const float* src, void* stream)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    if (src == nullptr) { set_error("set_state: src is NULL"); return ARL2_ERR_INVALID_ARG; }
+    size_t n = (size_t)ctx->cfg.B * ctx->cfg.H * ctx->cfg.D * ctx->cfg.D;
+    cudaStream_t st = as_stream(stream);
+    cudaError_t e = cudaMemcpyAsync(ctx->state, src, n * sizeof(float), cudaMemcpyDefault, st);
+    if (e != cudaSuccess) {
+        set_error("set_state: %s", cudaGetErrorString(e));
+        return ARL2_ERR_CUDA;
+    }
+    if (ctx->use_tc)
+        return account(ctx, state_to_bf16(ctx->state,
+                                          reinterpret_cast<__nv_bfloat16*>(ctx->ws + ctx->lay.state_bf16),
+                                          n, st));
+    return ARL2_OK;
+}
+
+int arl2_sync_status(arl2_ctx* ctx, void* stream)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    cudaStream_t st = as_stream(stream);
+    uint32_t words[2] = {0, 0};
+    cudaError_t e = cudaMemcpyAsync(words, ctx->ws + ctx->lay.status, sizeof(words),
+                                    cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) {
+        set_error("sync_status: %s", cudaGetErrorString(e));
+        return ARL2_ERR_CUDA;
+    }
+    if (words[0] != 0) {
+        set_error("a bounded wait inside a kernel expired (code %u, site %u)", words[0], words[1]);
+        int r = account(ctx, fill_zero(ctx->ws + ctx->lay.status, kStatusWords * sizeof(uint32_t), st));
+        if (r != ARL2_OK) return r;
+        return ARL2_ERR_TIMEOUT;
+    }
+    return ARL2_OK;
+}
+
+uint64_t arl2_launch_count(const arl2_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* arl2_step_kernel_name(const arl2_ctx* ctx)
+{
+    if (ctx == nullptr) return "";
+    return ctx->use_tc ? "tcgen05" : "simt";
+}
+
+void arl2_destroy(arl2_ctx* ctx) { delete ctx; }
+
+}  // extern "C"

@@ -1,0 +1,76 @@
+// Internal declarations shared by the host API and the kernel translation units.
+// Nothing here is part of the public ABI (see include/arl2.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "arl2.h"
+
+namespace arl2 {
+
+// Words of the device status block at the start of the workspace.
+enum StatusWord : int {
+    kStatusError = 0,    // first error code a kernel recorded (0 = none)
+    kStatusWhere = 1,    // which wait gave up (kernel-specific tag)
+    kStatusSched = 2,    // persistent tile scheduler counter (step kernel)
+    kStatusWords = 64
+};
+
+constexpr int kCommitChunk = 512;  // tokens per partial sum of the commit reduction
+
+struct Shape {
+    int B, H, L, D;
+    float scale_log2;  // softmax scale * log2(e): scores are exponentiated in base 2
+    float eps;
+};
+
+// Everything a step launch needs; plain pointers only.
+struct StepArgs {
+    Shape s;
+    const void* q;
+    const void* k_rot;      // K after RoPE (or the caller's K when there is no rotation)
+    const void* v;
+    const float* gate;      // [B, L, H]
+    const float* state;     // [B, H, D, D] fp32, read only
+    const void* wq;         // [H, D, D] (in, out) io dtype, or nullptr
+    const float* rope_cos;  // [L, D/2] or nullptr
+    const float* rope_sin;
+    void* out;
+    uint32_t* status;
+};
+
+struct CommitArgs {
+    Shape s;
+    const void* k;
+    const void* v;
+    const float* decay;     // [B, H]
+    const void* wk;
+    const void* wv;
+    const float* rope_cos;
+    const float* rope_sin;
+    float* state;           // [B, H, D, D] fp32, read-modify-write by the reduce kernel
+    float* partials;        // [B, H, nsplit, D, D] fp32
+    __nv_bfloat16* state_bf16;  // operand copy refreshed by the reduce kernel, or nullptr
+    int nsplit;
+    uint32_t* status;
+};
+
+// ---- plain-FMA kernels (arl2_simt.cu) -------------------------------------------------
+// Each returns the number of kernels it launched (>= 0) or a negative arl2_status.
+int simt_rope_k(const Shape& s, int dtype, const void* k, const float* cos_t, const float* sin_t,
+                void* k_rot, cudaStream_t st);
+int simt_step(const StepArgs& a, int dtype, cudaStream_t st);
+int simt_commit(const CommitArgs& a, int dtype, cudaStream_t st);
+int commit_reduce(const CommitArgs& a, cudaStream_t st);  // fixed-order sum + gated decay
+int fill_zero(void* p, size_t bytes, cudaStream_t st);
+int state_to_bf16(const float* state, __nv_bfloat16* dst, size_t n, cudaStream_t st);
+
+// ---- tensor-core kernels (arl2_tc.cu) ---------------------------------------------------
+struct TcParams;  // opaque to the API file
+bool tc_supported(const arl2_config& c);
+
+void set_error(const char* fmt, ...);
+
+}  // namespace arl2
