@@ -207,6 +207,9 @@ class Layer:
 
     def set_profile_events(self, before: "torch.cuda.Event", after: "torch.cuda.Event"):
         """The next denoise_step records these events around its dominant kernel."""
+        for ev in (before, after):
+            if not ev.cuda_event:   # torch creates the CUDA event lazily, at its first record
+                ev.record()
         _check(load().arl2_set_profile_events(self._ctx, ctypes.c_void_p(before.cuda_event),
                                               ctypes.c_void_p(after.cuda_event)),
                "arl2_set_profile_events")

@@ -61,17 +61,17 @@ __device__ __forceinline__ void tile_gemm(float (&acc)[4][D / 16], const float* 
 }
 
 // Load rows [r0, r0+64) x cols [c0, c0+ncols) of a [B, L, H, D] tensor (head h, stream b) into
-// a row-major smem matrix dst[r*ld + c]; rows past L are zero.
+// a row-major smem matrix dst[r*ld + c]; rows at or past `row_end` are zero.
 template <typename T>
 __device__ __forceinline__ void load_rows(float* dst, int ld, const T* __restrict__ src, int b,
-                                          int h, int r0, int c0, int ncols, int L, int H, int D,
-                                          int tid)
+                                          int h, int r0, int c0, int ncols, int row_end, int L,
+                                          int H, int D, int tid)
 {
     for (int idx = tid; idx < BM * ncols; idx += NT) {
         int r = idx / ncols, c = idx % ncols;
         int row = r0 + r;
         float x = 0.0f;
-        if (row < L) x = to_f(src[(((size_t)b * L + row) * H + h) * D + c0 + c]);
+        if (row < row_end) x = to_f(src[(((size_t)b * L + row) * H + h) * D + c0 + c]);
         dst[r * ld + c] = x;
     }
 }
@@ -291,7 +291,7 @@ __global__ void __launch_bounds__(NT) simt_step_kernel(StepArgs a)
 
     // inter branch: raw Q tile -> Q' = L2Norm(RoPE(Q W_phi_q)) -> Q' S
     float* Qp = Qt;  // [64][LD]
-    load_rows<T>(Qp, LD, q, b, h, i0, 0, D, L, H, D, tid);
+    load_rows<T>(Qp, LD, q, b, h, i0, 0, D, L, L, H, D, tid);
     __syncthreads();
     feature_tile<D, T>(Qp, Vs, a.wq ? static_cast<const T*>(a.wq) + (size_t)h * D * D : nullptr,
                        i0, L, a.rope_cos, a.rope_sin, a.s.eps, true, tx, ty, tid);
@@ -355,8 +355,8 @@ __global__ void __launch_bounds__(NT) simt_commit_partial_kernel(CommitArgs a)
         __syncthreads();
         // rows past l1 belong to the next chunk (or do not exist): zero them
         const int lim = l1;
-        load_rows<T>(Ks, LD, kc, b, h, r0, 0, D, lim, H, D, tid);
-        load_rows<T>(Vs2, LD, vc, b, h, r0, 0, D, lim, H, D, tid);
+        load_rows<T>(Ks, LD, kc, b, h, r0, 0, D, lim, L, H, D, tid);
+        load_rows<T>(Vs2, LD, vc, b, h, r0, 0, D, lim, L, H, D, tid);
         __syncthreads();
         feature_tile<D, T>(Ks, Ws, wk, r0, lim, a.rope_cos, a.rope_sin, a.s.eps, true, tx, ty, tid);
         feature_tile<D, T>(Vs2, Ws, wv, r0, lim, nullptr, nullptr, a.s.eps, false, tx, ty, tid);

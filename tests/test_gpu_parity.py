@@ -45,7 +45,7 @@ def test_tiny_full_schedule_fp32(oracle):
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
-@pytest.mark.parametrize("D,L", [(64, 1), (64, 24), (128, 127), (128, 129), (64, 200), (128, 333)])
+@pytest.mark.parametrize("D,L", [(64, 1), (64, 24), (128, 127), (128, 129), (64, 200), (128, 333), (64, 1100)])
 def test_ragged_shapes(oracle, dtype, D, L):
     """Edge sizes: a single token, tails shorter and longer than a tile, several tiles."""
     cfg = workload.custom(B=2, H=3, D=D, L=L, dtype=dtype, cfg_id=11)
