@@ -175,11 +175,21 @@ int arl2_create(const arl2_config* cfg, void* d_state, void* d_workspace, size_t
     ctx->ws = static_cast<uint8_t*>(d_workspace);
     ctx->wq = ctx->wk = ctx->wv = nullptr;
     ctx->rope_cos = ctx->rope_sin = nullptr;
-    ctx->use_tc = false;  // the tensor-core path is selected here once it is built
+    ctx->use_tc = tc_supported(*cfg);
     ctx->launches = 0;
     ctx->ev_before = ctx->ev_after = nullptr;
     int r = account(ctx, fill_zero(ctx->ws + lay.status, kStatusWords * sizeof(uint32_t),
                                    as_stream(stream)));
+    if (r == ARL2_OK && ctx->use_tc) {
+        // operand copies the tensor-core kernels read: identity feature maps until
+        // arl2_set_params, and the bf16 mirror of whatever the state buffer holds now
+        r = account(ctx, tc_prepare_map(nullptr, reinterpret_cast<__nv_bfloat16*>(ctx->ws + lay.wq_op),
+                                        cfg->H, as_stream(stream)));
+        if (r == ARL2_OK)
+            r = account(ctx, state_to_bf16(ctx->state,
+                                           reinterpret_cast<__nv_bfloat16*>(ctx->ws + lay.state_bf16),
+                                           (size_t)cfg->B * cfg->H * cfg->D * cfg->D, as_stream(stream)));
+    }
     if (r != ARL2_OK) { delete ctx; return r; }
     *out = ctx;
     return ARL2_OK;
@@ -188,14 +198,20 @@ int arl2_create(const arl2_config* cfg, void* d_state, void* d_workspace, size_t
 int arl2_set_params(arl2_ctx* ctx, const void* d_wphi_q, const void* d_wphi_k, const void* d_wphi_v,
                     const float* d_rope_cos, const float* d_rope_sin, void* stream)
 {
-    (void)stream;
     if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
     if ((d_rope_cos == nullptr) != (d_rope_sin == nullptr)) {
         set_error("rope_cos and rope_sin must both be given or both be NULL");
         return ARL2_ERR_INVALID_ARG;
     }
+    if (reinterpret_cast<uintptr_t>(d_rope_cos) % 16 != 0 || reinterpret_cast<uintptr_t>(d_rope_sin) % 16 != 0) {
+        set_error("rope tables must be 16-byte aligned");
+        return ARL2_ERR_INVALID_ARG;
+    }
     ctx->wq = d_wphi_q; ctx->wk = d_wphi_k; ctx->wv = d_wphi_v;
     ctx->rope_cos = d_rope_cos; ctx->rope_sin = d_rope_sin;
+    if (ctx->use_tc)
+        return account(ctx, tc_prepare_map(d_wphi_q, reinterpret_cast<__nv_bfloat16*>(ctx->ws + ctx->lay.wq_op),
+                                           ctx->cfg.H, as_stream(stream)));
     return ARL2_OK;
 }
 
@@ -209,6 +225,11 @@ int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const voi
     }
     if (d_out == d_q || d_out == d_k || d_out == d_v) {
         set_error("denoise_step: out must not alias an input");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    if ((reinterpret_cast<uintptr_t>(d_q) | reinterpret_cast<uintptr_t>(d_k) |
+         reinterpret_cast<uintptr_t>(d_v) | reinterpret_cast<uintptr_t>(d_out)) % 16 != 0) {
+        set_error("denoise_step: q, k, v and out must be 16-byte aligned");
         return ARL2_ERR_INVALID_ARG;
     }
     cudaStream_t st = as_stream(stream);
@@ -230,7 +251,12 @@ int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const voi
     cudaEvent_t e0 = ctx->ev_before, e1 = ctx->ev_after;
     ctx->ev_before = ctx->ev_after = nullptr;
     if (e0 != nullptr) cudaEventRecord(e0, st);
-    int r = account(ctx, simt_step(a, ctx->cfg.io_dtype, st));
+    int r;
+    if (ctx->use_tc)
+        r = account(ctx, tc_step(a, reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wq_op),
+                                 reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.state_bf16), st));
+    else
+        r = account(ctx, simt_step(a, ctx->cfg.io_dtype, st));
     if (e1 != nullptr) cudaEventRecord(e1, st);
     return r;
 }

@@ -68,8 +68,11 @@ int fill_zero(void* p, size_t bytes, cudaStream_t st);
 int state_to_bf16(const float* state, __nv_bfloat16* dst, size_t n, cudaStream_t st);
 
 // ---- tensor-core kernels (arl2_tc.cu) ---------------------------------------------------
-struct TcParams;  // opaque to the API file
 bool tc_supported(const arl2_config& c);
+// w: [H, 128, 128] (in, out) bf16 or nullptr (identity) -> w_op: [H, out, in] bf16
+int tc_prepare_map(const void* w, __nv_bfloat16* w_op, int H, cudaStream_t st);
+int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* state_bf16,
+            cudaStream_t st);
 
 void set_error(const char* fmt, ...);
 
