@@ -102,6 +102,7 @@ struct arl2_ctx {
     const float *rope_cos, *rope_sin;
     bool use_tc;
     uint64_t launches;
+    uint32_t step_calls;   // parity selects the scheduler counter of the next step launch
     cudaEvent_t ev_before, ev_after;  // one-shot timing hook around the step kernel
 };
 
@@ -177,6 +178,7 @@ int arl2_create(const arl2_config* cfg, void* d_state, void* d_workspace, size_t
     ctx->rope_cos = ctx->rope_sin = nullptr;
     ctx->use_tc = tc_supported(*cfg);
     ctx->launches = 0;
+    ctx->step_calls = 0;
     ctx->ev_before = ctx->ev_after = nullptr;
     int r = account(ctx, fill_zero(ctx->ws + lay.status, kStatusWords * sizeof(uint32_t),
                                    as_stream(stream)));
@@ -248,6 +250,7 @@ int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const voi
     a.rope_cos = ctx->rope_cos; a.rope_sin = ctx->rope_sin;
     a.out = d_out;
     a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status);
+    a.launch_parity = (int)(ctx->step_calls++ & 1u);
     cudaEvent_t e0 = ctx->ev_before, e1 = ctx->ev_after;
     ctx->ev_before = ctx->ev_after = nullptr;
     if (e0 != nullptr) cudaEventRecord(e0, st);

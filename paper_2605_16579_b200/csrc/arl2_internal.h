@@ -14,7 +14,7 @@ namespace arl2 {
 enum StatusWord : int {
     kStatusError = 0,    // first error code a kernel recorded (0 = none)
     kStatusWhere = 1,    // which wait gave up (kernel-specific tag)
-    kStatusSched = 2,    // persistent tile scheduler counter (step kernel)
+    kStatusSched = 2,    // two item counters of the persistent step kernel (words 2 and 3)
     kStatusWords = 64
 };
 
@@ -39,6 +39,7 @@ struct StepArgs {
     const float* rope_sin;
     void* out;
     uint32_t* status;
+    int launch_parity;      // step launches so far on this context, mod 2 (scheduler counters)
 };
 
 struct CommitArgs {

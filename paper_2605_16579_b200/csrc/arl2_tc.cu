@@ -1,17 +1,21 @@
 // Tensor-core (tcgen05 / TMEM / TMA) kernels of the ARL^2 layer for bf16 I/O, D = 128.
 //
-// Step kernel: one CTA per (stream b, head h, pair of 128-row query tiles).   (Eq. 2, 3, 5-8)
+// Step kernel (Eq. 2, 3, 5-8): persistent, one CTA per SM, work item = (stream b, head h, pair
+// of 128-row query tiles), items handed out by an atomic counter (pairs first, the single
+// ragged tiles last).
 //   warps 0-3 / 4-7  softmax group of query tile 0 / 1 (one thread per query row)
-//   warp 8           TMA producer: Q tiles, then K_j, V_j tiles through a 3-slot ring, then the
-//                    head's feature map W_phi_q^T and the bf16 copy of the state S as the
-//                    last two "tiles" of the ring
-//   warp 9           MMA issuer (one thread): S_t = Q~_t K_j^T and O_t += P_t V_j into TMEM
+//   warp 8           TMA producer and scheduler: the Q tiles, then through a 5-slot ring K_j, V_j
+//                    for every key tile, then W_phi_q^T, the raw Q tiles again and the bf16
+//                    copy of the state S
+//   warp 9 / 10      MMA issuer of tile 0 / 1 (one thread each): S_t = Q~_t K_j^T and
+//                    O_t += P_t V_j into TMEM
 // TMEM (512 columns): S_0 | S_1 | O_0 | O_1, 128 fp32 columns each; the bf16 probabilities P_t
 // overwrite the first 64 columns of S_t and feed the second MMA straight from TMEM.
-// The inter branch reuses the loop as one more iteration: "S" = Q W_phi_q (A = raw Q tile),
-// the group turns each row into sigmoid(g) * l * L2Norm(RoPE(.)) (l = softmax row sum) and
-// the "PV" MMA multiplies it by the state, accumulating into O_t, so the final O_t / l is
-// O_intra + sigmoid(g) O_inter.  The state is only read.
+// RoPE(Q) is applied in place in shared memory by the softmax groups; K arrives rotated.
+// The inter branch reuses the loop as one more iteration: "S" = Q W_phi_q (A = the raw Q tile
+// from the ring), the group turns each row into sigmoid(g) * l * L2Norm(RoPE(.)) (l = softmax
+// row sum) and the "PV" MMA multiplies it by the state, accumulating into O_t, so that the
+// final O_t / l is O_intra + sigmoid(g) O_inter.  The state is only read.
 //
 // Every wait is bounded: when a limit expires the thread records ARL2_ERR_TIMEOUT in the
 // device status block, raises the CTA's abort flag and every role falls through to the exit.
@@ -29,28 +33,40 @@ using namespace ptx;
 constexpr int kTile = 128;               // query rows per tile = keys per tile = head dim
 constexpr int kTileBytes = kTile * kTile * 2;
 constexpr int kHalfBytes = kTileBytes / 2;  // one 64-column TMA box of a tile
-constexpr int kStages = 3;
-constexpr int kThreads = 320;
+constexpr int kStages = 5;
+constexpr int kThreads = 384;              // 3 warpgroups: softmax 0, softmax 1, {TMA, MMA, 2 idle}
+constexpr int kRegsSoftmax = 232;          // per-thread registers after the warpgroups rebalance
+constexpr int kRegsOther = 40;
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units of slack before O is rescaled
+#ifndef ARL2_POLY_COUNT
+#define ARL2_POLY_COUNT 0
+#endif
+#ifndef ARL2_POLY_PERIOD
+#define ARL2_POLY_PERIOD 2
+#endif
+constexpr int kPolyCount = ARL2_POLY_COUNT;    // of every kPolyPeriod element pairs, this many take the
+constexpr int kPolyPeriod = ARL2_POLY_PERIOD;  // polynomial exponential, the rest the special-function unit
 
 // shared memory map (offsets from a 1024-byte aligned base)
-constexpr int kOffQRaw = 0;                              // 2 tiles, as loaded
-constexpr int kOffQRot = kOffQRaw + 2 * kTileBytes;      // 2 tiles, after RoPE
-constexpr int kOffRing = kOffQRot + 2 * kTileBytes;      // kStages tiles
+constexpr int kOffQ = 0;                                 // 2 query tiles (rotated in place)
+constexpr int kOffRing = kOffQ + 2 * kTileBytes;         // kStages tiles
 constexpr int kOffBars = kOffRing + kStages * kTileBytes;
 constexpr int kSmemBytes = kOffBars + 256 + 1024;        // barriers + alignment slack
 
 enum Bar : int {
-    kBarQFull = 0,
-    kBarQRot0, kBarQRot1,
+    kBarQFull = 0,                              // producer -> all: Q tiles (and the item id) landed
+    kBarQFree,                                  // MMA -> producer: last MMA reading Q~ is done
+    kBarQRot0, kBarQRot1,                       // softmax group t -> MMA: Q~_t rotated
     kBarFull0,                                  // kStages of them
     kBarEmpty0 = kBarFull0 + kStages,           // kStages of them
     kBarSFull0 = kBarEmpty0 + kStages, kBarSFull1,
     kBarPFull0, kBarPFull1,
-    kBarOFinal,
+    kBarOFinal0, kBarOFinal1,
+    kBarTok0, kBarTok1,                         // softmax groups take turns in the exponential phase
     kNumBars
 };
+// after the barriers: TMEM base (4 B), abort flag (4 B), two item-id slots (8 B)
 static_assert(kNumBars * 8 + 16 <= 256, "barrier block");
 
 struct TcStepParams {
@@ -60,7 +76,11 @@ struct TcStepParams {
     const float* rope_sin;
     __nv_bfloat16* out;
     uint32_t* status;
-    int n_kv;      // key tiles per head
+    uint32_t* sched_counter;   // this launch's item counter (zero on entry)
+    uint32_t* sched_next;      // the next launch's counter: cleared by this launch
+    int n_kv;                  // key tiles per head = query tiles per head
+    int n_pair_items;          // B * H * (n_kv / 2): items with two query tiles
+    int n_items;               // + B * H single-tile items when n_kv is odd
 };
 
 struct Abort {
@@ -87,176 +107,335 @@ __device__ __forceinline__ void drain_bar(uint32_t bar, uint32_t parity)
         if (mbar_try_wait(bar, parity)) return;
 }
 
+#ifdef ARL2_TRACE
+// Timeline probe for tuning builds: one thread of CTA 0 stamps the SM clock into the status
+// block for two loop iterations of its first item.  Not compiled into the product library.
+#define ARL2_STAMP(cond, slot) do { if (cond) p.status[(slot)] = (uint32_t)clock64(); } while (0)
+#else
+#define ARL2_STAMP(cond, slot) do { } while (0)
+#endif
+
 __device__ __forceinline__ float sigmoid_fast(float x) { return 1.0f / (1.0f + __expf(-x)); }
 
-// One softmax group thread: owns query row `r` of tile `t`.
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// packed pairs of fp32 (one 64-bit register pair per operand)
+__device__ __forceinline__ uint64_t pack2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// 2^x for a pair of values without the special-function unit: x = j + f with j = round(x),
+// f in [-0.5, 0.5]; 2^f by a cubic (max relative error 7.5e-5, well under the bf16 rounding of
+// the probabilities), 2^j by adding j to the exponent field.  x is clamped at -126.
+__device__ __forceinline__ void exp2_poly2(float x0, float x1, float& r0, float& r1)
+{
+    const float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
+    x0 = fmaxf(x0, -126.0f);
+    x1 = fmaxf(x1, -126.0f);
+    const uint64_t x2 = pack2(x0, x1);
+    const uint64_t t2 = add2(x2, pack2(kMagic, kMagic));
+    const uint64_t j2 = add2(t2, pack2(-kMagic, -kMagic));
+    const uint64_t f2 = fma2(j2, pack2(-1.0f, -1.0f), x2);
+    uint64_t p2 = fma2(pack2(0.05517132207751274f, 0.05517132207751274f), f2,
+                       pack2(0.24261054396629333f, 0.24261054396629333f));
+    p2 = fma2(p2, f2, pack2(0.6932609677314758f, 0.6932609677314758f));
+    p2 = fma2(p2, f2, pack2(0.9999281167984009f, 0.9999281167984009f));
+    float t0, t1, q0, q1;
+    unpack2(t2, t0, t1);
+    unpack2(p2, q0, q1);
+    r0 = __int_as_float(__float_as_int(q0) + (__float_as_int(t0) << 23));
+    r1 = __int_as_float(__float_as_int(q1) + (__float_as_int(t1) << 23));
+}
+
+struct Item {
+    int b, h, q_row0;
+    bool two;   // the pair's second tile exists
+};
+
+// Items [0, n_pair_items) are pairs of full tiles, (b, h)-major so that neighbours share K and V
+// in L2; the rest are the single ragged tiles, which fill the tail of the schedule.
+__device__ __forceinline__ Item decode_item(int id, const TcStepParams& p)
+{
+    Item it;
+    int bh, pair;
+    const int full_pairs = p.n_kv >> 1;
+    if (id < p.n_pair_items) {
+        bh = id / full_pairs;
+        pair = id - bh * full_pairs;
+        it.two = true;
+    } else {
+        bh = id - p.n_pair_items;
+        pair = full_pairs;
+        it.two = false;
+    }
+    it.b = bh / p.s.H;
+    it.h = bh - it.b * p.s.H;
+    it.q_row0 = pair * 2 * kTile;
+    return it;
+}
+
+// One softmax group thread: owns query row `r` of tile `t` of every item.
 __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* smem, uint32_t bars,
-                                             uint32_t tmem_base, const Abort& ab, int t, int r,
-                                             int warp_in_group, int b, int h, int q_row0,
-                                             bool tile_active)
+                                             uint32_t tmem_base, const Abort& ab,
+                                             const volatile int* item_slots, int t, int r,
+                                             int warp_in_group)
 {
     const int L = p.s.L, H = p.s.H;
-    const int row = q_row0 + r;
-    const bool valid_row = row < L;
     const uint32_t lane_base = tmem_base + ((uint32_t)(warp_in_group * 32) << 16);
     const uint32_t s_addr = lane_base + (uint32_t)(t * kTile);
     const uint32_t o_addr = lane_base + (uint32_t)(2 * kTile + t * kTile);
     const uint32_t bar_s = bars + 8 * (kBarSFull0 + t);
     const uint32_t bar_p = bars + 8 * (kBarPFull0 + t);
-
-    // ---- Q~ = RoPE(Q): rotate this thread's row from the raw tile into the MMA operand tile
-    if (!wait_bar(bars + 8 * kBarQFull, 0, ab, 10)) return;
-    if (!tile_active) return;
-    if (p.rope_cos != nullptr) {
-        const uint8_t* src = smem + kOffQRaw + t * kTileBytes;
-        uint8_t* dst = smem + kOffQRot + t * kTileBytes;
-        const float* cs = p.rope_cos + (size_t)(valid_row ? row : 0) * (kTile / 2);
-        const float* sn = p.rope_sin + (size_t)(valid_row ? row : 0) * (kTile / 2);
-#pragma unroll 4
-        for (int c = 0; c < 16; ++c) {
-            int off = (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
-            uint4 raw = *reinterpret_cast<const uint4*>(src + off);
-            float4 cv = *reinterpret_cast<const float4*>(cs + c * 4);
-            float4 sv = *reinterpret_cast<const float4*>(sn + c * 4);
-            uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-            float cc[4] = {cv.x, cv.y, cv.z, cv.w}, ss[4] = {sv.x, sv.y, sv.z, sv.w};
-#pragma unroll
-            for (int m = 0; m < 4; ++m) {
-                float x0 = __uint_as_float(w[m] << 16);
-                float x1 = __uint_as_float(w[m] & 0xFFFF0000u);
-                w[m] = pack_bf16(x0 * cc[m] - x1 * ss[m], x0 * ss[m] + x1 * cc[m]);
-            }
-            *reinterpret_cast<uint4*>(dst + off) = make_uint4(w[0], w[1], w[2], w[3]);
-        }
-        fence_proxy_async_smem();
-    }
-    mbar_arrive(bars + 8 * (kBarQRot0 + t));
-
-    float m_ref = -INFINITY;   // reference maximum (scaled, base 2) the probabilities use
-    float l_sum = 0.0f;        // running row sum relative to m_ref
     const float c2 = p.s.scale_log2;
+    const uint64_t c2x2 = pack2(c2, c2);
     const int n_kv = p.n_kv;
+    uint32_t s_cnt = 0;   // phases of bar_s consumed so far
+    uint32_t of_cnt = 0;  // phases of this tile's final-O barrier consumed so far
+    uint32_t tok_cnt = 0; // turns taken in the exponential phase
     uint32_t sreg[128];
 
-    for (int j = 0; j < n_kv; ++j) {
-        if (!wait_bar(bar_s, (uint32_t)(j & 1), ab, 20 + t)) return;
-        tc_fence_after();
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-            tmem_ld32(s_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
-        tmem_wait_ld();
+    for (uint32_t item = 0;; ++item) {
+        if (!wait_bar(bars + 8 * kBarQFull, item & 1, ab, 10)) return;
+        const int id = item_slots[item & 1];
+        if (id < 0) return;
+        const Item it = decode_item(id, p);
+        const int b = it.b, h = it.h;
+        const int row = it.q_row0 + t * kTile + r;
+        const bool valid_row = row < L;
+        const bool active = t == 0 || it.two;
 
-        const int n_valid = L - j * kTile;  // keys of this tile that exist
-        if (n_valid < kTile) {   // ragged last tile: zero-filled key rows must not count
+        if (active) {
+            // ---- Q~ = RoPE(Q): rotate this thread's row of the tile in place          (Eq. 2)
+            if (p.rope_cos != nullptr) {
+                uint8_t* tile = smem + kOffQ + t * kTileBytes;
+                const float* cs = p.rope_cos + (size_t)(valid_row ? row : 0) * (kTile / 2);
+                const float* sn = p.rope_sin + (size_t)(valid_row ? row : 0) * (kTile / 2);
+#pragma unroll 4
+                for (int c = 0; c < 16; ++c) {
+                    int off = (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+                    uint4 raw = *reinterpret_cast<const uint4*>(tile + off);
+                    float4 cv = *reinterpret_cast<const float4*>(cs + c * 4);
+                    float4 sv = *reinterpret_cast<const float4*>(sn + c * 4);
+                    uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+                    float cc[4] = {cv.x, cv.y, cv.z, cv.w}, ss[4] = {sv.x, sv.y, sv.z, sv.w};
 #pragma unroll
-            for (int c = 0; c < 128; ++c)
-                if (c >= n_valid) sreg[c] = __float_as_uint(-INFINITY);
-        }
-        float mx = -INFINITY;
-#pragma unroll
-        for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(sreg[c]));
-        float m_new = fmaxf(m_ref, mx * c2);
-        bool need = (m_new - m_ref) > kRescaleThreshold;   // first tile: inf > threshold
-        if (__any_sync(0xffffffffu, need)) {
-            float alpha = 1.0f;
-            if (need) {
-                alpha = ex2_approx(m_ref - m_new);
-                m_ref = m_new;
-                l_sum *= alpha;
+                    for (int m = 0; m < 4; ++m) {
+                        float x0 = __uint_as_float(w[m] << 16);
+                        float x1 = __uint_as_float(w[m] & 0xFFFF0000u);
+                        w[m] = pack_bf16(x0 * cc[m] - x1 * ss[m], x0 * ss[m] + x1 * cc[m]);
+                    }
+                    *reinterpret_cast<uint4*>(tile + off) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+                fence_proxy_async_smem();
             }
-            if (j > 0) {
-                // the MMA that last accumulated into O_t finished before S_t(j) was signalled,
-                // and the next one waits for this group's arrival below: O_t is ours for now
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(o_addr + c * 32, o);
-                    tmem_wait_ld();
+            mbar_arrive(bars + 8 * (kBarQRot0 + t));
+
+            float m_ref = -INFINITY;   // reference maximum (scaled, base 2) of the probabilities
+            uint64_t l2 = pack2(0.0f, 0.0f);   // running row sum relative to m_ref, two lanes
+
+            for (int j = 0; j < n_kv; ++j) {
+#ifdef ARL2_TRACE
+                const bool tr = blockIdx.x == 0 && item == 0 && r == 0 && (j == 8 || j == 9);
+                const int ts = 8 + t * 16 + (j - 8) * 8;
+#endif
+                ARL2_STAMP(tr, ts + 0);
+                if (!wait_bar(bar_s, s_cnt & 1, ab, 20 + t)) return;
+                ++s_cnt;
+                tc_fence_after();
+                ARL2_STAMP(tr, ts + 1);
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                    tmem_st32(o_addr + c * 32, o);
+                for (int c = 0; c < 4; ++c)
+                    tmem_ld32(s_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
+                tmem_wait_ld();
+                ARL2_STAMP(tr, ts + 2);
+
+                const int n_valid = L - j * kTile;  // keys of this tile that exist
+                if (n_valid < kTile) {   // ragged last tile: zero-filled key rows must not count
+#pragma unroll
+                    for (int c = 0; c < 128; ++c)
+                        if (c >= n_valid) sreg[c] = __float_as_uint(-INFINITY);
+                }
+                float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                for (int c = 0; c < 128; c += 8) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        m4[k] = max3(m4[k], __uint_as_float(sreg[c + 2 * k]), __uint_as_float(sreg[c + 2 * k + 1]));
+                }
+                const float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+                const float m_new = fmaxf(m_ref, mx * c2);
+                const bool need = (m_new - m_ref) > kRescaleThreshold;   // first tile: inf > threshold
+                ARL2_STAMP(tr, ts + 3);
+                if (__any_sync(0xffffffffu, need)) {
+                    float alpha = 1.0f;
+                    if (need) {
+                        alpha = ex2_approx(m_ref - m_new);
+                        m_ref = m_new;
+                        l2 = fma2(l2, pack2(alpha, alpha), pack2(0.0f, 0.0f));
+                    }
+                    if (j > 0) {
+                        // the MMA that last accumulated into O_t finished before S_t(j) was
+                        // signalled, and the next one waits for this group's arrival below
+#pragma unroll 1
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t o[32];
+                            tmem_ld32(o_addr + c * 32, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                            tmem_st32(o_addr + c * 32, o);
+                        }
+                    }
+                }
+                const uint64_t neg_m2 = pack2(-m_ref, -m_ref);
+                if (it.two) {
+                    // the two groups alternate in the exponential phase, so that one group's
+                    // exponentials overlap the other tile's MMAs instead of its exponentials
+                    const uint32_t par = (t == 0) ? ((tok_cnt + 1) & 1) : (tok_cnt & 1);
+                    if (!wait_bar(bars + 8 * (kBarTok0 + t), par, ab, 24 + t)) return;
+                    ++tok_cnt;
+                }
+                ARL2_STAMP(tr, ts + 4);
+#ifndef ARL2_SOFTMAX_SCALAR
+#pragma unroll
+                for (int c = 0; c < 64; ++c) {
+                    float x0, x1, p0, p1;
+                    unpack2(fma2(pack2(__uint_as_float(sreg[2 * c]), __uint_as_float(sreg[2 * c + 1])), c2x2, neg_m2),
+                            x0, x1);
+                    if ((c % kPolyPeriod) < kPolyCount) {
+                        exp2_poly2(x0, x1, p0, p1);      // FMA / integer pipes
+                    } else {
+                        p0 = ex2_approx(x0);             // special-function unit
+                        p1 = ex2_approx(x1);
+                    }
+                    l2 = add2(l2, pack2(p0, p1));
+                    sreg[c] = pack_bf16(p0, p1);
+                }
+#else
+                {
+                    float la, lb;
+                    unpack2(l2, la, lb);
+                    const float nm = -m_ref;
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) {
+                        const float p0 = ex2_approx(fmaf(__uint_as_float(sreg[2 * c]), c2, nm));
+                        const float p1 = ex2_approx(fmaf(__uint_as_float(sreg[2 * c + 1]), c2, nm));
+                        la += p0;
+                        lb += p1;
+                        sreg[c] = pack_bf16(p0, p1);
+                    }
+                    l2 = pack2(la, lb);
+                }
+#endif
+                if (it.two) mbar_arrive(bars + 8 * (kBarTok0 + (t ^ 1)));
+                ARL2_STAMP(tr, ts + 5);
+                tmem_st32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sreg[0]));
+                tmem_st32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[32]));
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar_p);
+                ARL2_STAMP(tr, ts + 6);
+            }
+            float l_lo, l_hi;
+            unpack2(l2, l_lo, l_hi);
+            const float l_sum = l_lo + l_hi;
+
+            // ---- inter branch: U = Q W_phi_q arrives in the S columns                  (Eq. 3)
+            if (!wait_bar(bar_s, s_cnt & 1, ab, 30 + t)) return;
+            ++s_cnt;
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                tmem_ld32(s_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
+            tmem_wait_ld();
+            {
+                if (p.rope_cos != nullptr && valid_row) {
+                    const float* cs = p.rope_cos + (size_t)row * (kTile / 2);
+                    const float* sn = p.rope_sin + (size_t)row * (kTile / 2);
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        float4 cv = *reinterpret_cast<const float4*>(cs + c * 4);
+                        float4 sv = *reinterpret_cast<const float4*>(sn + c * 4);
+                        float cc[4] = {cv.x, cv.y, cv.z, cv.w}, s4[4] = {sv.x, sv.y, sv.z, sv.w};
+#pragma unroll
+                        for (int m = 0; m < 4; ++m) {
+                            float x0 = __uint_as_float(sreg[c * 8 + 2 * m]);
+                            float x1 = __uint_as_float(sreg[c * 8 + 2 * m + 1]);
+                            sreg[c * 8 + 2 * m] = __float_as_uint(x0 * cc[m] - x1 * s4[m]);
+                            sreg[c * 8 + 2 * m + 1] = __float_as_uint(x0 * s4[m] + x1 * cc[m]);
+                        }
+                    }
+                }
+                float ss4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+                for (int c = 0; c < 128; c += 4) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        ss4[k] = fmaf(__uint_as_float(sreg[c + k]), __uint_as_float(sreg[c + k]), ss4[k]);
+                }
+                const float ss = (ss4[0] + ss4[1]) + (ss4[2] + ss4[3]);
+                const float gate = valid_row ? sigmoid_fast(p.gate[((size_t)b * L + row) * H + h]) : 0.0f;
+                // scaled by the row sum so that the common 1/l of the epilogue leaves gate * Q' S
+                const float f = rsqrtf(ss + p.s.eps) * gate * l_sum;
+#pragma unroll
+                for (int c = 0; c < 64; ++c)
+                    sreg[c] = pack_bf16(__uint_as_float(sreg[2 * c]) * f, __uint_as_float(sreg[2 * c + 1]) * f);
+            }
+            tmem_st32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sreg[0]));
+            tmem_st32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[32]));
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar_p);
+
+            // ---- epilogue: O_t / l -> bf16 -> global                              (Eq. 6-7)
+            if (!wait_bar(bars + 8 * (kBarOFinal0 + t), of_cnt & 1, ab, 40 + t)) return;
+            ++of_cnt;
+            tc_fence_after();
+            const float inv_l = 1.0f / l_sum;
+            __nv_bfloat16* orow = p.out + (((size_t)b * L + (valid_row ? row : 0)) * H + h) * kTile;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                uint32_t o[32];
+                tmem_ld32(o_addr + c * 32, o);
+                tmem_wait_ld();
+                if (valid_row) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        uint4 v;
+                        v.x = pack_bf16(__uint_as_float(o[e * 8 + 0]) * inv_l, __uint_as_float(o[e * 8 + 1]) * inv_l);
+                        v.y = pack_bf16(__uint_as_float(o[e * 8 + 2]) * inv_l, __uint_as_float(o[e * 8 + 3]) * inv_l);
+                        v.z = pack_bf16(__uint_as_float(o[e * 8 + 4]) * inv_l, __uint_as_float(o[e * 8 + 5]) * inv_l);
+                        v.w = pack_bf16(__uint_as_float(o[e * 8 + 6]) * inv_l, __uint_as_float(o[e * 8 + 7]) * inv_l);
+                        *reinterpret_cast<uint4*>(orow + c * 32 + e * 8) = v;
+                    }
                 }
             }
-        }
-        const float neg_m = -m_ref;
-#pragma unroll
-        for (int c = 0; c < 64; ++c) {
-            float p0 = ex2_approx(fmaf(__uint_as_float(sreg[2 * c]), c2, neg_m));
-            float p1 = ex2_approx(fmaf(__uint_as_float(sreg[2 * c + 1]), c2, neg_m));
-            l_sum += p0 + p1;
-            sreg[c] = pack_bf16(p0, p1);
-        }
-        tmem_st32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sreg[0]));
-        tmem_st32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[32]));
-        tmem_wait_st();
-        tc_fence_before();
-        mbar_arrive(bar_p);
-    }
-
-    // ---- inter branch: U = Q W_phi_q arrives in the S columns                       (Eq. 3)
-    if (!wait_bar(bar_s, (uint32_t)(n_kv & 1), ab, 30 + t)) return;
-    tc_fence_after();
-#pragma unroll
-    for (int c = 0; c < 4; ++c)
-        tmem_ld32(s_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
-    tmem_wait_ld();
-    {
-        float ss = 0.0f;
-        if (p.rope_cos != nullptr && valid_row) {
-            const float* cs = p.rope_cos + (size_t)row * (kTile / 2);
-            const float* sn = p.rope_sin + (size_t)row * (kTile / 2);
-#pragma unroll
-            for (int c = 0; c < 16; ++c) {
-                float4 cv = *reinterpret_cast<const float4*>(cs + c * 4);
-                float4 sv = *reinterpret_cast<const float4*>(sn + c * 4);
-                float cc[4] = {cv.x, cv.y, cv.z, cv.w}, s4[4] = {sv.x, sv.y, sv.z, sv.w};
-#pragma unroll
-                for (int m = 0; m < 4; ++m) {
-                    float x0 = __uint_as_float(sreg[c * 8 + 2 * m]);
-                    float x1 = __uint_as_float(sreg[c * 8 + 2 * m + 1]);
-                    sreg[c * 8 + 2 * m] = __float_as_uint(x0 * cc[m] - x1 * s4[m]);
-                    sreg[c * 8 + 2 * m + 1] = __float_as_uint(x0 * s4[m] + x1 * cc[m]);
-                }
-            }
-        }
-#pragma unroll
-        for (int c = 0; c < 128; ++c) ss = fmaf(__uint_as_float(sreg[c]), __uint_as_float(sreg[c]), ss);
-        float gate = valid_row ? sigmoid_fast(p.gate[((size_t)b * L + row) * H + h]) : 0.0f;
-        // scaled by the row sum so that the common 1/l of the epilogue leaves gate * Q' S
-        float f = rsqrtf(ss + p.s.eps) * gate * l_sum;
-#pragma unroll
-        for (int c = 0; c < 64; ++c)
-            sreg[c] = pack_bf16(__uint_as_float(sreg[2 * c]) * f, __uint_as_float(sreg[2 * c + 1]) * f);
-    }
-    tmem_st32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sreg[0]));
-    tmem_st32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[32]));
-    tmem_wait_st();
-    tc_fence_before();
-    mbar_arrive(bar_p);
-
-    // ---- epilogue: O_t / l -> bf16 -> global                                   (Eq. 6-7)
-    if (!wait_bar(bars + 8 * kBarOFinal, 0, ab, 40 + t)) return;
-    tc_fence_after();
-    const float inv_l = 1.0f / l_sum;
-    __nv_bfloat16* orow = p.out + (((size_t)b * L + (valid_row ? row : 0)) * H + h) * kTile;
-#pragma unroll 1
-    for (int c = 0; c < 4; ++c) {
-        uint32_t o[32];
-        tmem_ld32(o_addr + c * 32, o);
-        tmem_wait_ld();
-        if (valid_row) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                uint4 v;
-                v.x = pack_bf16(__uint_as_float(o[e * 8 + 0]) * inv_l, __uint_as_float(o[e * 8 + 1]) * inv_l);
-                v.y = pack_bf16(__uint_as_float(o[e * 8 + 2]) * inv_l, __uint_as_float(o[e * 8 + 3]) * inv_l);
-                v.z = pack_bf16(__uint_as_float(o[e * 8 + 4]) * inv_l, __uint_as_float(o[e * 8 + 5]) * inv_l);
-                v.w = pack_bf16(__uint_as_float(o[e * 8 + 6]) * inv_l, __uint_as_float(o[e * 8 + 7]) * inv_l);
-                *reinterpret_cast<uint4*>(orow + c * 32 + e * 8) = v;
-            }
+            tc_fence_before();
         }
     }
-    tc_fence_before();
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -271,32 +450,33 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const uint32_t bars = smem_base + kOffBars;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffBars + kNumBars * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffBars + kNumBars * 8 + 4);
+    volatile int* item_slots = reinterpret_cast<volatile int*>(smem + kOffBars + kNumBars * 8 + 8);
     const Abort ab{abort_flag, p.status};
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int pair = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-    const int L = p.s.L, H = p.s.H;
-    const int q_row0 = pair * 2 * kTile;
-    const bool two = q_row0 + kTile < L;   // the pair's second tile exists
     const int n_kv = p.n_kv;
-    const int n_it = n_kv + 1;             // key tiles + the inter-branch iteration
 
     if (threadIdx.x == 0) {
         mbar_init(bars + 8 * kBarQFull, 1);
+        mbar_init(bars + 8 * kBarQFree, 2);
         mbar_init(bars + 8 * kBarQRot0, 128);
         mbar_init(bars + 8 * kBarQRot1, 128);
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bars + 8 * (kBarFull0 + s), 1);
-            mbar_init(bars + 8 * (kBarEmpty0 + s), 1);
+            mbar_init(bars + 8 * (kBarEmpty0 + s), 2);   // both MMA issuers release every entry
         }
         mbar_init(bars + 8 * kBarSFull0, 1);
         mbar_init(bars + 8 * kBarSFull1, 1);
         mbar_init(bars + 8 * kBarPFull0, 128);
         mbar_init(bars + 8 * kBarPFull1, 128);
-        mbar_init(bars + 8 * kBarOFinal, 1);
+        mbar_init(bars + 8 * kBarOFinal0, 1);
+        mbar_init(bars + 8 * kBarOFinal1, 1);
+        mbar_init(bars + 8 * kBarTok0, 128);
+        mbar_init(bars + 8 * kBarTok1, 128);
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async_smem();
+        if (blockIdx.x == 0) *p.sched_next = 0;   // the next launch starts from a clean counter
     }
     if (warp == 9) {
         tmem_alloc(smem_u32(tmem_slot), 512);
@@ -308,128 +488,216 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp < 8) {
-        const int t = warp >> 2;
-        softmax_role(p, smem, bars, tmem_base, ab, t, (warp & 3) * 32 + lane, warp & 3, b, h,
-                     q_row0 + t * kTile, t == 0 || two);
-    } else if (warp == 8) {
-        // ---------------- TMA producer ----------------
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
+        softmax_role(p, smem, bars, tmem_base, ab, item_slots, warp >> 2, (warp & 3) * 32 + lane, warp & 3);
+    } else {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+    }
+    if (warp == 8) {
+        // ---------------- TMA producer and scheduler ----------------
         if (lane == 0) {
             prefetch_tensormap(&tm_q);
             prefetch_tensormap(&tm_k);
             prefetch_tensormap(&tm_v);
+            prefetch_tensormap(&tm_w);
+            prefetch_tensormap(&tm_s);
             const uint32_t bar_q = bars + 8 * kBarQFull;
-            mbar_expect_tx(bar_q, two ? 2 * kTileBytes : kTileBytes);
-            for (int t = 0; t < (two ? 2 : 1); ++t) {
-                uint32_t dst = smem_base + kOffQRaw + t * kTileBytes;
-                tma_load_4d(dst, &tm_q, bar_q, 0, h, q_row0 + t * kTile, b);
-                tma_load_4d(dst + kHalfBytes, &tm_q, bar_q, 64, h, q_row0 + t * kTile, b);
-            }
-            const int n_loads = 2 * n_kv + 2;
-            int n = 0;
+            uint32_t n = 0;       // ring entries produced so far (all items)
             bool ok = true;
-            for (; n < n_loads && ok; ++n) {
-                const int slot = n % kStages;
-                if (n >= kStages)
-                    ok = wait_bar(bars + 8 * (kBarEmpty0 + slot), (uint32_t)(((n / kStages) - 1) & 1), ab, 50);
+            bool q_in_flight = false;
+            int id = (int)blockIdx.x;
+            for (uint32_t item = 0; ok; ++item) {
+                if (item > 0) ok = wait_bar(bars + 8 * kBarQFree, (item - 1) & 1, ab, 50);
                 if (!ok) break;
-                const uint32_t bar = bars + 8 * (kBarFull0 + slot);
-                const uint32_t dst = smem_base + kOffRing + slot * kTileBytes;
-                mbar_expect_tx(bar, kTileBytes);
-                if (n < 2 * n_kv) {
-                    const CUtensorMap* tm = (n & 1) ? &tm_v : &tm_k;
-                    const int row0 = (n >> 1) * kTile;
-                    tma_load_4d(dst, tm, bar, 0, h, row0, b);
-                    tma_load_4d(dst + kHalfBytes, tm, bar, 64, h, row0, b);
-                } else if (n == 2 * n_kv) {
-                    tma_load_2d(dst, &tm_w, bar, 0, h * kTile);
-                    tma_load_2d(dst + kHalfBytes, &tm_w, bar, 64, h * kTile);
-                } else {
-                    tma_load_2d(dst, &tm_s, bar, 0, (b * H + h) * kTile);
-                    tma_load_2d(dst + kHalfBytes, &tm_s, bar, 64, (b * H + h) * kTile);
+                if (id >= p.n_items) {
+                    item_slots[item & 1] = -1;
+                    mbar_arrive(bar_q);
+                    break;
                 }
-            }
-            if (!ok || *abort_flag) {
-                // do not leave the CTA while bulk copies into its shared memory are in flight
-                drain_bar(bar_q, 0);
-                for (int m = (n > kStages ? n - kStages : 0); m < n; ++m)
-                    drain_bar(bars + 8 * (kBarFull0 + m % kStages), (uint32_t)((m / kStages) & 1));
-            }
-        }
-    } else {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            constexpr uint32_t idesc_qk = idesc_bf16(kTile, kTile, 0, 0);  // A, B K-major
-            constexpr uint32_t idesc_pv = idesc_bf16(kTile, kTile, 0, 1);  // A in TMEM, B N-contiguous
-            const bool rotated = p.rope_cos != nullptr;
-            const uint32_t q_op = smem_base + (rotated ? kOffQRot : kOffQRaw);
-            const uint32_t q_raw = smem_base + kOffQRaw;
-            const uint32_t s_col[2] = {tmem_base, tmem_base + kTile};
-            const uint32_t o_col[2] = {tmem_base + 2 * kTile, tmem_base + 3 * kTile};
-            const int ntile = two ? 2 : 1;
-
-            // S_t (or U_t) = A_t * B^T with both operands K-major, 8 k-steps of 16
-            auto issue_qk = [&](int t, uint32_t a_tile, uint32_t b_tile) {
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    uint32_t koff = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                    mma_ss(s_col[t], smem_desc_sw128(a_tile + koff, 16), smem_desc_sw128(b_tile + koff, 16),
-                           idesc_qk, ks > 0);
-                }
-            };
-            // O_t (+)= P_t * V with P in TMEM and V rows = contraction index, 8 k-steps of 16
-            auto issue_pv = [&](int t, uint32_t v_tile, bool accumulate) {
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    mma_ts(o_col[t], s_col[t] + ks * 8, smem_desc_sw128(v_tile + ks * 2048, kHalfBytes),
-                           idesc_pv, (accumulate || ks > 0) ? 1u : 0u);
-            };
-
-            bool ok = wait_bar(bars + 8 * kBarQFull, 0, ab, 60);
-            for (int t = 0; t < ntile && ok; ++t) ok = wait_bar(bars + 8 * (kBarQRot0 + t), 0, ab, 61);
-            tc_fence_after();
-            int cons = 0;   // ring entries consumed so far
-            if (ok) ok = wait_bar(bars + 8 * (kBarFull0 + 0), 0, ab, 62);
-            if (ok) {
-                tc_fence_after();
-                const uint32_t k_tile = smem_base + kOffRing;
+                item_slots[item & 1] = id;
+                const Item it = decode_item(id, p);
+                const int ntile = it.two ? 2 : 1;
+                mbar_expect_tx(bar_q, ntile * kTileBytes);
+                q_in_flight = true;
                 for (int t = 0; t < ntile; ++t) {
-                    issue_qk(t, (n_kv > 0 ? q_op : q_raw) + t * kTileBytes, k_tile);
-                    mma_commit(bars + 8 * (kBarSFull0 + t));
+                    uint32_t dst = smem_base + kOffQ + t * kTileBytes;
+                    tma_load_4d(dst, &tm_q, bar_q, 0, it.h, it.q_row0 + t * kTile, it.b);
+                    tma_load_4d(dst + kHalfBytes, &tm_q, bar_q, 64, it.h, it.q_row0 + t * kTile, it.b);
                 }
-                mma_commit(bars + 8 * (kBarEmpty0 + 0));
-                cons = 1;
-            }
-            for (int j = 0; j < n_it && ok; ++j) {
-                const int vslot = cons % kStages;
-                const uint32_t v_tile = smem_base + kOffRing + vslot * kTileBytes;
-                ok = wait_bar(bars + 8 * (kBarFull0 + vslot), (uint32_t)((cons / kStages) & 1), ab, 63);
-                if (!ok) break;
-                const bool has_next = j + 1 < n_it;
-                const int kslot = (cons + 1) % kStages;
-                const uint32_t k_tile = smem_base + kOffRing + kslot * kTileBytes;
-                const uint32_t a_next = (j + 1 == n_kv) ? q_raw : q_op;   // the last "S" is Q W
-                for (int t = 0; t < ntile && ok; ++t) {
-                    ok = wait_bar(bars + 8 * (kBarPFull0 + t), (uint32_t)(j & 1), ab, 64 + t);
+                // ring entries: K_0 V_0 ... K_{n-1} V_{n-1} | W | Qraw_0 [Qraw_1] | S
+                const int entries = 2 * n_kv + 2 + ntile;
+                for (int e = 0; e < entries && ok; ++e, ++n) {
+                    const uint32_t slot = n % kStages;
+                    if (n >= (uint32_t)kStages)
+                        ok = wait_bar(bars + 8 * (kBarEmpty0 + slot), ((n / kStages) - 1) & 1, ab, 51);
                     if (!ok) break;
-                    tc_fence_after();
-                    issue_pv(t, v_tile, j > 0);
-                    if (has_next) {
-                        if (t == 0) {
-                            ok = wait_bar(bars + 8 * (kBarFull0 + kslot),
-                                          (uint32_t)(((cons + 1) / kStages) & 1), ab, 66);
-                            if (!ok) break;
-                            tc_fence_after();
-                        }
-                        issue_qk(t, a_next + t * kTileBytes, k_tile);
-                        mma_commit(bars + 8 * (kBarSFull0 + t));
+                    const uint32_t bar = bars + 8 * (kBarFull0 + slot);
+                    const uint32_t dst = smem_base + kOffRing + slot * kTileBytes;
+                    mbar_expect_tx(bar, kTileBytes);
+                    ARL2_STAMP(blockIdx.x == 0 && item == 0 && e >= 16 && e < 20, 56 + (e - 16));
+                    if (e < 2 * n_kv) {
+                        const CUtensorMap* tm = (e & 1) ? &tm_v : &tm_k;
+                        const int row0 = (e >> 1) * kTile;
+                        tma_load_4d(dst, tm, bar, 0, it.h, row0, it.b);
+                        tma_load_4d(dst + kHalfBytes, tm, bar, 64, it.h, row0, it.b);
+                    } else if (e == 2 * n_kv) {
+                        tma_load_2d(dst, &tm_w, bar, 0, it.h * kTile);
+                        tma_load_2d(dst + kHalfBytes, &tm_w, bar, 64, it.h * kTile);
+                    } else if (e < 2 * n_kv + 1 + ntile) {
+                        const int t = e - (2 * n_kv + 1);
+                        tma_load_4d(dst, &tm_q, bar, 0, it.h, it.q_row0 + t * kTile, it.b);
+                        tma_load_4d(dst + kHalfBytes, &tm_q, bar, 64, it.h, it.q_row0 + t * kTile, it.b);
+                    } else {
+                        tma_load_2d(dst, &tm_s, bar, 0, (it.b * p.s.H + it.h) * kTile);
+                        tma_load_2d(dst + kHalfBytes, &tm_s, bar, 64, (it.b * p.s.H + it.h) * kTile);
                     }
                 }
                 if (!ok) break;
-                mma_commit(bars + 8 * (kBarEmpty0 + vslot));
-                if (has_next) mma_commit(bars + 8 * (kBarEmpty0 + kslot));
-                cons += has_next ? 2 : 1;
+                id = (int)gridDim.x + (int)atomicAdd(p.sched_counter, 1u);
             }
-            if (ok) mma_commit(bars + 8 * kBarOFinal);
+            if (!ok || *abort_flag) {
+                // do not leave the CTA while bulk copies into its shared memory are in flight
+                if (q_in_flight) {
+                    drain_bar(bar_q, 0);
+                    drain_bar(bar_q, 1);
+                }
+                for (uint32_t m = (n > (uint32_t)kStages ? n - kStages : 0); m < n; ++m)
+                    drain_bar(bars + 8 * (kBarFull0 + m % kStages), (m / kStages) & 1);
+            }
+        }
+    } else if (warp == 9 || warp == 10) {
+        // ---------------- MMA issuers: warp 9 drives query tile 0, warp 10 tile 1 ----------------
+        // Issuing a tcgen05.mma holds the thread until the tensor pipe accepts it, and every
+        // wait / commit between two MMAs is time the pipe may idle; with one issuer per tile the
+        // synchronisation of one tile overlaps the MMAs of the other.  Both issuers walk the
+        // same sequence of ring entries and both release every entry (the empty barriers count
+        // two arrivals), whether or not they read it.
+        if (lane == 0) {
+            const int t = warp - 9;
+            constexpr uint32_t idesc_qk = idesc_bf16(kTile, kTile, 0, 0);  // A, B K-major
+            constexpr uint32_t idesc_pv = idesc_bf16(kTile, kTile, 0, 1);  // A in TMEM, B N-contiguous
+            const uint32_t q_tile = smem_base + kOffQ + t * kTileBytes;
+            const uint32_t s_col = tmem_base + t * kTile;
+            const uint32_t o_col = tmem_base + 2 * kTile + t * kTile;
+            const uint32_t bar_s = bars + 8 * (kBarSFull0 + t);
+            const uint32_t bar_p = bars + 8 * (kBarPFull0 + t);
+
+            // Matrix descriptors are built once: the high word is constant (stride between 8-row
+            // groups, version, swizzle) and a k-step only adds to the 16-byte-unit start address.
+            const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0, 0) >> 32);
+            constexpr uint32_t kLboK = 1u << 16;                                // K-major: unused field
+            constexpr uint32_t kLboMN = (uint32_t)(kHalfBytes >> 4) << 16;      // 64-column groups of V
+            auto desc64 = [&](uint32_t lo) {
+                uint64_t d;
+                asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(desc_hi));
+                return d;
+            };
+            // S_t (or U_t) = A_t * B^T with both operands K-major, 8 k-steps of 16
+            auto issue_qk = [&](uint32_t a_tile, uint32_t b_tile) {
+                const uint32_t a_lo = (a_tile >> 4) | kLboK, b_lo = (b_tile >> 4) | kLboK;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t koff = (uint32_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
+                    mma_ss(s_col, desc64(a_lo + koff), desc64(b_lo + koff), idesc_qk, ks > 0);
+                }
+            };
+            // O_t (+)= P_t * V with P in TMEM and V rows = contraction index, 8 k-steps of 16
+            auto issue_pv = [&](uint32_t v_tile, bool accumulate) {
+                const uint32_t v_lo = (v_tile >> 4) | kLboMN;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    mma_ts(o_col, s_col + ks * 8, desc64(v_lo + (uint32_t)(ks * (2048 >> 4))), idesc_pv,
+                           (accumulate || ks > 0) ? 1u : 0u);
+            };
+            auto slot_addr = [&](uint32_t entry) { return smem_base + kOffRing + (entry % kStages) * kTileBytes; };
+            auto wait_full = [&](uint32_t entry, int site) {
+                return wait_bar(bars + 8 * (kBarFull0 + entry % kStages), (entry / kStages) & 1, ab, site);
+            };
+            auto release = [&](uint32_t entry) { mma_commit(bars + 8 * (kBarEmpty0 + entry % kStages)); };
+
+            uint32_t cons = 0;        // ring entries consumed so far (all items)
+            uint32_t p_cnt = 0;       // phases of bar_p consumed
+            uint32_t qrot_cnt = 0, of_cnt = 0;
+            bool ok = true;
+            for (uint32_t item = 0; ok; ++item) {
+                ok = wait_bar(bars + 8 * kBarQFull, item & 1, ab, 60);
+                if (!ok) break;
+                const int id = item_slots[item & 1];
+                if (id < 0) break;
+                const Item it = decode_item(id, p);
+                const int ntile = it.two ? 2 : 1;
+                const bool active = t < ntile;
+                if (active) {
+                    ok = wait_bar(bars + 8 * (kBarQRot0 + t), qrot_cnt & 1, ab, 61);
+                    ++qrot_cnt;
+                    if (!ok) break;
+                }
+                // S_t(0) = Q~_t K_0^T
+                ok = wait_full(cons, 62);
+                if (!ok) break;
+                if (active) {
+                    tc_fence_after();
+                    issue_qk(q_tile, slot_addr(cons));
+                    mma_commit(bar_s);
+                }
+                release(cons);
+                ++cons;
+                if (n_kv == 1) mma_commit(bars + 8 * kBarQFree);
+
+                for (int j = 0; j < n_kv && ok; ++j) {
+                    const uint32_t v_entry = cons;              // V_j
+                    const bool next_is_kv = j + 1 < n_kv;       // else the inter-branch "S" = Q W
+                    const uint32_t b_entry = cons + 1;          // K_{j+1} or W
+#ifdef ARL2_TRACE
+                    const bool tr = blockIdx.x == 0 && item == 0 && (j == 8 || j == 9);
+                    const int ts = 40 + t * 8 + (j - 8) * 4;
+#endif
+                    ok = wait_full(v_entry, 63);
+                    if (ok) ok = wait_full(b_entry, 66);
+                    if (ok && !next_is_kv)
+                        for (int u = 0; u < ntile && ok; ++u) ok = wait_full(b_entry + 1 + u, 68);   // raw Q tiles
+                    if (!ok) break;
+                    if (active) {
+                        ARL2_STAMP(tr, ts + 0);
+                        ok = wait_bar(bar_p, p_cnt & 1, ab, 64 + t);
+                        ++p_cnt;
+                        if (!ok) break;
+                        tc_fence_after();
+                        ARL2_STAMP(tr, ts + 1);
+                        issue_pv(slot_addr(v_entry), j > 0);
+                        issue_qk(next_is_kv ? q_tile : slot_addr(b_entry + 1 + t), slot_addr(b_entry));
+                        mma_commit(bar_s);
+                        ARL2_STAMP(tr, ts + 2);
+                    }
+                    release(v_entry);
+                    release(b_entry);
+                    if (next_is_kv) {
+                        cons += 2;
+                        if (j + 1 == n_kv - 1) mma_commit(bars + 8 * kBarQFree);   // last use of Q~
+                    } else {
+                        for (int u = 0; u < ntile; ++u) release(b_entry + 1 + u);
+                        cons += 2 + ntile;
+                    }
+                }
+                if (!ok) break;
+                // inter branch: O_t += Q''_t S
+                ok = wait_full(cons, 69);
+                if (!ok) break;
+                if (active) {
+                    ok = wait_bar(bar_p, p_cnt & 1, ab, 70 + t);
+                    ++p_cnt;
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(slot_addr(cons), true);
+                }
+                release(cons);
+                ++cons;
+                if (active) {
+                    mma_commit(bars + 8 * (kBarOFinal0 + t));
+                    ++of_cnt;
+                }
+            }
+            (void)of_cnt;
         }
     }
 
@@ -527,7 +795,14 @@ int tc_prepare_map(const void* w, __nv_bfloat16* w_op, int H, cudaStream_t st)
 int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* state_bf16, cudaStream_t st)
 {
     static bool attr_set = false;
+    static int num_sms = 0;
     if (!attr_set) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0) {
+            set_error("cannot read the SM count");
+            return ARL2_ERR_CUDA;
+        }
         cudaError_t e = cudaFuncSetAttribute(tc_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) { set_error("cudaFuncSetAttribute(tc_step_kernel, %d): %s", kSmemBytes, cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
         attr_set = true;
@@ -546,8 +821,13 @@ int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* 
     p.out = static_cast<__nv_bfloat16*>(a.out);
     p.status = a.status;
     p.n_kv = (a.s.L + kTile - 1) / kTile;
-    const int n_qtiles = p.n_kv;
-    dim3 grid((n_qtiles + 1) / 2, a.s.H, a.s.B);
+    const int bh = a.s.B * a.s.H;
+    p.n_pair_items = bh * (p.n_kv / 2);
+    p.n_items = p.n_pair_items + ((p.n_kv & 1) ? bh : 0);
+    // two item counters alternate between launches: a launch consumes one and clears the other
+    p.sched_counter = a.status + kStatusSched + (a.launch_parity & 1);
+    p.sched_next = a.status + kStatusSched + ((a.launch_parity + 1) & 1);
+    const int grid = p.n_items < num_sms ? p.n_items : num_sms;
     tc_step_kernel<<<grid, kThreads, kSmemBytes, st>>>(tm_q, tm_k, tm_v, tm_w, tm_s, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_error("launch of tc_step_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
