@@ -185,8 +185,10 @@ int arl2_create(const arl2_config* cfg, void* d_state, void* d_workspace, size_t
     if (r == ARL2_OK && ctx->use_tc) {
         // operand copies the tensor-core kernels read: identity feature maps until
         // arl2_set_params, and the bf16 mirror of whatever the state buffer holds now
-        r = account(ctx, tc_prepare_map(nullptr, reinterpret_cast<__nv_bfloat16*>(ctx->ws + lay.wq_op),
-                                        cfg->H, as_stream(stream)));
+        const size_t ops[3] = {lay.wq_op, lay.wk_op, lay.wv_op};
+        for (int i = 0; i < 3 && r == ARL2_OK; ++i)
+            r = account(ctx, tc_prepare_map(nullptr, reinterpret_cast<__nv_bfloat16*>(ctx->ws + ops[i]),
+                                            cfg->H, as_stream(stream)));
         if (r == ARL2_OK)
             r = account(ctx, state_to_bf16(ctx->state,
                                            reinterpret_cast<__nv_bfloat16*>(ctx->ws + lay.state_bf16),
@@ -211,9 +213,15 @@ int arl2_set_params(arl2_ctx* ctx, const void* d_wphi_q, const void* d_wphi_k, c
     }
     ctx->wq = d_wphi_q; ctx->wk = d_wphi_k; ctx->wv = d_wphi_v;
     ctx->rope_cos = d_rope_cos; ctx->rope_sin = d_rope_sin;
-    if (ctx->use_tc)
-        return account(ctx, tc_prepare_map(d_wphi_q, reinterpret_cast<__nv_bfloat16*>(ctx->ws + ctx->lay.wq_op),
-                                           ctx->cfg.H, as_stream(stream)));
+    if (ctx->use_tc) {
+        const void* src[3] = {d_wphi_q, d_wphi_k, d_wphi_v};
+        const size_t ops[3] = {ctx->lay.wq_op, ctx->lay.wk_op, ctx->lay.wv_op};
+        for (int i = 0; i < 3; ++i) {
+            int r = account(ctx, tc_prepare_map(src[i], reinterpret_cast<__nv_bfloat16*>(ctx->ws + ops[i]),
+                                                ctx->cfg.H, as_stream(stream)));
+            if (r != ARL2_OK) return r;
+        }
+    }
     return ARL2_OK;
 }
 
@@ -291,6 +299,14 @@ int arl2_commit(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
                                : nullptr;
     a.nsplit = ctx->lay.nsplit;
     a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status);
+    if ((reinterpret_cast<uintptr_t>(d_k_clean) | reinterpret_cast<uintptr_t>(d_v_clean)) % 16 != 0) {
+        set_error("commit: k_clean and v_clean must be 16-byte aligned");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    if (ctx->use_tc)
+        return account(ctx, tc_commit(a, reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wk_op),
+                                      reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wv_op),
+                                      as_stream(stream)));
     return account(ctx, simt_commit(a, ctx->cfg.io_dtype, as_stream(stream)));
 }
 

@@ -74,6 +74,8 @@ bool tc_supported(const arl2_config& c);
 int tc_prepare_map(const void* w, __nv_bfloat16* w_op, int H, cudaStream_t st);
 int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* state_bf16,
             cudaStream_t st);
+int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat16* wv_op,
+              cudaStream_t st);   // partial sums on tensor cores, then commit_reduce
 
 void set_error(const char* fmt, ...);
 

@@ -709,6 +709,243 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Commit kernel (Eq. 3, Eq. 4 in its gated-linear form): one CTA per (stream b, head h, chunk of
+// 512 tokens), 128 threads.  Per 128-token tile:
+//   U_k = K_c W_phi_k, U_v = V_c W_phi_v            two MMAs into TMEM (columns 0-127, 128-255)
+//   K'  = L2Norm(RoPE(U_k)), V' = U_v               one thread per token; written as bf16 over
+//                                                   the raw tiles, in the swizzled tile layout
+//   dS += K'^T V'                                   MMA with both operands token-major (the
+//                                                   contraction runs over the tile's tokens)
+// dS (TMEM columns 256-383, fp32) is written to this chunk's slot of the partial-sum buffer; the
+// reduce kernel adds the chunks in a fixed order and applies the gated decay.
+// ---------------------------------------------------------------------------------------------
+constexpr int kCOffWk = 0;
+constexpr int kCOffWv = kTileBytes;
+constexpr int kCOffPair = 2 * kTileBytes;                  // 2 pairs of (K tile, V tile)
+constexpr int kCOffBars = kCOffPair + 4 * kTileBytes;
+constexpr int kCommitSmemBytes = kCOffBars + 128 + 1024;
+constexpr int kCommitThreads = 128;
+
+enum CBar : int { kCBarW = 0, kCBarFull0, kCBarFull1, kCBarU, kCBarS, kCNumBars };
+
+struct TcCommitParams {
+    Shape s;
+    const float* rope_cos;
+    const float* rope_sin;
+    float* partials;     // [B, H, nsplit, 128, 128] fp32
+    uint32_t* status;
+    int nsplit;
+};
+
+__global__ void __launch_bounds__(kCommitThreads, 1)
+tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                 const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv,
+                 const TcCommitParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                               ~static_cast<uintptr_t>(1023));
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t bars = smem_base + kCOffBars;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kCOffBars + kCNumBars * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kCOffBars + kCNumBars * 8 + 4);
+    const Abort ab{abort_flag, p.status};
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int L = p.s.L, H = p.s.H;
+    const int l0 = split * kCommitChunk;
+    const int l1 = min(L, l0 + kCommitChunk);
+    const int ntiles = (l1 - l0 + kTile - 1) / kTile;
+
+    if (tid == 0) {
+        for (int i = 0; i < kCNumBars; ++i) mbar_init(bars + 8 * i, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+        fence_proxy_async_smem();
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+
+    auto load_pair = [&](int i) {   // tile i of the chunk into pair i & 1
+        const uint32_t bar = bars + 8 * (kCBarFull0 + (i & 1));
+        const uint32_t dst = smem_base + kCOffPair + (i & 1) * 2 * kTileBytes;
+        mbar_expect_tx(bar, 2 * kTileBytes);
+        tma_load_4d(dst, &tm_k, bar, 0, h, l0 + i * kTile, b);
+        tma_load_4d(dst + kHalfBytes, &tm_k, bar, 64, h, l0 + i * kTile, b);
+        tma_load_4d(dst + kTileBytes, &tm_v, bar, 0, h, l0 + i * kTile, b);
+        tma_load_4d(dst + kTileBytes + kHalfBytes, &tm_v, bar, 64, h, l0 + i * kTile, b);
+    };
+
+    bool ok = true;
+    int loads_issued = 0;
+    if (tid == 0) {
+        prefetch_tensormap(&tm_k);
+        prefetch_tensormap(&tm_v);
+        const uint32_t bar_w = bars + 8 * kCBarW;
+        mbar_expect_tx(bar_w, 2 * kTileBytes);
+        tma_load_2d(smem_base + kCOffWk, &tm_wk, bar_w, 0, h * kTile);
+        tma_load_2d(smem_base + kCOffWk + kHalfBytes, &tm_wk, bar_w, 64, h * kTile);
+        tma_load_2d(smem_base + kCOffWv, &tm_wv, bar_w, 0, h * kTile);
+        tma_load_2d(smem_base + kCOffWv + kHalfBytes, &tm_wv, bar_w, 64, h * kTile);
+        for (int i = 0; i < 2 && i < ntiles; ++i, ++loads_issued) load_pair(i);
+        ok = wait_bar(bar_w, 0, ab, 80);
+    }
+
+    const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0, 0) >> 32);
+    constexpr uint32_t kLboK = 1u << 16;
+    constexpr uint32_t kLboMN = (uint32_t)(kHalfBytes >> 4) << 16;
+    auto desc64 = [&](uint32_t lo) {
+        uint64_t d;
+        asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(desc_hi));
+        return d;
+    };
+    constexpr uint32_t idesc_u = idesc_bf16(kTile, kTile, 0, 0);    // tile x map: both K-major
+    constexpr uint32_t idesc_ds = idesc_bf16(kTile, kTile, 1, 1);   // K'^T V': both token-major
+
+    uint32_t sreg[128];
+    for (int i = 0; i < ntiles; ++i) {
+        const int s = i & 1;
+        uint8_t* pair = smem + kCOffPair + s * 2 * kTileBytes;
+        const uint32_t pair_addr = smem_base + kCOffPair + s * 2 * kTileBytes;
+        if (tid == 0 && ok) {
+            ok = wait_bar(bars + 8 * (kCBarFull0 + s), (uint32_t)((i >> 1) & 1), ab, 81);
+            if (ok) {
+                tc_fence_after();
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {   // U_k then U_v
+                    const uint32_t a_lo = ((pair_addr + u * kTileBytes) >> 4) | kLboK;
+                    const uint32_t b_lo = ((smem_base + (u ? kCOffWv : kCOffWk)) >> 4) | kLboK;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t koff = (uint32_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
+                        mma_ss(tmem_base + u * kTile, desc64(a_lo + koff), desc64(b_lo + koff), idesc_u, ks > 0);
+                    }
+                }
+                mma_commit(bars + 8 * kCBarU);
+            }
+        }
+        if (!wait_bar(bars + 8 * kCBarU, (uint32_t)(i & 1), ab, 82)) break;
+        tc_fence_after();
+
+        const int r = tid;                       // token row of the tile
+        const int row = l0 + i * kTile + r;
+        const bool valid_row = row < L;
+        // ---- K' = L2Norm(RoPE(U_k))
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            tmem_ld32(lane_base + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
+        tmem_wait_ld();
+        if (p.rope_cos != nullptr && valid_row) {
+            const float* cs = p.rope_cos + (size_t)row * (kTile / 2);
+            const float* sn = p.rope_sin + (size_t)row * (kTile / 2);
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+                float4 cv = *reinterpret_cast<const float4*>(cs + c * 4);
+                float4 sv = *reinterpret_cast<const float4*>(sn + c * 4);
+                float cc[4] = {cv.x, cv.y, cv.z, cv.w}, s4[4] = {sv.x, sv.y, sv.z, sv.w};
+#pragma unroll
+                for (int m = 0; m < 4; ++m) {
+                    float x0 = __uint_as_float(sreg[c * 8 + 2 * m]);
+                    float x1 = __uint_as_float(sreg[c * 8 + 2 * m + 1]);
+                    sreg[c * 8 + 2 * m] = __float_as_uint(x0 * cc[m] - x1 * s4[m]);
+                    sreg[c * 8 + 2 * m + 1] = __float_as_uint(x0 * s4[m] + x1 * cc[m]);
+                }
+            }
+        }
+        {
+            float ss4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+            for (int c = 0; c < 128; c += 4) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    ss4[k] = fmaf(__uint_as_float(sreg[c + k]), __uint_as_float(sreg[c + k]), ss4[k]);
+            }
+            const float f = rsqrtf((ss4[0] + ss4[1]) + (ss4[2] + ss4[3]) + p.s.eps);
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+                uint4 v;
+                v.x = pack_bf16(__uint_as_float(sreg[c * 8 + 0]) * f, __uint_as_float(sreg[c * 8 + 1]) * f);
+                v.y = pack_bf16(__uint_as_float(sreg[c * 8 + 2]) * f, __uint_as_float(sreg[c * 8 + 3]) * f);
+                v.z = pack_bf16(__uint_as_float(sreg[c * 8 + 4]) * f, __uint_as_float(sreg[c * 8 + 5]) * f);
+                v.w = pack_bf16(__uint_as_float(sreg[c * 8 + 6]) * f, __uint_as_float(sreg[c * 8 + 7]) * f);
+                const int off = (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+                *reinterpret_cast<uint4*>(pair + off) = v;
+            }
+        }
+        // ---- V' = U_v
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            tmem_ld32(lane_base + kTile + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
+        tmem_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+            uint4 v;
+            v.x = pack_bf16(__uint_as_float(sreg[c * 8 + 0]), __uint_as_float(sreg[c * 8 + 1]));
+            v.y = pack_bf16(__uint_as_float(sreg[c * 8 + 2]), __uint_as_float(sreg[c * 8 + 3]));
+            v.z = pack_bf16(__uint_as_float(sreg[c * 8 + 4]), __uint_as_float(sreg[c * 8 + 5]));
+            v.w = pack_bf16(__uint_as_float(sreg[c * 8 + 6]), __uint_as_float(sreg[c * 8 + 7]));
+            const int off = (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+            *reinterpret_cast<uint4*>(pair + kTileBytes + off) = v;
+        }
+        fence_proxy_async_smem();
+        tc_fence_before();
+        __syncthreads();
+
+        if (tid == 0 && ok) {
+            tc_fence_after();
+            const uint32_t a_lo = (pair_addr >> 4) | kLboMN;
+            const uint32_t b_lo = ((pair_addr + kTileBytes) >> 4) | kLboMN;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks)   // 16 tokens per step
+                mma_ss(tmem_base + 2 * kTile, desc64(a_lo + (uint32_t)(ks * (2048 >> 4))),
+                       desc64(b_lo + (uint32_t)(ks * (2048 >> 4))), idesc_ds, (i > 0 || ks > 0) ? 1u : 0u);
+            mma_commit(bars + 8 * kCBarS);
+            // the pair may be overwritten (and TMEM columns 0-255 reused) once this MMA is done
+            ok = wait_bar(bars + 8 * kCBarS, (uint32_t)(i & 1), ab, 83);
+            if (ok && i + 2 < ntiles) {
+                load_pair(i + 2);
+                ++loads_issued;
+            }
+        }
+    }
+
+    // ---- epilogue: dS row d_k = tid -> this chunk's partial
+    if (ntiles > 0 && wait_bar(bars + 8 * kCBarS, (uint32_t)((ntiles - 1) & 1), ab, 84)) {
+        tc_fence_after();
+        float* dst = p.partials + ((((size_t)b * H + h) * p.nsplit + split) * kTile + tid) * kTile;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+            uint32_t o[32];
+            tmem_ld32(lane_base + 2 * kTile + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+                *reinterpret_cast<uint4*>(dst + c * 32 + e * 4) = make_uint4(o[e * 4], o[e * 4 + 1], o[e * 4 + 2], o[e * 4 + 3]);
+        }
+    }
+    if (tid == 0 && (!ok || *abort_flag)) {
+        // leave no bulk copy in flight into this CTA's shared memory
+        drain_bar(bars + 8 * kCBarW, 0);
+        for (int m = (loads_issued > 2 ? loads_issued - 2 : 0); m < loads_issued; ++m)
+            drain_bar(bars + 8 * (kCBarFull0 + (m & 1)), (uint32_t)((m >> 1) & 1));
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
 // out[h][o][i] = w[h][i][o] (bf16), or the identity when w is null: the K-major B operand of
 // U = Q W_phi (B[n][k] = W[k][n]).
 __global__ void transpose_map_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ out,
@@ -832,6 +1069,36 @@ int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* 
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_error("launch of tc_step_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
     return 1;
+}
+
+int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat16* wv_op, cudaStream_t st)
+{
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_commit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kCommitSmemBytes);
+        if (e != cudaSuccess) { set_error("cudaFuncSetAttribute(tc_commit_kernel, %d): %s", kCommitSmemBytes, cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
+        attr_set = true;
+    }
+    CUtensorMap tm_k, tm_v, tm_wk, tm_wv;
+    if (int r = make_map_blhd(&tm_k, a.k, a.s)) return r;
+    if (int r = make_map_blhd(&tm_v, a.v, a.s)) return r;
+    if (int r = make_map_rows(&tm_wk, wk_op, (size_t)a.s.H * kTile)) return r;
+    if (int r = make_map_rows(&tm_wv, wv_op, (size_t)a.s.H * kTile)) return r;
+    TcCommitParams p;
+    p.s = a.s;
+    p.rope_cos = a.rope_cos;
+    p.rope_sin = a.rope_sin;
+    p.partials = a.partials;
+    p.status = a.status;
+    p.nsplit = a.nsplit;
+    dim3 grid(a.nsplit, a.s.H, a.s.B);
+    tc_commit_kernel<<<grid, kCommitThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, tm_wv, p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_error("launch of tc_commit_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
+    int m = commit_reduce(a, st);
+    if (m < 0) return m;
+    return 1 + m;
 }
 
 }  // namespace arl2
