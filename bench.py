@@ -76,7 +76,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "50", "-i", str(self.index)],
+                 "-lms", "25", "-i", str(self.index)],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -203,6 +203,28 @@ def run_reference(args):
 # the CUDA arm
 # ------------------------------------------------------------------------------------------
 
+def max_over_ranks(values, world, device):
+    """Device times of the replicas -> the slowest rank's (all ranks get the same list)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
+
+
+def rank_seeds(rank):
+    """Each replica draws its own inputs: step-input seeds and the commit block index."""
+    return [s + 10 * rank for s in range(RING)], rank
+
+
+def whole_job_value(cfg, world, ms_block):
+    """tokens/s through the denoise passes of all replicas, commit time included."""
+    return world * cfg.B * cfg.L * cfg.steps / (ms_block * 1e-3)
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -227,8 +249,9 @@ def run_ours(args):
     cos, sin = (t.to(dev) for t in workload.rope_tables(cfg.L, cfg.D))
     layer.set_params(wq, wk, wv, cos, sin)
 
-    host_sets = [workload.step_inputs(cfg, 0, s + 10 * rank) for s in range(RING)]
-    host_commit = workload.commit_inputs(cfg, rank)
+    step_seeds, commit_block = rank_seeds(rank)
+    host_sets = [workload.step_inputs(cfg, 0, s) for s in step_seeds]
+    host_commit = workload.commit_inputs(cfg, commit_block)
     dev_sets = [tuple(t.to(dev) for t in hs) for hs in host_sets]
     dev_commit = tuple(t.to(dev) for t in host_commit)
     out = torch.empty(cfg.B, cfg.L, cfg.H, cfg.D, dtype=cfg.torch_dtype, device=dev)
@@ -303,25 +326,19 @@ def run_ours(args):
     h2d = cfg.steps * set_bytes + commit_bytes
     d2h = cfg.steps * out.numel() * out.element_size()
 
-    if world > 1:
-        t = torch.tensor([ms_total, ms_e2e, statistics.mean(kern_ms)], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e, kern_mean = (float(x) for x in t.tolist())
-    else:
-        kern_mean = statistics.mean(kern_ms)
+    ms_total, ms_e2e, kern_mean = max_over_ranks([ms_total, ms_e2e, statistics.mean(kern_ms)], world, dev)
 
     if rank == 0:
         pk = peaks()
-        tokens_per_block = world * cfg.B * cfg.L * cfg.steps
         ms_block = ms_total / args.steps
-        value = tokens_per_block / (ms_block * 1e-3)
+        value = whole_job_value(cfg, world, ms_block)
         timed_seconds = ms_total * 1e-3
         # a kernel timed inside a seconds-long loop runs under the power cap: sustained figure
         use_sustained = timed_seconds > 1.0
         peak = pk["bf16_tflops_sustained"] if use_sustained else pk["bf16_tflops"]
         achieved = step_flops(cfg) / (kern_mean * 1e-3) / 1e12
         traffic = None
-        tpath = os.path.join(ROOT, "profiles", "step_kernel_traffic.json")
+        tpath = os.path.join(ROOT, "profiles", "step_kernel_traffic.txt")
         if os.path.exists(tpath):
             with open(tpath) as f:
                 rec = json.load(f)
@@ -360,6 +377,7 @@ def run_ours(args):
         if world == 1 and not args.no_cpu_baseline:
             s = CpuSample(cfg)
             t = s.time_rows(s.threads)
+            t = min(t, s.time_rows(s.threads))  # the first call pays for page faults
             n_rows = max(s.threads, int(s.threads * 12.0 / max(t, 1e-6)))
             tr = s.time_rows(n_rows)
             n_heads = min(s.threads, cfg.B * cfg.H)
@@ -379,7 +397,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="long", choices=["tiny", "small", "chunked", "batched", "long"])

@@ -107,6 +107,14 @@ __device__ __forceinline__ void drain_bar(uint32_t bar, uint32_t parity)
         if (mbar_try_wait(bar, parity)) return;
 }
 
+#ifdef ARL2_TRACE_ITER
+// Per-iteration log of tuning builds run WITHOUT RoPE: the words after the status block belong
+// to the rotated-K buffer, which is unused then.
+#define ARL2_ITER(cond, slot) do { if (blockIdx.x == 0 && item < 2 && r == 0 && (cond)) p.status[64 + (slot)] = (uint32_t)clock64(); } while (0)
+#else
+#define ARL2_ITER(cond, slot) do { } while (0)
+#endif
+
 #ifdef ARL2_TRACE
 // Timeline probe for tuning builds: one thread of CTA 0 stamps the SM clock into the status
 // block for two loop iterations of its first item.  Not compiled into the product library.
@@ -219,6 +227,7 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
 
     for (uint32_t item = 0;; ++item) {
         if (!wait_bar(bars + 8 * kBarQFull, item & 1, ab, 10)) return;
+        ARL2_ITER(true, 256 + item * 16 + t * 8 + 5);
         const int id = item_slots[item & 1];
         if (id < 0) return;
         const Item it = decode_item(id, p);
@@ -252,6 +261,7 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                 fence_proxy_async_smem();
             }
             mbar_arrive(bars + 8 * (kBarQRot0 + t));
+            ARL2_ITER(true, 256 + item * 16 + t * 8 + 6);
 
             float m_ref = -INFINITY;   // reference maximum (scaled, base 2) of the probabilities
             uint64_t l2 = pack2(0.0f, 0.0f);   // running row sum relative to m_ref, two lanes
@@ -266,6 +276,7 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                 ++s_cnt;
                 tc_fence_after();
                 ARL2_STAMP(tr, ts + 1);
+                ARL2_ITER(j < 60, item * 128 + t * 64 + j);
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
                     tmem_ld32(s_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
@@ -364,8 +375,10 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
             const float l_sum = l_lo + l_hi;
 
             // ---- inter branch: U = Q W_phi_q arrives in the S columns                  (Eq. 3)
+            ARL2_ITER(true, 256 + item * 16 + t * 8 + 0);
             if (!wait_bar(bar_s, s_cnt & 1, ab, 30 + t)) return;
             ++s_cnt;
+            ARL2_ITER(true, 256 + item * 16 + t * 8 + 1);
             tc_fence_after();
 #pragma unroll
             for (int c = 0; c < 4; ++c)
@@ -411,7 +424,9 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
             mbar_arrive(bar_p);
 
             // ---- epilogue: O_t / l -> bf16 -> global                              (Eq. 6-7)
+            ARL2_ITER(true, 256 + item * 16 + t * 8 + 2);
             if (!wait_bar(bars + 8 * (kBarOFinal0 + t), of_cnt & 1, ab, 40 + t)) return;
+            ARL2_ITER(true, 256 + item * 16 + t * 8 + 3);
             ++of_cnt;
             tc_fence_after();
             const float inv_l = 1.0f / l_sum;
@@ -434,6 +449,7 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                 }
             }
             tc_fence_before();
+            ARL2_ITER(true, 256 + item * 16 + t * 8 + 4);
         }
     }
 }
