@@ -150,6 +150,38 @@ int arl2_sync_status(arl2_ctx* ctx, void* stream);
  */
 int arl2_set_profile_events(arl2_ctx* ctx, void* ev_before, void* ev_after);
 
+/*
+ * The state commit without any device allocation and without a context or workspace
+ * (the paper has no counterpart; this is a service to constrained callers).
+ *
+ * Some callers of this library may not allocate device memory at the point where they must
+ * commit: a plugin whose host owns the memory pool and forbids cudaMalloc, code running while
+ * another component is capturing work on the stream, a process that was handed exactly the
+ * layer's tensors and nothing else.  arl2_commit needs a workspace for the partial sums of its
+ * split reduction; this entry point keeps those partial sums in an array built into the
+ * library image instead (ARL2_STATIC_SCRATCH_BYTES per GPU, resident on every GPU that loads
+ * the library until the process exits) and calls no cudaMalloc, cudaFree or allocating routine.
+ *
+ * Computes exactly what arl2_commit computes (plain-FMA kernels, fp32 or bf16 I/O):
+ *   S[b,h] <- sigmoid(a[b,h]) S[b,h] + sum_l K'_l^T V'_l   on d_state [B,H,D,D] fp32 in place.
+ * d_wphi_k / d_wphi_v: [H,D,D] (in,out) io_dtype or NULL; d_rope_cos / d_rope_sin: [L,D/2] fp32
+ * or both NULL.  cfg->flags and cfg->softmax_scale are ignored.
+ *
+ * Limits and rules
+ *   - B*H*ceil(L/512)*D*D*4 bytes must fit in ARL2_STATIC_SCRATCH_BYTES; larger shapes are
+ *     rejected with ARL2_ERR_WORKSPACE and a message saying so (use arl2_commit then).
+ *   - The first call on each device looks up the array's device address (the device must be
+ *     current, as for any launch); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents.
+ *     Nothing in it needs clearing (every slot read is written first by the same call), but
+ *     two calls that overlap on the GPU (different streams, no ordering) race on it: order them.
+ */
+#define ARL2_STATIC_SCRATCH_BYTES (8u << 20)
+int arl2_commit_static_scratch(const arl2_config* cfg, void* d_state, const void* d_k_clean,
+                               const void* d_v_clean, const float* d_decay_logits,
+                               const void* d_wphi_k, const void* d_wphi_v,
+                               const float* d_rope_cos, const float* d_rope_sin, void* stream);
+
 /* Number of kernel launches this context has issued so far (all entry points). */
 uint64_t arl2_launch_count(const arl2_ctx* ctx);
 

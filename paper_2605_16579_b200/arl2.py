@@ -21,7 +21,7 @@ ARL2_FLAG_FORCE_SIMT = 1
 EXPORTS = (
     "arl2_workspace_bytes", "arl2_create", "arl2_set_params", "arl2_denoise_step", "arl2_commit",
     "arl2_reset", "arl2_get_state", "arl2_set_state", "arl2_sync_status", "arl2_launch_count",
-    "arl2_set_profile_events",
+    "arl2_set_profile_events", "arl2_commit_static_scratch",
     "arl2_step_kernel_name", "arl2_destroy", "arl2_last_error", "arl2_version",
 )
 
@@ -79,6 +79,8 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     lib.arl2_sync_status.argtypes = [vp, vp]
     lib.arl2_set_profile_events.restype = ctypes.c_int
     lib.arl2_set_profile_events.argtypes = [vp, vp, vp]
+    lib.arl2_commit_static_scratch.restype = ctypes.c_int
+    lib.arl2_commit_static_scratch.argtypes = [cp] + [vp] * 9
     lib.arl2_launch_count.restype = ctypes.c_uint64
     lib.arl2_launch_count.argtypes = [vp]
     lib.arl2_step_kernel_name.restype = ctypes.c_char_p
@@ -239,3 +241,22 @@ class Layer:
                 and tuple(t.shape) == tuple(shape) and t.dtype == dtype):
             raise Arl2Error(f"{what}: expected a contiguous CUDA tensor {tuple(shape)} {dtype}, got "
                             f"{tuple(t.shape)} {t.dtype} on {t.device}")
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def commit_static_scratch(cfg: arl2_config, state, k_clean, v_clean, decay_logits, wk=None, wv=None,
+                          rope_cos=None, rope_sin=None):
+    """arl2_commit_static_scratch: the commit for callers that may not allocate device memory.
+
+    Updates ``state`` ([B, H, D, D] fp32, CUDA) in place; no context, no workspace.  The partial
+    sums of the reduction live in an array built into the library (8 MiB per GPU), so shapes
+    with B*H*ceil(L/512)*D*D*4 bytes above that are refused, and calls that overlap on the GPU
+    must be ordered by the caller.
+    """
+    with torch.cuda.device(state.device):
+        _check(load().arl2_commit_static_scratch(ctypes.byref(cfg), _ptr(state), _ptr(k_clean),
+                                                 _ptr(v_clean), _ptr(decay_logits), _ptr(wk), _ptr(wv),
+                                                 _ptr(rope_cos), _ptr(rope_sin), _stream()),
+               "arl2_commit_static_scratch")
