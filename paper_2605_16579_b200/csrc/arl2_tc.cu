@@ -80,7 +80,7 @@ struct TcStepParams {
     uint32_t* sched_next;      // the next launch's counter: cleared by this launch
     int n_kv;                  // key tiles per head = query tiles per head
     int n_pair_items;          // B * H * (n_kv / 2): items with two query tiles
-    int n_items;               // + B * H single-tile items when n_kv is odd
+    int n_items;               // + ceil(B * H / 2) items of ragged last tiles when n_kv is odd
 };
 
 struct Abort {
@@ -178,31 +178,86 @@ __device__ __forceinline__ void exp2_poly2(float x0, float x1, float& r0, float&
     r1 = __int_as_float(__float_as_int(q1) + (__float_as_int(t1) << 23));
 }
 
+// A work item drives up to two 128-row query tiles.  A "pair" item holds two consecutive tiles of
+// one (stream, head): they share every K/V tile.  A "ragged" item holds the last, partial tiles
+// of two different (stream, head) units (or of one, when the number of units is odd): each tile
+// then streams its own K/V, W_phi_q and state through the ring.
 struct Item {
-    int b, h, q_row0;
-    bool two;   // the pair's second tile exists
+    int b[2], h[2], row0[2];
+    int ntile;    // active tiles: 1 or 2
+    bool shared;  // both tiles read the same K, V, W_phi_q and state
 };
 
 // Items [0, n_pair_items) are pairs of full tiles, (b, h)-major so that neighbours share K and V
-// in L2; the rest are the single ragged tiles, which fill the tail of the schedule.
+// in L2; the rest pack the ragged last tiles two by two.
 __device__ __forceinline__ Item decode_item(int id, const TcStepParams& p)
 {
     Item it;
-    int bh, pair;
     const int full_pairs = p.n_kv >> 1;
+    const int units = p.s.B * p.s.H;
     if (id < p.n_pair_items) {
-        bh = id / full_pairs;
-        pair = id - bh * full_pairs;
-        it.two = true;
+        const int bh = id / full_pairs;
+        const int pair = id - bh * full_pairs;
+        it.b[0] = it.b[1] = bh / p.s.H;
+        it.h[0] = it.h[1] = bh - it.b[0] * p.s.H;
+        it.row0[0] = pair * 2 * kTile;
+        it.row0[1] = it.row0[0] + kTile;
+        it.ntile = 2;
+        it.shared = true;
     } else {
-        bh = id - p.n_pair_items;
-        pair = full_pairs;
-        it.two = false;
+        const int u = id - p.n_pair_items;
+        it.ntile = (2 * u + 1 < units) ? 2 : 1;
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            const int bh = min(2 * u + t, units - 1);
+            it.b[t] = bh / p.s.H;
+            it.h[t] = bh - it.b[t] * p.s.H;
+            it.row0[t] = full_pairs * 2 * kTile;
+        }
+        it.shared = false;
     }
-    it.b = bh / p.s.H;
-    it.h = bh - it.b * p.s.H;
-    it.q_row0 = pair * 2 * kTile;
     return it;
+}
+
+// The ring entries of an item, in the order both MMA issuers walk them.
+enum EntryKind : int { kEntK = 0, kEntV, kEntW, kEntQRaw, kEntState };
+struct Entry {
+    int kind, tile, j;   // j: key tile index for K / V
+};
+// pair item:   K_0 | V_0 K_1 | V_1 K_2 | ... | V_{n-1} W Qraw_0 Qraw_1 | S
+// ragged item: K^0_0 K^1_0 | V^0_0 K^0_1 V^1_0 K^1_1 | ... | V^0_{n-1} W^0 Qraw_0 V^1_{n-1} W^1 Qraw_1 | S^0 S^1
+__device__ __forceinline__ int item_entries(const Item& it, int n_kv)
+{
+    return it.shared ? 2 * n_kv + 2 + it.ntile : it.ntile * (2 * n_kv + 3);
+}
+__device__ __forceinline__ Entry item_entry(const Item& it, int n_kv, int e)
+{
+    Entry en;
+    if (it.shared) {
+        en.tile = 0;
+        if (e == 0) { en.kind = kEntK; en.j = 0; }
+        else if (e < 2 * n_kv) { en.kind = (e & 1) ? kEntV : kEntK; en.j = (e & 1) ? (e - 1) >> 1 : e >> 1; }
+        else if (e == 2 * n_kv) { en.kind = kEntW; en.j = 0; }
+        else if (e < 2 * n_kv + 1 + it.ntile) { en.kind = kEntQRaw; en.tile = e - (2 * n_kv + 1); en.j = 0; }
+        else { en.kind = kEntState; en.j = 0; }
+    } else {
+        const int nt = it.ntile;
+        const int body = nt + 2 * nt * (n_kv - 1);   // entries before the last key iteration
+        if (e < nt) { en.kind = kEntK; en.tile = e; en.j = 0; }
+        else if (e < body) {
+            const int x = e - nt, jj = x / (2 * nt), y = x - jj * 2 * nt;
+            en.tile = y >> 1;
+            en.kind = (y & 1) ? kEntK : kEntV;
+            en.j = (y & 1) ? jj + 1 : jj;
+        } else if (e < body + 3 * nt) {
+            const int y = e - body;
+            en.tile = y / 3;
+            const int z = y - en.tile * 3;
+            en.kind = z == 0 ? kEntV : z == 1 ? kEntW : kEntQRaw;
+            en.j = n_kv - 1;
+        } else { en.kind = kEntState; en.tile = e - (body + 3 * nt); en.j = 0; }
+    }
+    return en;
 }
 
 // One softmax group thread: owns query row `r` of tile `t` of every item.
@@ -231,10 +286,10 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
         const int id = item_slots[item & 1];
         if (id < 0) return;
         const Item it = decode_item(id, p);
-        const int b = it.b, h = it.h;
-        const int row = it.q_row0 + t * kTile + r;
+        const int b = it.b[t], h = it.h[t];
+        const int row = it.row0[t] + r;
         const bool valid_row = row < L;
-        const bool active = t == 0 || it.two;
+        const bool active = t < it.ntile;
 
         if (active) {
             // ---- Q~ = RoPE(Q): rotate this thread's row of the tile in place          (Eq. 2)
@@ -322,7 +377,7 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                     }
                 }
                 const uint64_t neg_m2 = pack2(-m_ref, -m_ref);
-                if (it.two) {
+                if (it.ntile == 2) {
                     // the two groups alternate in the exponential phase, so that one group's
                     // exponentials overlap the other tile's MMAs instead of its exponentials
                     const uint32_t par = (t == 0) ? ((tok_cnt + 1) & 1) : (tok_cnt & 1);
@@ -361,7 +416,7 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                     l2 = pack2(la, lb);
                 }
 #endif
-                if (it.two) mbar_arrive(bars + 8 * (kBarTok0 + (t ^ 1)));
+                if (it.ntile == 2) mbar_arrive(bars + 8 * (kBarTok0 + (t ^ 1)));
                 ARL2_STAMP(tr, ts + 5);
                 tmem_st32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sreg[0]));
                 tmem_st32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[32]));
@@ -532,16 +587,15 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 }
                 item_slots[item & 1] = id;
                 const Item it = decode_item(id, p);
-                const int ntile = it.two ? 2 : 1;
+                const int ntile = it.ntile;
                 mbar_expect_tx(bar_q, ntile * kTileBytes);
                 q_in_flight = true;
                 for (int t = 0; t < ntile; ++t) {
                     uint32_t dst = smem_base + kOffQ + t * kTileBytes;
-                    tma_load_4d(dst, &tm_q, bar_q, 0, it.h, it.q_row0 + t * kTile, it.b);
-                    tma_load_4d(dst + kHalfBytes, &tm_q, bar_q, 64, it.h, it.q_row0 + t * kTile, it.b);
+                    tma_load_4d(dst, &tm_q, bar_q, 0, it.h[t], it.row0[t], it.b[t]);
+                    tma_load_4d(dst + kHalfBytes, &tm_q, bar_q, 64, it.h[t], it.row0[t], it.b[t]);
                 }
-                // ring entries: K_0 V_0 ... K_{n-1} V_{n-1} | W | Qraw_0 [Qraw_1] | S
-                const int entries = 2 * n_kv + 2 + ntile;
+                const int entries = item_entries(it, n_kv);
                 for (int e = 0; e < entries && ok; ++e, ++n) {
                     const uint32_t slot = n % kStages;
                     if (n >= (uint32_t)kStages)
@@ -550,22 +604,21 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     const uint32_t bar = bars + 8 * (kBarFull0 + slot);
                     const uint32_t dst = smem_base + kOffRing + slot * kTileBytes;
                     mbar_expect_tx(bar, kTileBytes);
-                    ARL2_STAMP(blockIdx.x == 0 && item == 0 && e >= 16 && e < 20, 56 + (e - 16));
-                    if (e < 2 * n_kv) {
-                        const CUtensorMap* tm = (e & 1) ? &tm_v : &tm_k;
-                        const int row0 = (e >> 1) * kTile;
-                        tma_load_4d(dst, tm, bar, 0, it.h, row0, it.b);
-                        tma_load_4d(dst + kHalfBytes, tm, bar, 64, it.h, row0, it.b);
-                    } else if (e == 2 * n_kv) {
-                        tma_load_2d(dst, &tm_w, bar, 0, it.h * kTile);
-                        tma_load_2d(dst + kHalfBytes, &tm_w, bar, 64, it.h * kTile);
-                    } else if (e < 2 * n_kv + 1 + ntile) {
-                        const int t = e - (2 * n_kv + 1);
-                        tma_load_4d(dst, &tm_q, bar, 0, it.h, it.q_row0 + t * kTile, it.b);
-                        tma_load_4d(dst + kHalfBytes, &tm_q, bar, 64, it.h, it.q_row0 + t * kTile, it.b);
+                    const Entry en = item_entry(it, n_kv, e);
+                    const int tb = it.b[en.tile], th = it.h[en.tile];
+                    if (en.kind == kEntK || en.kind == kEntV) {
+                        const CUtensorMap* tm = en.kind == kEntV ? &tm_v : &tm_k;
+                        tma_load_4d(dst, tm, bar, 0, th, en.j * kTile, tb);
+                        tma_load_4d(dst + kHalfBytes, tm, bar, 64, th, en.j * kTile, tb);
+                    } else if (en.kind == kEntW) {
+                        tma_load_2d(dst, &tm_w, bar, 0, th * kTile);
+                        tma_load_2d(dst + kHalfBytes, &tm_w, bar, 64, th * kTile);
+                    } else if (en.kind == kEntQRaw) {
+                        tma_load_4d(dst, &tm_q, bar, 0, th, it.row0[en.tile], tb);
+                        tma_load_4d(dst + kHalfBytes, &tm_q, bar, 64, th, it.row0[en.tile], tb);
                     } else {
-                        tma_load_2d(dst, &tm_s, bar, 0, (it.b * p.s.H + it.h) * kTile);
-                        tma_load_2d(dst + kHalfBytes, &tm_s, bar, 64, (it.b * p.s.H + it.h) * kTile);
+                        tma_load_2d(dst, &tm_s, bar, 0, (tb * p.s.H + th) * kTile);
+                        tma_load_2d(dst + kHalfBytes, &tm_s, bar, 64, (tb * p.s.H + th) * kTile);
                     }
                 }
                 if (!ok) break;
@@ -641,77 +694,84 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const int id = item_slots[item & 1];
                 if (id < 0) break;
                 const Item it = decode_item(id, p);
-                const int ntile = it.two ? 2 : 1;
+                const int ntile = it.ntile;
                 const bool active = t < ntile;
+                const bool shared = it.shared;
+                // An entry both tiles read (K, V, W, S of a pair item) is released once by each
+                // issuer; an entry only one tile reads is released twice by that tile's issuer
+                // (the empty barriers always count two arrivals) and ignored by the other.
+                auto release_mine = [&](uint32_t e, bool exclusive) {
+                    release(e);
+                    if (exclusive) release(e);
+                };
+                auto q_free = [&]() {
+                    mma_commit(bars + 8 * kBarQFree);
+                    if (ntile == 1) mma_commit(bars + 8 * kBarQFree);   // on behalf of the idle issuer
+                };
                 if (active) {
                     ok = wait_bar(bars + 8 * (kBarQRot0 + t), qrot_cnt & 1, ab, 61);
                     ++qrot_cnt;
                     if (!ok) break;
-                }
-                // S_t(0) = Q~_t K_0^T
-                ok = wait_full(cons, 62);
-                if (!ok) break;
-                if (active) {
+                    // S_t(0) = Q~_t K_0^T
+                    const uint32_t e_k = cons + (shared ? 0 : t);
+                    ok = wait_full(e_k, 62);
+                    if (!ok) break;
                     tc_fence_after();
-                    issue_qk(q_tile, slot_addr(cons));
+                    issue_qk(q_tile, slot_addr(e_k));
                     mma_commit(bar_s);
+                    release_mine(e_k, !shared);
+                    if (n_kv == 1) q_free();
                 }
-                release(cons);
-                ++cons;
-                if (n_kv == 1) mma_commit(bars + 8 * kBarQFree);
+                cons += shared ? 1 : ntile;
 
                 for (int j = 0; j < n_kv && ok; ++j) {
-                    const uint32_t v_entry = cons;              // V_j
-                    const bool next_is_kv = j + 1 < n_kv;       // else the inter-branch "S" = Q W
-                    const uint32_t b_entry = cons + 1;          // K_{j+1} or W
+                    const bool last = j + 1 == n_kv;     // then the next "S" is the inter branch's Q W
+                    const int per_tile = last ? 3 : 2;   // ragged item: V, K or W, [Qraw] per tile
+                    const int group = shared ? (last ? 2 + ntile : 2) : per_tile * ntile;
 #ifdef ARL2_TRACE
                     const bool tr = blockIdx.x == 0 && item == 0 && (j == 8 || j == 9);
                     const int ts = 40 + t * 8 + (j - 8) * 4;
 #endif
-                    ok = wait_full(v_entry, 63);
-                    if (ok) ok = wait_full(b_entry, 66);
-                    if (ok && !next_is_kv)
-                        for (int u = 0; u < ntile && ok; ++u) ok = wait_full(b_entry + 1 + u, 68);   // raw Q tiles
-                    if (!ok) break;
                     if (active) {
+                        const uint32_t e_v = shared ? cons : cons + per_tile * t;   // V_j
+                        const uint32_t e_b = e_v + 1;                               // K_{j+1} or W
+                        const uint32_t e_q = shared ? cons + 2 + t : e_v + 2;       // raw Q tile (last only)
+                        ok = wait_full(e_v, 63);
+                        if (ok) ok = wait_full(e_b, 66);
+                        if (ok && last) ok = wait_full(e_q, 68);
+                        if (!ok) break;
                         ARL2_STAMP(tr, ts + 0);
                         ok = wait_bar(bar_p, p_cnt & 1, ab, 64 + t);
                         ++p_cnt;
                         if (!ok) break;
                         tc_fence_after();
                         ARL2_STAMP(tr, ts + 1);
-                        issue_pv(slot_addr(v_entry), j > 0);
-                        issue_qk(next_is_kv ? q_tile : slot_addr(b_entry + 1 + t), slot_addr(b_entry));
+                        issue_pv(slot_addr(e_v), j > 0);
+                        issue_qk(last ? slot_addr(e_q) : q_tile, slot_addr(e_b));
                         mma_commit(bar_s);
                         ARL2_STAMP(tr, ts + 2);
+                        release_mine(e_v, !shared);
+                        release_mine(e_b, !shared);
+                        if (last) release_mine(e_q, true);
+                        if (j + 2 == n_kv) q_free();   // S_t(n_kv - 1) was the last use of Q~
                     }
-                    release(v_entry);
-                    release(b_entry);
-                    if (next_is_kv) {
-                        cons += 2;
-                        if (j + 1 == n_kv - 1) mma_commit(bars + 8 * kBarQFree);   // last use of Q~
-                    } else {
-                        for (int u = 0; u < ntile; ++u) release(b_entry + 1 + u);
-                        cons += 2 + ntile;
-                    }
+                    cons += group;
                 }
                 if (!ok) break;
                 // inter branch: O_t += Q''_t S
-                ok = wait_full(cons, 69);
-                if (!ok) break;
                 if (active) {
-                    ok = wait_bar(bar_p, p_cnt & 1, ab, 70 + t);
+                    const uint32_t e_s = cons + (shared ? 0 : t);
+                    ok = wait_full(e_s, 69);
+                    if (ok) ok = wait_bar(bar_p, p_cnt & 1, ab, 70 + t);
                     ++p_cnt;
                     if (!ok) break;
                     tc_fence_after();
-                    issue_pv(slot_addr(cons), true);
-                }
-                release(cons);
-                ++cons;
-                if (active) {
+                    issue_pv(slot_addr(e_s), true);
+                    release_mine(e_s, !shared);
                     mma_commit(bars + 8 * (kBarOFinal0 + t));
                     ++of_cnt;
                 }
+                cons += shared ? 1 : ntile;
             }
             (void)of_cnt;
         }
@@ -1076,7 +1136,7 @@ int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* 
     p.n_kv = (a.s.L + kTile - 1) / kTile;
     const int bh = a.s.B * a.s.H;
     p.n_pair_items = bh * (p.n_kv / 2);
-    p.n_items = p.n_pair_items + ((p.n_kv & 1) ? bh : 0);
+    p.n_items = p.n_pair_items + ((p.n_kv & 1) ? (bh + 1) / 2 : 0);   // ragged tiles go two by two
     // two item counters alternate between launches: a launch consumes one and clears the other
     p.sched_counter = a.status + kStatusSched + (a.launch_parity & 1);
     p.sched_next = a.status + kStatusSched + ((a.launch_parity + 1) & 1);
