@@ -27,7 +27,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, k_rot, partials, state_bf16, wq_op, wk_op, wv_op, total;
+    size_t status, k_rot, partials, state_bf16, wq_op, wk_op, wv_op, rope_h, total;
     int nsplit;
 };
 
@@ -83,6 +83,7 @@ Layout make_layout(const arl2_config& c)
     l.wq_op = off;      off += align_up((size_t)c.H * dd * 2);
     l.wk_op = off;      off += align_up((size_t)c.H * dd * 2);
     l.wv_op = off;      off += align_up((size_t)c.H * dd * 2);
+    l.rope_h = off;     off += align_up((size_t)((c.L + 127) / 128) * 128 * (c.D / 2) * 4);
     l.total = off;
     return l;
 }
@@ -221,6 +222,11 @@ int arl2_set_params(arl2_ctx* ctx, const void* d_wphi_q, const void* d_wphi_k, c
                                                 ctx->cfg.H, as_stream(stream)));
             if (r != ARL2_OK) return r;
         }
+        if (d_rope_cos != nullptr) {
+            int r = account(ctx, tc_prepare_rope(d_rope_cos, d_rope_sin, ctx->ws + ctx->lay.rope_h, ctx->cfg.L,
+                                                 as_stream(stream)));
+            if (r != ARL2_OK) return r;
+        }
     }
     return ARL2_OK;
 }
@@ -259,6 +265,7 @@ int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const voi
     a.out = d_out;
     a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status);
     a.launch_parity = (int)(ctx->step_calls++ & 1u);
+    a.rope_h = (ctx->use_tc && ctx->rope_cos != nullptr) ? ctx->ws + ctx->lay.rope_h : nullptr;
     cudaEvent_t e0 = ctx->ev_before, e1 = ctx->ev_after;
     ctx->ev_before = ctx->ev_after = nullptr;
     if (e0 != nullptr) cudaEventRecord(e0, st);

@@ -40,6 +40,7 @@ struct StepArgs {
     void* out;
     uint32_t* status;
     int launch_parity;      // step launches so far on this context, mod 2 (scheduler counters)
+    const void* rope_h;     // [L, D/2] half2 (cos, sin) copy of the tables (tensor-core path), or nullptr
 };
 
 struct CommitArgs {
@@ -72,6 +73,8 @@ int state_to_bf16(const float* state, __nv_bfloat16* dst, size_t n, cudaStream_t
 bool tc_supported(const arl2_config& c);
 // w: [H, 128, 128] (in, out) bf16 or nullptr (identity) -> w_op: [H, out, in] bf16
 int tc_prepare_map(const void* w, __nv_bfloat16* w_op, int H, cudaStream_t st);
+// cos, sin [L, 64] fp32 -> out [L, 64] half2 (cos, sin): one 256-byte row per token
+int tc_prepare_rope(const float* cos_t, const float* sin_t, void* out, int L, cudaStream_t st);
 int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* state_bf16,
             cudaStream_t st);
 int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat16* wv_op,

@@ -20,6 +20,7 @@
 // Every wait is bounded: when a limit expires the thread records ARL2_ERR_TIMEOUT in the
 // device status block, raises the CTA's abort flag and every role falls through to the exit.
 #include <cuda.h>
+#include <cuda_fp16.h>
 
 #include "arl2_internal.h"
 #include "tc_ptx.cuh"
@@ -74,6 +75,7 @@ struct TcStepParams {
     const float* gate;
     const float* rope_cos;
     const float* rope_sin;
+    const uint4* rope_h;       // half2 (cos, sin) table, warp-interleaved (see pack_rope_kernel), or nullptr
     __nv_bfloat16* out;
     uint32_t* status;
     uint32_t* sched_counter;   // this launch's item counter (zero on entry)
@@ -182,6 +184,15 @@ __device__ __forceinline__ void exp2_poly2(float x0, float x1, float& r0, float&
 // one (stream, head): they share every K/V tile.  A "ragged" item holds the last, partial tiles
 // of two different (stream, head) units (or of one, when the number of units is odd): each tile
 // then streams its own K/V, W_phi_q and state through the ring.
+// (cos, sin) of one rotation pair, stored as half2
+__device__ __forceinline__ void unpack_cs(uint32_t h2, float& c, float& s)
+{
+    const __half2 v = *reinterpret_cast<const __half2*>(&h2);
+    const float2 f = __half22float2(v);
+    c = f.x;
+    s = f.y;
+}
+
 struct Item {
     int b[2], h[2], row0[2];
     int ntile;    // active tiles: 1 or 2
@@ -293,26 +304,30 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
 
         if (active) {
             // ---- Q~ = RoPE(Q): rotate this thread's row of the tile in place          (Eq. 2)
-            if (p.rope_cos != nullptr) {
+            if (p.rope_h != nullptr) {
                 uint8_t* tile = smem + kOffQ + t * kTileBytes;
-                const float* cs = p.rope_cos + (size_t)(valid_row ? row : 0) * (kTile / 2);
-                const float* sn = p.rope_sin + (size_t)(valid_row ? row : 0) * (kTile / 2);
-#pragma unroll 4
+                // all 16 table loads of the row go out before the first one is used
+                const uint4* tab = p.rope_h + ((size_t)(row >> 5) * 16) * 32 + (row & 31);
+                uint4 cs[16];
+#pragma unroll
+                for (int c = 0; c < 16; ++c) cs[c] = __ldg(tab + c * 32);
+#pragma unroll
                 for (int c = 0; c < 16; ++c) {
                     int off = (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
                     uint4 raw = *reinterpret_cast<const uint4*>(tile + off);
-                    float4 cv = *reinterpret_cast<const float4*>(cs + c * 4);
-                    float4 sv = *reinterpret_cast<const float4*>(sn + c * 4);
                     uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-                    float cc[4] = {cv.x, cv.y, cv.z, cv.w}, ss[4] = {sv.x, sv.y, sv.z, sv.w};
+                    const uint32_t h2[4] = {cs[c].x, cs[c].y, cs[c].z, cs[c].w};
 #pragma unroll
                     for (int m = 0; m < 4; ++m) {
+                        float cc, ss;
+                        unpack_cs(h2[m], cc, ss);
                         float x0 = __uint_as_float(w[m] << 16);
                         float x1 = __uint_as_float(w[m] & 0xFFFF0000u);
-                        w[m] = pack_bf16(x0 * cc[m] - x1 * ss[m], x0 * ss[m] + x1 * cc[m]);
+                        w[m] = pack_bf16(x0 * cc - x1 * ss, x0 * ss + x1 * cc);
                     }
                     *reinterpret_cast<uint4*>(tile + off) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
+                ARL2_ITER(true, 256 + item * 16 + t * 8 + 7);
                 fence_proxy_async_smem();
             }
             mbar_arrive(bars + 8 * (kBarQRot0 + t));
@@ -430,6 +445,14 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
             const float l_sum = l_lo + l_hi;
 
             // ---- inter branch: U = Q W_phi_q arrives in the S columns                  (Eq. 3)
+            // the row's rotation table is fetched while the MMA is still running
+            uint4 cs[16];
+            const bool rotate_u = p.rope_h != nullptr && valid_row;
+            if (rotate_u) {
+                const uint4* tab = p.rope_h + ((size_t)(row >> 5) * 16) * 32 + (row & 31);
+#pragma unroll
+                for (int c = 0; c < 16; ++c) cs[c] = __ldg(tab + c * 32);
+            }
             ARL2_ITER(true, 256 + item * 16 + t * 8 + 0);
             if (!wait_bar(bar_s, s_cnt & 1, ab, 30 + t)) return;
             ++s_cnt;
@@ -440,20 +463,18 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                 tmem_ld32(s_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
             tmem_wait_ld();
             {
-                if (p.rope_cos != nullptr && valid_row) {
-                    const float* cs = p.rope_cos + (size_t)row * (kTile / 2);
-                    const float* sn = p.rope_sin + (size_t)row * (kTile / 2);
+                if (rotate_u) {
 #pragma unroll
                     for (int c = 0; c < 16; ++c) {
-                        float4 cv = *reinterpret_cast<const float4*>(cs + c * 4);
-                        float4 sv = *reinterpret_cast<const float4*>(sn + c * 4);
-                        float cc[4] = {cv.x, cv.y, cv.z, cv.w}, s4[4] = {sv.x, sv.y, sv.z, sv.w};
+                        const uint32_t h2[4] = {cs[c].x, cs[c].y, cs[c].z, cs[c].w};
 #pragma unroll
                         for (int m = 0; m < 4; ++m) {
+                            float cc, s1;
+                            unpack_cs(h2[m], cc, s1);
                             float x0 = __uint_as_float(sreg[c * 8 + 2 * m]);
                             float x1 = __uint_as_float(sreg[c * 8 + 2 * m + 1]);
-                            sreg[c * 8 + 2 * m] = __float_as_uint(x0 * cc[m] - x1 * s4[m]);
-                            sreg[c * 8 + 2 * m + 1] = __float_as_uint(x0 * s4[m] + x1 * cc[m]);
+                            sreg[c * 8 + 2 * m] = __float_as_uint(x0 * cc - x1 * s1);
+                            sreg[c * 8 + 2 * m + 1] = __float_as_uint(x0 * s1 + x1 * cc);
                         }
                     }
                 }
@@ -1022,6 +1043,22 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     }
 }
 
+// The rotation table in the form the step kernel reads: half2 (cos, sin) per pair, 16 vectors of
+// 4 pairs per token, stored so that the 32 tokens a warp owns are interleaved -- vector c of
+// token l sits at uint4 index ((l / 32) * 16 + c) * 32 + l % 32 -- and each of a warp's 16 loads is
+// one contiguous 512-byte segment.  Tokens past L (padding up to a whole tile) read as zero.
+// fp16 keeps 11 bits of the unit-range values.
+__global__ void pack_rope_kernel(const float* __restrict__ cos_t, const float* __restrict__ sin_t,
+                                 __half2* __restrict__ out, int L, size_t total)
+{
+    size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= total) return;
+    const int l = (int)(t / 64), m = (int)(t % 64);
+    const int c = m >> 2, w = m & 3;
+    const size_t dst = ((((size_t)(l >> 5) * 16 + c) * 32 + (l & 31)) << 2) + w;
+    out[dst] = l < L ? __floats2half2_rn(cos_t[t], sin_t[t]) : __floats2half2_rn(0.0f, 0.0f);
+}
+
 // out[h][o][i] = w[h][i][o] (bf16), or the identity when w is null: the K-major B operand of
 // U = Q W_phi (B[n][k] = W[k][n]).
 __global__ void transpose_map_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ out,
@@ -1105,6 +1142,16 @@ int tc_prepare_map(const void* w, __nv_bfloat16* w_op, int H, cudaStream_t st)
     return 1;
 }
 
+int tc_prepare_rope(const float* cos_t, const float* sin_t, void* out, int L, cudaStream_t st)
+{
+    size_t total = (size_t)((L + kTile - 1) / kTile) * kTile * (kTile / 2);   // padded to whole tiles
+    pack_rope_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(cos_t, sin_t, static_cast<__half2*>(out), L,
+                                                                         total);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_error("launch of pack_rope_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
+    return 1;
+}
+
 int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* state_bf16, cudaStream_t st)
 {
     static bool attr_set = false;
@@ -1131,6 +1178,7 @@ int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* 
     p.gate = a.gate;
     p.rope_cos = a.rope_cos;
     p.rope_sin = a.rope_sin;
+    p.rope_h = static_cast<const uint4*>(a.rope_h);
     p.out = static_cast<__nv_bfloat16*>(a.out);
     p.status = a.status;
     p.n_kv = (a.s.L + kTile - 1) / kTile;
