@@ -305,6 +305,7 @@ int arl2_commit(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
     a.state_bf16 = ctx->use_tc ? reinterpret_cast<__nv_bfloat16*>(ctx->ws + ctx->lay.state_bf16)
                                : nullptr;
     a.nsplit = ctx->lay.nsplit;
+    a.rope_h = (ctx->use_tc && ctx->rope_cos != nullptr) ? ctx->ws + ctx->lay.rope_h : nullptr;
     a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status);
     if ((reinterpret_cast<uintptr_t>(d_k_clean) | reinterpret_cast<uintptr_t>(d_v_clean)) % 16 != 0) {
         set_error("commit: k_clean and v_clean must be 16-byte aligned");

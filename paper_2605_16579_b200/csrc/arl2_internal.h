@@ -56,6 +56,7 @@ struct CommitArgs {
     float* partials;        // [B, H, nsplit, D, D] fp32
     __nv_bfloat16* state_bf16;  // operand copy refreshed by the reduce kernel, or nullptr
     int nsplit;
+    const void* rope_h;     // half2 (cos, sin) copy of the tables (tensor-core path), or nullptr
     uint32_t* status;
 };
 

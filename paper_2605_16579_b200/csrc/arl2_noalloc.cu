@@ -100,6 +100,7 @@ extern "C" int arl2_commit_static_scratch(const arl2_config* cfg, void* d_state,
     a.partials = scratch;        // every slot the reduce reads is written by the partial kernel
     a.state_bf16 = nullptr;
     a.nsplit = nsplit;
+    a.rope_h = nullptr;
     a.status = nullptr;          // the plain-FMA kernels have no waits and report nothing
     int n = simt_commit(a, cfg->io_dtype, static_cast<cudaStream_t>(stream));
     return n < 0 ? n : ARL2_OK;

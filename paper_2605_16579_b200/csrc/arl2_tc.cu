@@ -828,8 +828,7 @@ enum CBar : int { kCBarW = 0, kCBarFull0, kCBarFull1, kCBarU, kCBarS, kCNumBars 
 
 struct TcCommitParams {
     Shape s;
-    const float* rope_cos;
-    const float* rope_sin;
+    const uint4* rope_h;   // warp-interleaved half2 (cos, sin) table, or nullptr
     float* partials;     // [B, H, nsplit, 128, 128] fp32
     uint32_t* status;
     int nsplit;
@@ -935,26 +934,28 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 
         const int r = tid;                       // token row of the tile
         const int row = l0 + i * kTile + r;
-        const bool valid_row = row < L;
         // ---- K' = L2Norm(RoPE(U_k))
 #pragma unroll
         for (int c = 0; c < 4; ++c)
             tmem_ld32(lane_base + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
         tmem_wait_ld();
-        if (p.rope_cos != nullptr && valid_row) {
-            const float* cs = p.rope_cos + (size_t)row * (kTile / 2);
-            const float* sn = p.rope_sin + (size_t)row * (kTile / 2);
+        if (p.rope_h != nullptr) {
+            // rows of the warp-interleaved table: padding rows past L read as zero
+            const uint4* tab = p.rope_h + ((size_t)(row >> 5) * 16) * 32 + (row & 31);
+            uint4 cs[16];
+#pragma unroll
+            for (int c = 0; c < 16; ++c) cs[c] = __ldg(tab + c * 32);
 #pragma unroll
             for (int c = 0; c < 16; ++c) {
-                float4 cv = *reinterpret_cast<const float4*>(cs + c * 4);
-                float4 sv = *reinterpret_cast<const float4*>(sn + c * 4);
-                float cc[4] = {cv.x, cv.y, cv.z, cv.w}, s4[4] = {sv.x, sv.y, sv.z, sv.w};
+                const uint32_t h2[4] = {cs[c].x, cs[c].y, cs[c].z, cs[c].w};
 #pragma unroll
                 for (int m = 0; m < 4; ++m) {
+                    float cc, s1;
+                    unpack_cs(h2[m], cc, s1);
                     float x0 = __uint_as_float(sreg[c * 8 + 2 * m]);
                     float x1 = __uint_as_float(sreg[c * 8 + 2 * m + 1]);
-                    sreg[c * 8 + 2 * m] = __float_as_uint(x0 * cc[m] - x1 * s4[m]);
-                    sreg[c * 8 + 2 * m + 1] = __float_as_uint(x0 * s4[m] + x1 * cc[m]);
+                    sreg[c * 8 + 2 * m] = __float_as_uint(x0 * cc - x1 * s1);
+                    sreg[c * 8 + 2 * m + 1] = __float_as_uint(x0 * s1 + x1 * cc);
                 }
             }
         }
@@ -1211,8 +1212,7 @@ int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat
     if (int r = make_map_rows(&tm_wv, wv_op, (size_t)a.s.H * kTile)) return r;
     TcCommitParams p;
     p.s = a.s;
-    p.rope_cos = a.rope_cos;
-    p.rope_sin = a.rope_sin;
+    p.rope_h = static_cast<const uint4*>(a.rope_h);
     p.partials = a.partials;
     p.status = a.status;
     p.nsplit = a.nsplit;
