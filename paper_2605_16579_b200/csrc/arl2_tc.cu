@@ -447,6 +447,7 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
             // ---- inter branch: U = Q W_phi_q arrives in the S columns                  (Eq. 3)
             // the row's rotation table is fetched while the MMA is still running
             uint4 cs[16];
+            const float gate_logit = valid_row ? __ldg(p.gate + ((size_t)b * L + row) * H + h) : 0.0f;   // fetched early too
             const bool rotate_u = p.rope_h != nullptr && valid_row;
             if (rotate_u) {
                 const uint4* tab = p.rope_h + ((size_t)(row >> 5) * 16) * 32 + (row & 31);
@@ -486,7 +487,7 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                         ss4[k] = fmaf(__uint_as_float(sreg[c + k]), __uint_as_float(sreg[c + k]), ss4[k]);
                 }
                 const float ss = (ss4[0] + ss4[1]) + (ss4[2] + ss4[3]);
-                const float gate = valid_row ? sigmoid_fast(p.gate[((size_t)b * L + row) * H + h]) : 0.0f;
+                const float gate = valid_row ? sigmoid_fast(gate_logit) : 0.0f;
                 // scaled by the row sum so that the common 1/l of the epilogue leaves gate * Q' S
                 const float f = rsqrtf(ss + p.s.eps) * gate * l_sum;
 #pragma unroll
@@ -513,14 +514,18 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                 tmem_ld32(o_addr + c * 32, o);
                 tmem_wait_ld();
                 if (valid_row) {
+                    // 32-byte stores: each one fills a whole sector of the row
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        uint4 v;
-                        v.x = pack_bf16(__uint_as_float(o[e * 8 + 0]) * inv_l, __uint_as_float(o[e * 8 + 1]) * inv_l);
-                        v.y = pack_bf16(__uint_as_float(o[e * 8 + 2]) * inv_l, __uint_as_float(o[e * 8 + 3]) * inv_l);
-                        v.z = pack_bf16(__uint_as_float(o[e * 8 + 4]) * inv_l, __uint_as_float(o[e * 8 + 5]) * inv_l);
-                        v.w = pack_bf16(__uint_as_float(o[e * 8 + 6]) * inv_l, __uint_as_float(o[e * 8 + 7]) * inv_l);
-                        *reinterpret_cast<uint4*>(orow + c * 32 + e * 8) = v;
+                    for (int e = 0; e < 2; ++e) {
+                        uint32_t w[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            w[i] = pack_bf16(__uint_as_float(o[e * 16 + 2 * i]) * inv_l,
+                                             __uint_as_float(o[e * 16 + 2 * i + 1]) * inv_l);
+                        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(
+                                         orow + c * 32 + e * 16),
+                                     "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                                     : "memory");
                     }
                 }
             }
