@@ -31,6 +31,7 @@ if ROOT not in sys.path:
 METRIC = "hybrid-attn layer tokens/s per denoise step"
 UNIT = "tokens/s"
 RING = 3  # pre-generated step-input sets the timed loop rotates through
+HORIZON_BLOCKS = 120  # blocks of the timed loop whose individual latency is recorded (config 5's horizon)
 
 
 def peaks():
@@ -215,6 +216,28 @@ def max_over_ranks(values, world, device):
     return [float(x) for x in t.tolist()]
 
 
+def horizon_report(block_ms, mem_marks, layer_bytes):
+    """Per-block latency and device memory against the number of past blocks: the layer keeps a
+    fixed-size state per (stream, head), so both must stay flat however long the video gets."""
+    n = len(block_ms)
+    if n < 4:
+        return None
+    q = max(n // 10, 1)
+    return {
+        "blocks": n,
+        "ms_first": statistics.mean(block_ms[:q]), "ms_last": statistics.mean(block_ms[-q:]),
+        "ms_min": min(block_ms), "ms_max": max(block_ms),
+        "last_over_first": statistics.mean(block_ms[-q:]) / statistics.mean(block_ms[:q]),
+        # the first blocks run before the power cap pulls the SM clock down; the middle and last
+        # thirds run at the settled clock and isolate the dependence on the horizon itself
+        "ms_mid_third": statistics.mean(block_ms[n // 3:2 * n // 3]),
+        "ms_last_third": statistics.mean(block_ms[2 * n // 3:]),
+        "last_third_over_mid_third": statistics.mean(block_ms[2 * n // 3:]) / statistics.mean(block_ms[n // 3:2 * n // 3]),
+        "device_bytes_first": mem_marks[0], "device_bytes_last": mem_marks[-1],
+        "state_plus_workspace_bytes": layer_bytes,
+    }
+
+
 def rank_seeds(rank):
     """Each replica draws its own inputs: step-input seeds and the commit block index."""
     return [s + 10 * rank for s in range(RING)], rank
@@ -284,14 +307,22 @@ def run_ours(args):
     launches0 = layer.launch_count
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
+    block_marks = [t0]      # one event per block boundary: per-block latency against the horizon
+    mem_marks = []
     for i in range(args.steps):
         block(i, True)
+        if i < HORIZON_BLOCKS:
+            ev = torch.cuda.Event(enable_timing=True)
+            ev.record()
+            block_marks.append(ev)
+            mem_marks.append(torch.cuda.memory_allocated(dev))
     t1.record()
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     launches = layer.launch_count - launches0
     ms_total = t0.elapsed_time(t1)
     kern_ms = [a.elapsed_time(b) for a, b in step_events]
+    block_ms = [block_marks[i].elapsed_time(block_marks[i + 1]) for i in range(len(block_marks) - 1)]
     layer.sync_status()
 
     # end to end through the same entry points with HOST buffers: every pass copies its inputs
@@ -374,12 +405,14 @@ def run_ours(args):
                     "blocks_timed": e2e_blocks},
             "gpu_launches": int(launches),
             "clocks": clocks,
+            "horizon": horizon_report(block_ms, mem_marks, layer.workspace_bytes + layer.state.numel() * 4),
         }
         if world == 1 and not args.no_cpu_baseline:
             s = CpuSample(cfg)
-            t = s.time_rows(s.threads)
-            t = min(t, s.time_rows(s.threads))  # the first call pays for page faults
-            n_rows = max(s.threads, int(s.threads * 12.0 / max(t, 1e-6)))
+            s.time_rows(s.threads)                      # the first call pays for page faults
+            cal = 64 * s.threads
+            t = s.time_rows(cal)
+            n_rows = max(cal, int(cal * 15.0 / max(t, 1e-6)))   # about 15 s of CPU work
             tr = s.time_rows(n_rows)
             n_heads = min(s.threads, cfg.B * cfg.H)
             th = s.time_heads(n_heads)
