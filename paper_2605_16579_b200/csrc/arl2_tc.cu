@@ -1,8 +1,8 @@
 // Tensor-core (tcgen05 / TMEM / TMA) kernels of the ARL^2 layer for bf16 I/O, D = 128.
 //
-// Step kernel (Eq. 2, 3, 5-8): persistent, one CTA per SM, work item = (stream b, head h, pair
-// of 128-row query tiles), items handed out by an atomic counter (pairs first, the single
-// ragged tiles last).
+// Step kernel (Eq. 2, 3, 5-8): persistent, one CTA per SM.  A work item drives two 128-row query
+// tiles: two consecutive tiles of one (stream, head), or the ragged last tiles of two different
+// (stream, head) units.  Items are handed out by an atomic counter, the pairs first.
 //   warps 0-3 / 4-7  softmax group of query tile 0 / 1 (one thread per query row)
 //   warp 8           TMA producer and scheduler: the Q tiles, then through a 5-slot ring K_j, V_j
 //                    for every key tile, then W_phi_q^T, the raw Q tiles again and the bf16

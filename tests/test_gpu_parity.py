@@ -188,3 +188,13 @@ def test_full_size_configs_sampled(oracle, name):
         o2, s2 = run_schedule(pair, 1, 1, full=False, heads_per_stream=2, rows_per_head=16)
         o, s = max(o, o2), max(s, s2)
     print(f"{name}: worst sampled output error {o:.2e}, worst state error {s:.2e}")
+
+
+@pytest.mark.parametrize("B,H,L", [(1, 1, 100), (1, 3, 333), (3, 1, 200), (1, 5, 640)])
+def test_odd_unit_counts_bf16(oracle, B, H, L):
+    """The tensor-core step kernel packs the ragged last tiles of two (stream, head) units into
+    one work item: odd numbers of units leave one of them alone, and L a multiple of the tile
+    leaves none."""
+    cfg = workload.custom(B=B, H=H, D=128, L=L, dtype="bf16", cfg_id=23)
+    pair = Pair(oracle, cfg)
+    run_schedule(pair, 2, 2, full=True)
