@@ -357,6 +357,24 @@ def run_ours(args):
     h2d = cfg.steps * set_bytes + commit_bytes
     d2h = cfg.steps * out.numel() * out.element_size()
 
+    # the two commit rules side by side (outside the timed regions above): the gated-linear commit
+    # the block uses, and the delta rule of Eq. 4 at block level
+    beta = workload.beta_logits(cfg, commit_block).to(dev)
+    commit_ms = {}
+    for name, call in (("gated_linear", lambda: layer.commit(*dev_commit)),
+                       ("delta", lambda: layer.commit_delta(*dev_commit, beta))):
+        layer.reset()
+        for _ in range(3):
+            call()
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record()
+        for _ in range(20):
+            call()
+        c1.record()
+        torch.cuda.synchronize()
+        commit_ms[name] = c0.elapsed_time(c1) / 20
+    layer.sync_status()
+
     ms_total, ms_e2e, kern_mean = max_over_ranks([ms_total, ms_e2e, statistics.mean(kern_ms)], world, dev)
 
     if rank == 0:
@@ -406,6 +424,7 @@ def run_ours(args):
             "gpu_launches": int(launches),
             "clocks": clocks,
             "horizon": horizon_report(block_ms, mem_marks, layer.workspace_bytes + layer.state.numel() * 4),
+            "commit_ms": commit_ms,
         }
         if world == 1 and not args.no_cpu_baseline:
             s = CpuSample(cfg)

@@ -124,6 +124,19 @@ int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const voi
 int arl2_commit(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
                 const float* d_decay_logits, void* stream);
 
+/*
+ * State commit with the delta rule of Eq. 4 as printed, applied once per block to the clean
+ * pass's tokens (all of them against the state as it stood before the call):
+ *   S[b,h] <- sigmoid(a[b,h]) S[b,h] + sum_l beta_l K'_l^T (V'_l - K'_l S_old[b,h]),
+ *   beta_l = sigmoid(d_beta_logits[b,l,h]),  K', V' as in arl2_commit.
+ * The result does not depend on the order of the tokens.  d_beta_logits: [B, L, H] fp32, or
+ * NULL for beta = 1.  Other arguments, reproducibility and error behaviour as arl2_commit.  With
+ * bf16 I/O and D = 128 the prediction K' S_old is a tensor-core contraction against the bf16
+ * operand copy of S_old.  Any context may mix calls of arl2_commit and arl2_commit_delta.
+ */
+int arl2_commit_delta(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
+                      const float* d_decay_logits, const float* d_beta_logits, void* stream);
+
 /* S <- 0 for stream `stream_index` (0..B-1) or all streams (-1): Algorithm 1, first line. */
 int arl2_reset(arl2_ctx* ctx, int32_t stream_index, void* stream);
 

@@ -21,7 +21,7 @@ ARL2_FLAG_FORCE_SIMT = 1
 EXPORTS = (
     "arl2_workspace_bytes", "arl2_create", "arl2_set_params", "arl2_denoise_step", "arl2_commit",
     "arl2_reset", "arl2_get_state", "arl2_set_state", "arl2_sync_status", "arl2_launch_count",
-    "arl2_set_profile_events", "arl2_commit_static_scratch",
+    "arl2_set_profile_events", "arl2_commit_static_scratch", "arl2_commit_delta",
     "arl2_step_kernel_name", "arl2_destroy", "arl2_last_error", "arl2_version",
 )
 
@@ -69,6 +69,8 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     lib.arl2_denoise_step.argtypes = [vp] * 7
     lib.arl2_commit.restype = ctypes.c_int
     lib.arl2_commit.argtypes = [vp] * 5
+    lib.arl2_commit_delta.restype = ctypes.c_int
+    lib.arl2_commit_delta.argtypes = [vp] * 6
     lib.arl2_reset.restype = ctypes.c_int
     lib.arl2_reset.argtypes = [vp, ctypes.c_int32, vp]
     lib.arl2_get_state.restype = ctypes.c_int
@@ -183,6 +185,18 @@ class Layer:
         with torch.cuda.device(self.device):
             _check(load().arl2_commit(self._ctx, _ptr(k_clean), _ptr(v_clean), _ptr(decay_logits),
                                       _stream()), "arl2_commit")
+
+    def commit_delta(self, k_clean, v_clean, decay_logits, beta_logits=None):
+        """Eq. 4 as printed, at block level: S <- sigmoid(a) S + K'^T diag(beta) (V' - K' S_old)."""
+        shape = (self.B, self.L, self.H, self.D)
+        self._want(k_clean, shape, self.dtype, "k_clean")
+        self._want(v_clean, shape, self.dtype, "v_clean")
+        self._want(decay_logits, (self.B, self.H), torch.float32, "decay_logits")
+        if beta_logits is not None:
+            self._want(beta_logits, (self.B, self.L, self.H), torch.float32, "beta_logits")
+        with torch.cuda.device(self.device):
+            _check(load().arl2_commit_delta(self._ctx, _ptr(k_clean), _ptr(v_clean), _ptr(decay_logits),
+                                            _ptr(beta_logits), _stream()), "arl2_commit_delta")
 
     def reset(self, stream_index: int = -1):
         with torch.cuda.device(self.device):

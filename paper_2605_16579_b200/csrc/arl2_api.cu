@@ -287,8 +287,11 @@ int arl2_set_profile_events(arl2_ctx* ctx, void* ev_before, void* ev_after)
     return ARL2_OK;
 }
 
-int arl2_commit(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
-                const float* d_decay_logits, void* stream)
+namespace {
+
+// Shared by arl2_commit (delta = false) and arl2_commit_delta.
+int commit_impl(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
+                const float* d_decay_logits, bool delta, const float* d_beta_logits, void* stream)
 {
     if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
     if (!d_k_clean || !d_v_clean || !d_decay_logits) {
@@ -307,6 +310,8 @@ int arl2_commit(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
     a.nsplit = ctx->lay.nsplit;
     a.rope_h = (ctx->use_tc && ctx->rope_cos != nullptr) ? ctx->ws + ctx->lay.rope_h : nullptr;
     a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status);
+    a.delta = delta;
+    a.beta = d_beta_logits;
     if ((reinterpret_cast<uintptr_t>(d_k_clean) | reinterpret_cast<uintptr_t>(d_v_clean)) % 16 != 0) {
         set_error("commit: k_clean and v_clean must be 16-byte aligned");
         return ARL2_ERR_INVALID_ARG;
@@ -316,6 +321,20 @@ int arl2_commit(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
                                       reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wv_op),
                                       as_stream(stream)));
     return account(ctx, simt_commit(a, ctx->cfg.io_dtype, as_stream(stream)));
+}
+
+}  // namespace
+
+int arl2_commit(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
+                const float* d_decay_logits, void* stream)
+{
+    return commit_impl(ctx, d_k_clean, d_v_clean, d_decay_logits, false, nullptr, stream);
+}
+
+int arl2_commit_delta(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
+                      const float* d_decay_logits, const float* d_beta_logits, void* stream)
+{
+    return commit_impl(ctx, d_k_clean, d_v_clean, d_decay_logits, true, d_beta_logits, stream);
 }
 
 int arl2_reset(arl2_ctx* ctx, int32_t stream_index, void* stream)

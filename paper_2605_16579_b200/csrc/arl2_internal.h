@@ -58,6 +58,8 @@ struct CommitArgs {
     int nsplit;
     const void* rope_h;     // half2 (cos, sin) copy of the tables (tensor-core path), or nullptr
     uint32_t* status;
+    bool delta = false;     // Eq. 4 as printed: value operand diag(beta) (V' - K' S_old)
+    const float* beta = nullptr;   // [B, L, H] learning-rate logits, or nullptr = 1 (delta only)
 };
 
 // ---- plain-FMA kernels (arl2_simt.cu) -------------------------------------------------

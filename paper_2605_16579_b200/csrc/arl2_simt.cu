@@ -360,6 +360,40 @@ __global__ void __launch_bounds__(NT) simt_commit_partial_kernel(CommitArgs a)
         __syncthreads();
         feature_tile<D, T>(Ks, Ws, wk, r0, lim, a.rope_cos, a.rope_sin, a.s.eps, true, tx, ty, tid);
         feature_tile<D, T>(Vs2, Ws, wv, r0, lim, nullptr, nullptr, a.s.eps, false, tx, ty, tid);
+        if (a.delta) {
+            // Eq. 4 as printed: the value rows become beta (V' - K' S_old); S_old is the state as
+            // it stands (the reduce kernel, a later launch, is the only writer)
+            float x[4][D / 16];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int e = 0; e < D / 16; ++e) x[i][e] = 0.0f;
+            const float* Sh = a.state + ((size_t)b * H + h) * D * D;
+            for (int c = 0; c < D / BN; ++c) {
+                __syncthreads();
+                load_mat_rows<float>(Ws, Sh, c * BN, D, tid);
+                __syncthreads();
+                tile_gemm<D>(x, Ks + c * BN, LD, Ws, tx, ty);
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int row = r0 + ty * 4 + i;
+                float beta = 1.0f;
+                if (a.beta != nullptr)
+                    beta = row < lim ? sigmoidf_(a.beta[((size_t)b * L + row) * H + h]) : 0.0f;
+#pragma unroll
+                for (int c = 0; c < D / 64; ++c) {
+                    float4* pv = reinterpret_cast<float4*>(Vs2 + (ty * 4 + i) * LD + c * 64 + tx * 4);
+                    float4 v = *pv;   // this thread is the only one to touch these four values
+                    v.x = beta * (v.x - x[i][c * 4 + 0]);
+                    v.y = beta * (v.y - x[i][c * 4 + 1]);
+                    v.z = beta * (v.z - x[i][c * 4 + 2]);
+                    v.w = beta * (v.w - x[i][c * 4 + 3]);
+                    *pv = v;
+                }
+            }
+            __syncthreads();
+        }
 #pragma unroll 2
         for (int r = 0; r < BM; ++r) {
             float ka[D / 16], vb[D / 16];

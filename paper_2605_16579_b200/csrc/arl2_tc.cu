@@ -825,24 +825,30 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 constexpr int kCOffWk = 0;
 constexpr int kCOffWv = kTileBytes;
 constexpr int kCOffPair = 2 * kTileBytes;                  // 2 pairs of (K tile, V tile)
-constexpr int kCOffBars = kCOffPair + 4 * kTileBytes;
+constexpr int kCOffState = kCOffPair + 4 * kTileBytes;     // bf16 copy of S_old (delta rule only)
+constexpr int kCOffBars = kCOffState + kTileBytes;
 constexpr int kCommitSmemBytes = kCOffBars + 128 + 1024;
 constexpr int kCommitThreads = 128;
 
-enum CBar : int { kCBarW = 0, kCBarFull0, kCBarFull1, kCBarU, kCBarS, kCNumBars };
+enum CBar : int { kCBarW = 0, kCBarFull0, kCBarFull1, kCBarU, kCBarS, kCBarP, kCNumBars };
 
 struct TcCommitParams {
     Shape s;
     const uint4* rope_h;   // warp-interleaved half2 (cos, sin) table, or nullptr
+    const float* beta;     // [B, L, H] learning-rate logits (delta rule), or nullptr = 1
     float* partials;     // [B, H, nsplit, 128, 128] fp32
     uint32_t* status;
     int nsplit;
 };
 
+// kDelta (Eq. 4 as printed, at block level): the value operand of the last MMA is
+// R = diag(beta) (V' - K' S_old) instead of V'; K' S_old is one more MMA per tile (A = K' as
+// written for the last MMA, read d-major; B = the bf16 copy of the state) into TMEM columns 384-511.
+template <bool kDelta>
 __global__ void __launch_bounds__(kCommitThreads, 1)
 tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                  const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv,
-                 const TcCommitParams p)
+                 const __grid_constant__ CUtensorMap tm_s, const TcCommitParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
@@ -892,7 +898,11 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         prefetch_tensormap(&tm_k);
         prefetch_tensormap(&tm_v);
         const uint32_t bar_w = bars + 8 * kCBarW;
-        mbar_expect_tx(bar_w, 2 * kTileBytes);
+        mbar_expect_tx(bar_w, (kDelta ? 3 : 2) * kTileBytes);
+        if (kDelta) {
+            tma_load_2d(smem_base + kCOffState, &tm_s, bar_w, 0, (b * H + h) * kTile);
+            tma_load_2d(smem_base + kCOffState + kHalfBytes, &tm_s, bar_w, 64, (b * H + h) * kTile);
+        }
         tma_load_2d(smem_base + kCOffWk, &tm_wk, bar_w, 0, h * kTile);
         tma_load_2d(smem_base + kCOffWk + kHalfBytes, &tm_wk, bar_w, 64, h * kTile);
         tma_load_2d(smem_base + kCOffWv, &tm_wv, bar_w, 0, h * kTile);
@@ -911,6 +921,7 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     };
     constexpr uint32_t idesc_u = idesc_bf16(kTile, kTile, 0, 0);    // tile x map: both K-major
     constexpr uint32_t idesc_ds = idesc_bf16(kTile, kTile, 1, 1);   // K'^T V': both token-major
+    constexpr uint32_t idesc_ps = idesc_bf16(kTile, kTile, 0, 1);   // K' S_old: A d-major, B = S rows
 
     uint32_t sreg[128];
     for (int i = 0; i < ntiles; ++i) {
@@ -984,11 +995,44 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 *reinterpret_cast<uint4*>(pair + off) = v;
             }
         }
-        // ---- V' = U_v
+        if (kDelta) {
+            // ---- prediction K' S_old                                                   (Eq. 4)
+            fence_proxy_async_smem();
+            tc_fence_before();
+            __syncthreads();
+            if (tid == 0 && ok) {
+                tc_fence_after();
+                const uint32_t a_lo = (pair_addr >> 4) | kLboK;
+                const uint32_t b_lo = ((smem_base + kCOffState) >> 4) | kLboMN;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t koff = (uint32_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
+                    mma_ss(tmem_base + 3 * kTile, desc64(a_lo + koff), desc64(b_lo + (uint32_t)(ks * (2048 >> 4))),
+                           idesc_ps, ks > 0);
+                }
+                mma_commit(bars + 8 * kCBarP);
+            }
+            if (!wait_bar(bars + 8 * kCBarP, (uint32_t)(i & 1), ab, 85)) break;
+            tc_fence_after();
+        }
+        // ---- V' = U_v, or R = beta (V' - K' S_old)
 #pragma unroll
         for (int c = 0; c < 4; ++c)
             tmem_ld32(lane_base + kTile + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
         tmem_wait_ld();
+        if (kDelta) {
+            float beta = 1.0f;
+            if (p.beta != nullptr) beta = row < L ? sigmoid_fast(__ldg(p.beta + ((size_t)b * L + row) * H + h)) : 0.0f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t pr[32];
+                tmem_ld32(lane_base + 3 * kTile + c * 32, pr);
+                tmem_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                    sreg[c * 32 + e] = __float_as_uint(beta * (__uint_as_float(sreg[c * 32 + e]) - __uint_as_float(pr[e])));
+            }
+        }
 #pragma unroll
         for (int c = 0; c < 16; ++c) {
             uint4 v;
@@ -1205,24 +1249,40 @@ int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat
 {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc_commit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(tc_commit_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kCommitSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(tc_commit_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kCommitSmemBytes);
         if (e != cudaSuccess) { set_error("cudaFuncSetAttribute(tc_commit_kernel, %d): %s", kCommitSmemBytes, cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
         attr_set = true;
     }
-    CUtensorMap tm_k, tm_v, tm_wk, tm_wv;
+    if (a.delta && a.state_bf16 == nullptr) {
+        set_error("tc_commit: the delta rule needs the bf16 copy of the state");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    CUtensorMap tm_k, tm_v, tm_wk, tm_wv, tm_s;
     if (int r = make_map_blhd(&tm_k, a.k, a.s)) return r;
     if (int r = make_map_blhd(&tm_v, a.v, a.s)) return r;
     if (int r = make_map_rows(&tm_wk, wk_op, (size_t)a.s.H * kTile)) return r;
     if (int r = make_map_rows(&tm_wv, wv_op, (size_t)a.s.H * kTile)) return r;
+    if (a.delta) {
+        if (int r = make_map_rows(&tm_s, a.state_bf16, (size_t)a.s.B * a.s.H * kTile)) return r;
+    } else {
+        tm_s = tm_wk;   // not read
+    }
     TcCommitParams p;
     p.s = a.s;
     p.rope_h = static_cast<const uint4*>(a.rope_h);
+    p.beta = a.beta;
     p.partials = a.partials;
     p.status = a.status;
     p.nsplit = a.nsplit;
     dim3 grid(a.nsplit, a.s.H, a.s.B);
-    tc_commit_kernel<<<grid, kCommitThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, tm_wv, p);
+    if (a.delta)
+        tc_commit_kernel<true><<<grid, kCommitThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, tm_wv, tm_s, p);
+    else
+        tc_commit_kernel<false><<<grid, kCommitThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, tm_wv, tm_s, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_error("launch of tc_commit_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
     int m = commit_reduce(a, st);

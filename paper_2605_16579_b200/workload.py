@@ -106,6 +106,16 @@ def commit_inputs(cfg: Config, block: int):
     return kc, vc, a
 
 
+def beta_logits(cfg: Config, block: int, mean: float = -3.0, std: float = 1.0):
+    """Learning-rate logits [B, L, H] fp32 for the delta-rule commit of one block.
+
+    The default mean keeps sigmoid(beta) near 0.05: with L >> D tokens applied against the same
+    old state, larger rates make the block-level step overshoot.
+    """
+    gen = _gen(cfg, block, COMMIT_STEP, salt=7)
+    return mean + std * torch.randn(cfg.B, cfg.L, cfg.H, generator=gen, dtype=torch.float32)
+
+
 def feature_weights(cfg: Config):
     """W_phi_q, W_phi_k, W_phi_v, each [H, D, D] (in, out) = I + 0.02 N(0, 1), config dtype."""
     gen = _gen(cfg, 0, 0, salt=5)

@@ -99,6 +99,23 @@ class Pair:
             err = err[mask]
         return float(err.max())
 
+    def commit_delta(self, kc, vc, a, beta, heads=None):
+        """Delta-rule commit (Eq. 4 at block level) on both sides; worst per-head error of S."""
+        d = self.dev
+        self.layer.commit_delta(kc.to(d), vc.to(d), a.to(d), None if beta is None else beta.to(d))
+        got = self.layer.get_state().numpy().astype(np.float64)
+        self.S_ref = self.oracle.commit(kc, vc, a, self.S_ref, self.wk, self.wv, self.cos, self.sin,
+                                        eps=self.eps, rule=1, beta_logit=beta, heads=heads)
+        assert np.isfinite(got).all()
+        err = head_errors(got, self.S_ref, head_axis_first=True)
+        if heads is not None:
+            mask = np.zeros(err.shape, dtype=bool)
+            for b, h in heads:
+                mask[b, h] = True
+            self.S_ref[~mask] = got[~mask]
+            err = err[mask]
+        return float(err.max())
+
     def reset(self, stream=-1):
         self.layer.reset(stream)
         self.S_ref = self.oracle.reset(self.S_ref, stream)
