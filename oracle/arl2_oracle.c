@@ -287,6 +287,65 @@ void arl2_oracle_commit(int B, int H, int L, int D,
     }
 }
 
+/*
+ * Eq. 4 applied token by token with per-token gates (the sentence after Eq. 4: the update
+ * runs sequentially over the L tokens of the frame, with gates alpha^(j), beta^(j)):
+ *   for j = 0..L-1:   S <- alpha_j S + beta_j K'_j^T (V'_j - K'_j S)
+ * where the S on the right is the state before token j (both uses), alpha_j =
+ * sigmoid(alpha_logit[b,j,h]), beta_j = sigmoid(beta_logit[b,j,h]).  Eq. 4 is taken as
+ * printed: the prediction K'_j S uses the undecayed previous state.
+ *   alpha_logit, beta_logit  [B, L, H]; NULL = gate fixed at 1.
+ */
+static void commit_head_tokens(int b, int h, int H, int L, int D,
+                               const double *kc, const double *vc,
+                               const double *alpha_logit, const double *beta_logit,
+                               const double *wk, const double *wv,
+                               const double *rope_cos, const double *rope_sin, double eps,
+                               double *S)
+{
+    double *Sh = S + ((size_t)b * H + h) * D * D;
+    double *kf = (double *)malloc(sizeof(double) * D);
+    double *vf = (double *)malloc(sizeof(double) * D);
+    double *err = (double *)malloc(sizeof(double) * D);
+    for (int j = 0; j < L; ++j) {
+        size_t off = (((size_t)b * L + j) * H + h) * D;
+        size_t gi = ((size_t)b * L + j) * H + h;
+        phi(kc + off, wk, h, D, kf);
+        rope(kf, D, rope_cos, rope_sin, j);
+        l2norm(kf, D, eps);
+        phi(vc + off, wv, h, D, vf);
+        double alpha = alpha_logit ? sigmoid(alpha_logit[gi]) : 1.0;
+        double beta = beta_logit ? sigmoid(beta_logit[gi]) : 1.0;
+        for (int e = 0; e < D; ++e) {   /* V'_j - K'_j S, with the state before this token */
+            double acc = 0.0;
+            for (int d = 0; d < D; ++d) acc += kf[d] * Sh[(size_t)d * D + e];
+            err[e] = vf[e] - acc;
+        }
+        for (int d = 0; d < D; ++d)
+            for (int e = 0; e < D; ++e)
+                Sh[(size_t)d * D + e] = alpha * Sh[(size_t)d * D + e] + beta * kf[d] * err[e];
+    }
+    free(err); free(vf); free(kf);
+}
+
+/* heads: optional list of n_heads (b, h) pairs to commit; NULL = all of them. */
+void arl2_oracle_commit_tokens(int B, int H, int L, int D,
+                               const double *kc, const double *vc,
+                               const double *alpha_logit, const double *beta_logit,
+                               const double *wk, const double *wv,
+                               const double *rope_cos, const double *rope_sin, double eps,
+                               int n_heads, const int *bs, const int *hs, double *S)
+{
+    int total = bs ? n_heads : B * H;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int t = 0; t < total; ++t) {
+        int b = bs ? bs[t] : t / H;
+        int h = bs ? hs[t] : t % H;
+        commit_head_tokens(b, h, H, L, D, kc, vc, alpha_logit, beta_logit, wk, wv, rope_cos,
+                           rope_sin, eps, S);
+    }
+}
+
 /* S <- 0 for stream `stream` (or all streams when stream < 0): Algorithm 1, first line. */
 void arl2_oracle_reset(int B, int H, int D, int stream, double *S)
 {

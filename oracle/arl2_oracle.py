@@ -145,6 +145,31 @@ def commit(kc, vc, a, S, wk=None, wv=None, rope_cos=None, rope_sin=None, eps=1e-
     return S
 
 
+def commit_tokens(kc, vc, S, alpha_logit=None, beta_logit=None, wk=None, wv=None, rope_cos=None,
+                  rope_sin=None, eps=1e-6, heads=None):
+    """Eq. 4 token by token with per-token gates [B, L, H] (None = gate 1).  Returns the new S."""
+    kc, vc = _f64(kc), _f64(vc)
+    wk, wv, rope_cos, rope_sin = _f64(wk), _f64(wv), _f64(rope_cos), _f64(rope_sin)
+    alpha_logit, beta_logit = _f64(alpha_logit), _f64(beta_logit)
+    S = _f64(S).copy()
+    B, L, H, D = kc.shape
+    assert S.shape == (B, H, D, D)
+    for g in (alpha_logit, beta_logit):
+        assert g is None or g.shape == (B, L, H)
+    if heads is None:
+        n, bs, hs = 0, None, None
+    else:
+        heads = np.asarray(heads, dtype=np.int32).reshape(-1, 2)
+        n = heads.shape[0]
+        bs = np.ascontiguousarray(heads[:, 0])
+        hs = np.ascontiguousarray(heads[:, 1])
+    _load().arl2_oracle_commit_tokens(
+        B, H, L, D, _p(kc), _p(vc), _p(alpha_logit), _p(beta_logit), _p(wk), _p(wv), _p(rope_cos),
+        _p(rope_sin), ctypes.c_double(eps), n, _p(bs), _p(hs), _p(S),
+    )
+    return S
+
+
 def reset(S, stream: int = -1):
     """S <- 0 for one stream or all (stream < 0).  Returns a new array."""
     S = _f64(S).copy()

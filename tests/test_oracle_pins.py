@@ -340,6 +340,83 @@ def test_delta_rules_overwrite_and_coincide(oracle):
     np.testing.assert_allclose(got, ref.numpy(), rtol=1e-11, atol=1e-13)
 
 
+def sig(x):
+    return 1.0 / (1.0 + np.exp(-x))
+
+
+def test_token_gates_matrix_product_form(oracle):
+    """Per-token Eq. 4 rewritten as S_j = (alpha_j I - beta_j k_j^T k_j) S_{j-1} + beta_j k_j^T v_j
+    and evaluated with explicit D x D transition matrices (library matmul), with feature maps,
+    rotation and normalisation taken from the library-pinned feature routine."""
+    B, L, H, D = 2, 9, 2, 8
+    k, v, S0 = rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, H, D, D)
+    al, bl = rnd(B, L, H) + 1.0, rnd(B, L, H)
+    wk, wv = np.eye(D) + 0.1 * rnd(H, D, D), np.eye(D) + 0.1 * rnd(H, D, D)
+    cos, sin = tables(L, D)
+    got = oracle.commit_tokens(k, v, S0, al, bl, wk, wv, cos, sin, eps=1e-6)
+    kf = oracle.feature(k, wk, cos, sin, 1e-6, 0)
+    vf = oracle.feature(v, wv, None, None, 1e-6, 1)
+    ref = S0.copy()
+    for b in range(B):
+        for h in range(H):
+            S = torch.from_numpy(S0[b, h])
+            for j in range(L):
+                kk = torch.from_numpy(kf[b, j, h])[None, :]          # 1 x D
+                vv = torch.from_numpy(vf[b, j, h])[None, :]
+                M = sig(al[b, j, h]) * torch.eye(D, dtype=torch.float64) - sig(bl[b, j, h]) * (kk.T @ kk)
+                S = M @ S + sig(bl[b, j, h]) * (kk.T @ vv)
+            ref[b, h] = S.numpy()
+    np.testing.assert_allclose(got, ref, rtol=1e-11, atol=1e-13)
+
+
+def test_token_gates_orthonormal_keys_closed_form(oracle):
+    """With orthonormal keys token j only rewrites row-space direction k_j: along it the state
+    holds (prod_{m<j} alpha_m) k_j S_0 before token j, becomes (alpha_j - beta_j) of that plus
+    beta_j v_j, and decays with the later alphas; the orthogonal complement only decays."""
+    B, L, H, D = 1, 5, 2, 8
+    k, v, S0 = orthonormal_keys(B, L, H, D), rnd(B, L, H, D), rnd(B, H, D, D)
+    al, bl = rnd(B, L, H) + 1.0, rnd(B, L, H)
+    got = oracle.commit_tokens(k, v, S0, al, bl, eps=0.0)
+    a, bt = sig(al), sig(bl)
+    for h in range(H):
+        total = np.prod(a[0, :, h])
+        proj = np.zeros((D, D))
+        for j in range(L):
+            kj = k[0, j, h]
+            before = np.prod(a[0, :j, h]) * (kj @ S0[0, h])
+            after_j = (a[0, j, h] - bt[0, j, h]) * before + bt[0, j, h] * v[0, j, h]
+            read = np.prod(a[0, j + 1:, h]) * after_j
+            np.testing.assert_allclose(kj @ got[0, h], read, rtol=1e-10, atol=1e-12)
+            proj += np.outer(kj, kj)
+        rest = (np.eye(D) - proj) @ got[0, h]
+        np.testing.assert_allclose(rest, total * (np.eye(D) - proj) @ S0[0, h], rtol=1e-10, atol=1e-12)
+
+
+def test_token_gates_special_cases(oracle):
+    B, L, H, D = 1, 7, 2, 8
+    k, v, S0 = rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, H, D, D)
+    al, bl = rnd(B, L, H) + 1.0, rnd(B, L, H)
+    # no learning: only the decays act
+    got = oracle.commit_tokens(k, v, S0, al, np.full((B, L, H), -800.0))
+    np.testing.assert_allclose(got, np.prod(sig(al), axis=1)[..., None, None] * S0, rtol=1e-12)
+    # alpha = 1 everywhere: the token-sequential rule with one block-level decay of 1 (rule 2)
+    got = oracle.commit_tokens(k, v, S0, None, bl)
+    ref = oracle.commit(k, v, np.full((B, H), 800.0), S0, rule=2, beta_logit=bl)
+    np.testing.assert_allclose(got, ref, rtol=1e-12, atol=1e-14)
+    # one token: Eq. 4 once, against library ops
+    k1, v1 = k[:, :1], v[:, :1]
+    got = oracle.commit_tokens(k1, v1, S0, al[:, :1], bl[:, :1])
+    kf = oracle.feature(k1, None, None, None, 1e-6, 0)
+    for h in range(H):
+        kk, vv = kf[0, 0, h][None, :], v1[0, 0, h][None, :]
+        ref = sig(al[0, 0, h]) * S0[0, h] + sig(bl[0, 0, h]) * kk.T @ (vv - kk @ S0[0, h])
+        np.testing.assert_allclose(got[0, h], ref, rtol=1e-12, atol=1e-14)
+    # heads subset leaves the others untouched
+    got = oracle.commit_tokens(k, v, S0, al, bl, heads=[(0, 1)])
+    np.testing.assert_array_equal(got[0, 0], S0[0, 0])
+    assert not np.allclose(got[0, 1], S0[0, 1])
+
+
 def test_state_norm_stays_bounded(oracle):
     """Unit-norm keys and alpha <= alpha_max < 1: |S_T|_F <= max_t |K'^T V'|_F / (1 - alpha_max)."""
     B, L, H, D, T = 1, 12, 2, 8, 60
