@@ -374,6 +374,22 @@ def run_ours(args):
         torch.cuda.synchronize()
         commit_ms[name] = c0.elapsed_time(c1) / 20
     layer.sync_status()
+    # Eq. 4 token by token with per-token gates: needs a context with the extra workspace
+    tok = arl2.Layer(cfg.B, cfg.H, cfg.L, cfg.D, cfg.dtype, device=dev, flags=arl2.ARL2_FLAG_TOKEN_GATES)
+    tok.set_params(wq, wk, wv, cos, sin)
+    tok.reset()
+    gates = tuple(t.to(dev) for t in workload.token_gate_logits(cfg, commit_block))
+    for _ in range(2):
+        tok.commit_tokens(dev_commit[0], dev_commit[1], *gates)
+    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    c0.record()
+    for _ in range(10):
+        tok.commit_tokens(dev_commit[0], dev_commit[1], *gates)
+    c1.record()
+    torch.cuda.synchronize()
+    commit_ms["token_gates"] = c0.elapsed_time(c1) / 10
+    tok.sync_status()
+    del tok
 
     ms_total, ms_e2e, kern_mean = max_over_ranks([ms_total, ms_e2e, statistics.mean(kern_ms)], world, dev)
 

@@ -52,6 +52,8 @@ typedef enum {
 
 /* arl2_config.flags */
 #define ARL2_FLAG_FORCE_SIMT 1u /* bf16 I/O through the plain-FMA kernels (debug / A-B checks) */
+#define ARL2_FLAG_TOKEN_GATES 2u /* reserve workspace for arl2_commit_tokens (3 fp32 copies of a
+                                    [B, H, ceil(L/64)*64, D] tensor)                             */
 
 typedef struct {
     uint32_t struct_size; /* sizeof(arl2_config), for versioning                            */
@@ -136,6 +138,21 @@ int arl2_commit(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
  */
 int arl2_commit_delta(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
                       const float* d_decay_logits, const float* d_beta_logits, void* stream);
+
+/*
+ * State commit with Eq. 4 applied token by token, in order, with per-token gates (the sentence
+ * after Eq. 4): for l = 0..L-1
+ *   S[b,h] <- alpha_l S[b,h] + beta_l K'_l^T (V'_l - K'_l S[b,h]),
+ *   alpha_l = sigmoid(d_alpha_logits[b,l,h]), beta_l = sigmoid(d_beta_logits[b,l,h]),
+ * both uses of S on the right being the state before token l (Eq. 4 as printed).  Computed in
+ * chunkwise form (64 tokens per chunk: a triangular solve per chunk in parallel, then one ordered
+ * pass over the chunks), in fp32 arithmetic for either I/O dtype; bitwise reproducible.
+ * d_alpha_logits, d_beta_logits: [B, L, H] fp32, each may be NULL (gate = 1).  The context must
+ * have been created with ARL2_FLAG_TOKEN_GATES (else ARL2_ERR_WORKSPACE).  K', V' as in
+ * arl2_commit; calls of the three commit entry points may be mixed on one context.
+ */
+int arl2_commit_tokens(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
+                       const float* d_alpha_logits, const float* d_beta_logits, void* stream);
 
 /* S <- 0 for stream `stream_index` (0..B-1) or all streams (-1): Algorithm 1, first line. */
 int arl2_reset(arl2_ctx* ctx, int32_t stream_index, void* stream);

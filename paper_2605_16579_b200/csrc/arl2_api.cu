@@ -27,8 +27,8 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, k_rot, partials, state_bf16, wq_op, wk_op, wv_op, rope_h, total;
-    int nsplit;
+    size_t status, k_rot, partials, state_bf16, wq_op, wk_op, wv_op, rope_h, tok_w, tok_u1, tok_kh, tok_gc, total;
+    int nsplit, nchunk;
 };
 
 bool valid_config(const arl2_config* c)
@@ -84,6 +84,16 @@ Layout make_layout(const arl2_config& c)
     l.wk_op = off;      off += align_up((size_t)c.H * dd * 2);
     l.wv_op = off;      off += align_up((size_t)c.H * dd * 2);
     l.rope_h = off;     off += align_up((size_t)((c.L + 127) / 128) * 128 * (c.D / 2) * 4);
+    // scratch of arl2_commit_tokens, only when the context asks for it
+    l.nchunk = (c.L + kTokenChunk - 1) / kTokenChunk;
+    l.tok_w = l.tok_u1 = l.tok_kh = l.tok_gc = 0;
+    if (c.flags & ARL2_FLAG_TOKEN_GATES) {
+        size_t per = align_up((size_t)c.B * c.H * l.nchunk * kTokenChunk * c.D * sizeof(float));
+        l.tok_w = off;  off += per;
+        l.tok_u1 = off; off += per;
+        l.tok_kh = off; off += per;
+        l.tok_gc = off; off += align_up((size_t)c.B * c.H * l.nchunk * sizeof(float));
+    }
     l.total = off;
     return l;
 }
@@ -329,6 +339,36 @@ int arl2_commit(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
                 const float* d_decay_logits, void* stream)
 {
     return commit_impl(ctx, d_k_clean, d_v_clean, d_decay_logits, false, nullptr, stream);
+}
+
+int arl2_commit_tokens(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
+                       const float* d_alpha_logits, const float* d_beta_logits, void* stream)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    if (!(ctx->cfg.flags & ARL2_FLAG_TOKEN_GATES)) {
+        set_error("commit_tokens: the context was created without ARL2_FLAG_TOKEN_GATES "
+                  "(its workspace has no room for the chunk factors)");
+        return ARL2_ERR_WORKSPACE;
+    }
+    if (!d_k_clean || !d_v_clean) {
+        set_error("commit_tokens: k_clean and v_clean must not be NULL");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    TokenCommitArgs a;
+    a.s = ctx->shape;
+    a.k = d_k_clean; a.v = d_v_clean;
+    a.alpha = d_alpha_logits; a.beta = d_beta_logits;
+    a.wk = ctx->wk; a.wv = ctx->wv;
+    a.rope_cos = ctx->rope_cos; a.rope_sin = ctx->rope_sin;
+    a.state = ctx->state;
+    a.state_bf16 = ctx->use_tc ? reinterpret_cast<__nv_bfloat16*>(ctx->ws + ctx->lay.state_bf16)
+                               : nullptr;
+    a.w = reinterpret_cast<float*>(ctx->ws + ctx->lay.tok_w);
+    a.u1 = reinterpret_cast<float*>(ctx->ws + ctx->lay.tok_u1);
+    a.kh = reinterpret_cast<float*>(ctx->ws + ctx->lay.tok_kh);
+    a.gc = reinterpret_cast<float*>(ctx->ws + ctx->lay.tok_gc);
+    a.nchunk = ctx->lay.nchunk;
+    return account(ctx, simt_commit_tokens(a, ctx->cfg.io_dtype, as_stream(stream)));
 }
 
 int arl2_commit_delta(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,

@@ -62,6 +62,27 @@ struct CommitArgs {
     const float* beta = nullptr;   // [B, L, H] learning-rate logits, or nullptr = 1 (delta only)
 };
 
+// Eq. 4 token by token with per-token gates (chunkwise form): the two launches share these.
+struct TokenCommitArgs {
+    Shape s;
+    const void* k;
+    const void* v;
+    const float* alpha;     // [B, L, H] forget-gate logits, or nullptr = 1
+    const float* beta;      // [B, L, H] learning-rate logits, or nullptr = 1
+    const void* wk;
+    const void* wv;
+    const float* rope_cos;
+    const float* rope_sin;
+    float* state;           // [B, H, D, D] fp32, updated in place
+    __nv_bfloat16* state_bf16;  // operand copy to refresh, or nullptr
+    float* w;               // [B, H, nchunk * 64, D] fp32 scratch
+    float* u1;              // same shape
+    float* kh;              // same shape
+    float* gc;              // [B, H, nchunk] decay of a whole chunk
+    int nchunk;             // ceil(L / 64)
+};
+constexpr int kTokenChunk = 64;
+
 // ---- plain-FMA kernels (arl2_simt.cu) -------------------------------------------------
 // Each returns the number of kernels it launched (>= 0) or a negative arl2_status.
 int simt_rope_k(const Shape& s, int dtype, const void* k, const float* cos_t, const float* sin_t,
@@ -69,6 +90,7 @@ int simt_rope_k(const Shape& s, int dtype, const void* k, const float* cos_t, co
 int simt_step(const StepArgs& a, int dtype, cudaStream_t st);
 int simt_commit(const CommitArgs& a, int dtype, cudaStream_t st);
 int commit_reduce(const CommitArgs& a, cudaStream_t st);  // fixed-order sum + gated decay
+int simt_commit_tokens(const TokenCommitArgs& a, int dtype, cudaStream_t st);
 int fill_zero(void* p, size_t bytes, cudaStream_t st);
 int state_to_bf16(const float* state, __nv_bfloat16* dst, size_t n, cudaStream_t st);
 

@@ -423,6 +423,245 @@ __global__ void __launch_bounds__(NT) simt_commit_partial_kernel(CommitArgs a)
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Eq. 4 token by token with per-token gates, in chunkwise form.  For the tokens j = 0..C-1 of a
+// chunk (C = 64) entering with state S_0, write g_j = alpha_0 ... alpha_j (g_{-1} = 1) and
+// u_j = beta_j (V'_j - K'_j S_{j-1}).  Unrolling S_j = alpha_j S_{j-1} + K'_j^T u_j gives
+//   (I + A) U = diag(beta) V' - diag(beta g_{j-1}) K' S_0,
+//   A_ji = beta_j (g_{j-1} / g_i) <K'_j, K'_i> for i < j (strictly lower triangular),
+//   S_C = g_{C-1} S_0 + Khat^T U,   Khat_i = (g_{C-1} / g_i) K'_i.
+// With T = (I + A)^-1:  U = U1 - W S_0,  U1 = T diag(beta) V',  W = T diag(beta g_{j-1}) K'.
+// Every ratio of g's is a product of alphas, so at most 1.  token_prepare_kernel computes W, U1,
+// Khat and g_{C-1} for every chunk in parallel; token_scan_kernel then walks the chunks in
+// order, each CTA owning 16 columns of one head's state (columns never mix).
+// ---------------------------------------------------------------------------------------------
+constexpr int kTokChunk = kTokenChunk;
+constexpr int LA = kTokChunk + 4;   // row stride of the C x C matrices
+
+template <int D, typename T>
+__global__ void __launch_bounds__(NT) token_prepare_kernel(TokenCommitArgs a)
+{
+    extern __shared__ __align__(16) float smem[];
+    constexpr int LD = D + PAD;
+    float* Ks = smem;                       // [64][LD]  K tile -> K'
+    float* Vs2 = Ks + BM * LD;              // [64][LD]  V tile -> V'
+    float* Ws = Vs2 + BM * LD;              // [64][D]   feature-map rows, then scaled K' / V'
+    float* As = Ws + BN * D;                // [64][LA]  A
+    float* Ts = As + kTokChunk * LA;        // [64][LA]  T = (I + A)^-1
+    float* cl = Ts + kTokChunk * LA;        // [65]      cl[j+1] = log g_j, cl[0] = 0
+    float* bet = cl + kTokChunk + 4;        // [64]      beta_j
+    float* lg = bet + kTokChunk;            // [64]      log alpha_j
+
+    const int tid = threadIdx.x, tx = tid % 16, ty = tid / 16;
+    const int L = a.s.L, H = a.s.H;
+    const int chunk = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int r0 = chunk * kTokChunk;
+    const T* kc = static_cast<const T*>(a.k);
+    const T* vc = static_cast<const T*>(a.v);
+    const T* wk = a.wk ? static_cast<const T*>(a.wk) + (size_t)h * D * D : nullptr;
+    const T* wv = a.wv ? static_cast<const T*>(a.wv) + (size_t)h * D * D : nullptr;
+
+    load_rows<T>(Ks, LD, kc, b, h, r0, 0, D, L, L, H, D, tid);
+    load_rows<T>(Vs2, LD, vc, b, h, r0, 0, D, L, L, H, D, tid);
+    if (tid < kTokChunk) {
+        // tokens past L: alpha = 1, beta = 0 -- they change nothing
+        const int row = r0 + tid;
+        float la = 0.0f, be = 0.0f;
+        if (row < L) {
+            const size_t gi = ((size_t)b * L + row) * H + h;
+            if (a.alpha != nullptr) {
+                const float x = a.alpha[gi];   // log sigmoid(x) = -log(1 + e^-x), stable on both sides
+                la = x >= 0.0f ? -log1pf(expf(-x)) : x - log1pf(expf(x));
+            }
+            be = a.beta != nullptr ? 1.0f / (1.0f + expf(-a.beta[gi])) : 1.0f;
+        }
+        lg[tid] = la;
+        bet[tid] = be;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        float run = 0.0f;
+        cl[0] = 0.0f;
+        for (int j = 0; j < kTokChunk; ++j) {
+            run += lg[j];
+            cl[j + 1] = run;
+        }
+    }
+    feature_tile<D, T>(Ks, Ws, wk, r0, L, a.rope_cos, a.rope_sin, a.s.eps, true, tx, ty, tid);
+    feature_tile<D, T>(Vs2, Ws, wv, r0, L, nullptr, nullptr, a.s.eps, false, tx, ty, tid);
+
+    // A: Gram matrix of the K' rows, masked and weighted
+    {
+        float g[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) g[i][e] = 0.0f;
+        for (int d4 = 0; d4 < D / 4; ++d4) {
+            float4 ar[4], bc[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                ar[i] = *reinterpret_cast<const float4*>(Ks + (ty * 4 + i) * LD + d4 * 4);
+                bc[i] = *reinterpret_cast<const float4*>(Ks + (tx * 4 + i) * LD + d4 * 4);
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    g[i][e] += ar[i].x * bc[e].x + ar[i].y * bc[e].y + ar[i].z * bc[e].z + ar[i].w * bc[e].w;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int row = ty * 4 + i, col = tx * 4 + e;
+                As[row * LA + col] = col < row ? bet[row] * expf(cl[row] - cl[col + 1]) * g[i][e] : 0.0f;
+            }
+    }
+    __syncthreads();
+    // T = (I + A)^-1 by forward substitution: thread c owns column c
+    if (tid < kTokChunk) {
+        float t[kTokChunk];
+#pragma unroll
+        for (int j = 0; j < kTokChunk; ++j) {
+            float acc = j == tid ? 1.0f : 0.0f;
+#pragma unroll
+            for (int i = 0; i < j; ++i) acc -= As[j * LA + i] * t[i];
+            t[j] = acc;
+            Ts[j * LA + tid] = acc;
+        }
+    }
+    __syncthreads();
+
+    const size_t rows_pad = (size_t)a.nchunk * kTokChunk;
+    const size_t base = (((size_t)b * H + h) * rows_pad + r0) * D;
+    // W = T diag(beta g_{j-1}) K', then U1 = T diag(beta) V'
+#pragma unroll 1
+    for (int pass = 0; pass < 2; ++pass) {
+        const float* src = pass == 0 ? Ks : Vs2;
+        for (int idx = tid; idx < kTokChunk * D; idx += NT) {
+            const int j = idx / D, d = idx % D;
+            const float sc = pass == 0 ? bet[j] * expf(cl[j]) : bet[j];
+            Ws[idx] = src[j * LD + d] * sc;
+        }
+        __syncthreads();
+        float acc[4][D / 16];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int e = 0; e < D / 16; ++e) acc[i][e] = 0.0f;
+        tile_gemm<D>(acc, Ts, LA, Ws, tx, ty);
+        float* dst = (pass == 0 ? a.w : a.u1) + base;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int c = 0; c < D / 64; ++c)
+                *reinterpret_cast<float4*>(dst + (size_t)(ty * 4 + i) * D + c * 64 + tx * 4) =
+                    make_float4(acc[i][c * 4 + 0], acc[i][c * 4 + 1], acc[i][c * 4 + 2], acc[i][c * 4 + 3]);
+        __syncthreads();
+    }
+    // Khat = diag(g_{C-1} / g_j) K'
+    for (int idx = tid; idx < kTokChunk * D; idx += NT) {
+        const int j = idx / D, d = idx % D;
+        a.kh[base + idx] = Ks[j * LD + d] * expf(cl[kTokChunk] - cl[j + 1]);
+    }
+    if (tid == 0) a.gc[((size_t)b * H + h) * a.nchunk + chunk] = expf(cl[kTokChunk]);
+}
+
+// The sequential pass: S <- g S + Khat^T (U1 - W S) chunk after chunk, for 16 columns of the
+// state of one (stream, head).  Reads and writes the fp32 state in place and refreshes the
+// bf16 operand copy when one is kept.
+constexpr int kScanCols = 16;
+template <int D>
+__global__ void __launch_bounds__(NT) token_scan_kernel(TokenCommitArgs a)
+{
+    extern __shared__ __align__(16) float smem[];
+    constexpr int LD = D + PAD;
+    constexpr int CP = D * kScanCols / NT;      // state columns per thread in the update: 8 or 4
+    constexpr int TPR = kScanCols / CP;         // threads per state row
+    float* Wt = smem;                           // [64][LD]
+    float* Kt = Wt + kTokChunk * LD;            // [64][LD]
+    float* U1t = Kt + kTokChunk * LD;           // [64][16]
+    float* Ut = U1t + kTokChunk * kScanCols;    // [64][16]
+    float* Ss = Ut + kTokChunk * kScanCols;     // [D][16]
+
+    const int tid = threadIdx.x;
+    const int H = a.s.H;
+    const int e0 = blockIdx.x * kScanCols, h = blockIdx.y, b = blockIdx.z;
+    const size_t bh = (size_t)b * H + h;
+    float* Sg = a.state + bh * D * D;
+    const size_t rows_pad = (size_t)a.nchunk * kTokChunk;
+
+    for (int idx = tid; idx < D * kScanCols; idx += NT)
+        Ss[idx] = Sg[(size_t)(idx / kScanCols) * D + e0 + idx % kScanCols];
+
+    const int r = tid >> 2, cg = tid & 3;       // U phase: row r, columns cg*4 .. cg*4+3
+    const int sd = tid / TPR, sc = (tid % TPR) * CP;   // update phase: state row sd, columns sc ..
+    for (int chunk = 0; chunk < a.nchunk; ++chunk) {
+        const size_t base = (bh * rows_pad + (size_t)chunk * kTokChunk) * D;
+        __syncthreads();   // the previous chunk's reads of the tiles and writes of Ss are done
+        for (int idx = tid; idx < kTokChunk * D / 4; idx += NT) {
+            const int j = idx / (D / 4), d4 = idx % (D / 4);
+            *reinterpret_cast<float4*>(Wt + j * LD + d4 * 4) =
+                *reinterpret_cast<const float4*>(a.w + base + (size_t)j * D + d4 * 4);
+            *reinterpret_cast<float4*>(Kt + j * LD + d4 * 4) =
+                *reinterpret_cast<const float4*>(a.kh + base + (size_t)j * D + d4 * 4);
+        }
+        {
+            const int j = tid >> 2, q = tid & 3;   // 64 rows x 4 float4
+            *reinterpret_cast<float4*>(U1t + j * kScanCols + q * 4) =
+                *reinterpret_cast<const float4*>(a.u1 + base + (size_t)j * D + e0 + q * 4);
+        }
+        const float g = a.gc[bh * a.nchunk + chunk];
+        __syncthreads();
+
+        // U = U1 - W S
+        float4 u = *reinterpret_cast<const float4*>(U1t + r * kScanCols + cg * 4);
+#pragma unroll 4
+        for (int d4 = 0; d4 < D / 4; ++d4) {
+            const float4 w = *reinterpret_cast<const float4*>(Wt + r * LD + d4 * 4);
+            const float wv[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int dd = 0; dd < 4; ++dd) {
+                const float4 s4 = *reinterpret_cast<const float4*>(Ss + (d4 * 4 + dd) * kScanCols + cg * 4);
+                u.x -= wv[dd] * s4.x;
+                u.y -= wv[dd] * s4.y;
+                u.z -= wv[dd] * s4.z;
+                u.w -= wv[dd] * s4.w;
+            }
+        }
+        *reinterpret_cast<float4*>(Ut + r * kScanCols + cg * 4) = u;
+        __syncthreads();
+
+        // S <- g S + Khat^T U   (this thread's CP elements of row sd)
+        float s[CP];
+#pragma unroll
+        for (int e = 0; e < CP; ++e) s[e] = g * Ss[sd * kScanCols + sc + e];
+#pragma unroll 4
+        for (int i = 0; i < kTokChunk; ++i) {
+            const float kv = Kt[i * LD + sd];
+#pragma unroll
+            for (int e4 = 0; e4 < CP / 4; ++e4) {
+                const float4 uu = *reinterpret_cast<const float4*>(Ut + i * kScanCols + sc + e4 * 4);
+                s[e4 * 4 + 0] += kv * uu.x;
+                s[e4 * 4 + 1] += kv * uu.y;
+                s[e4 * 4 + 2] += kv * uu.z;
+                s[e4 * 4 + 3] += kv * uu.w;
+            }
+        }
+        // every thread finished reading Ss in the U phase before the barrier above; in this phase
+        // each thread reads and writes only its own elements
+#pragma unroll
+        for (int e = 0; e < CP; ++e) Ss[sd * kScanCols + sc + e] = s[e];
+    }
+    __syncthreads();
+    for (int idx = tid; idx < D * kScanCols; idx += NT) {
+        const size_t at = (size_t)(idx / kScanCols) * D + e0 + idx % kScanCols;
+        Sg[at] = Ss[idx];
+        if (a.state_bf16 != nullptr) a.state_bf16[bh * D * D + at] = __float2bfloat16_rn(Ss[idx]);
+    }
+}
+
 }  // namespace
 
 // S[b,h] <- sigmoid(a[b,h]) S[b,h] + sum_split partial[b,h,split], splits added in index
@@ -599,6 +838,32 @@ int simt_step(const StepArgs& a, int dtype, cudaStream_t st)
     if (a.s.D == 64 && dtype == ARL2_BF16) return launch_step<64, __nv_bfloat16>(a, st);
     if (a.s.D == 128 && dtype == ARL2_BF16) return launch_step<128, __nv_bfloat16>(a, st);
     set_error("no plain-FMA step kernel for D=%d dtype=%d", a.s.D, dtype);
+    return ARL2_ERR_UNSUPPORTED;
+}
+
+template <int D, typename T>
+int launch_commit_tokens(const TokenCommitArgs& a, cudaStream_t st)
+{
+    size_t smem1 = sizeof(float) * (2 * BM * (D + PAD) + BN * D + 2 * kTokChunk * LA + 3 * kTokChunk + 8);
+    if (int r = set_smem(token_prepare_kernel<D, T>, smem1)) return r;
+    dim3 grid1(a.nchunk, a.s.H, a.s.B);
+    token_prepare_kernel<D, T><<<grid1, NT, smem1, st>>>(a);
+    if (int r = check_launch("token_prepare_kernel")) return r;
+    size_t smem2 = sizeof(float) * (2 * kTokChunk * (D + PAD) + 2 * kTokChunk * kScanCols + D * kScanCols);
+    if (int r = set_smem(token_scan_kernel<D>, smem2)) return r;
+    dim3 grid2(D / kScanCols, a.s.H, a.s.B);
+    token_scan_kernel<D><<<grid2, NT, smem2, st>>>(a);
+    if (int r = check_launch("token_scan_kernel")) return r;
+    return 2;
+}
+
+int simt_commit_tokens(const TokenCommitArgs& a, int dtype, cudaStream_t st)
+{
+    if (a.s.D == 64 && dtype == ARL2_FP32) return launch_commit_tokens<64, float>(a, st);
+    if (a.s.D == 128 && dtype == ARL2_FP32) return launch_commit_tokens<128, float>(a, st);
+    if (a.s.D == 64 && dtype == ARL2_BF16) return launch_commit_tokens<64, __nv_bfloat16>(a, st);
+    if (a.s.D == 128 && dtype == ARL2_BF16) return launch_commit_tokens<128, __nv_bfloat16>(a, st);
+    set_error("no token-gate commit kernel for D=%d dtype=%d", a.s.D, dtype);
     return ARL2_ERR_UNSUPPORTED;
 }
 

@@ -116,6 +116,16 @@ def beta_logits(cfg: Config, block: int, mean: float = -3.0, std: float = 1.0):
     return mean + std * torch.randn(cfg.B, cfg.L, cfg.H, generator=gen, dtype=torch.float32)
 
 
+def token_gate_logits(cfg: Config, block: int, alpha_mean: float = 7.0, beta_mean: float = 0.0):
+    """Per-token forget-gate and learning-rate logits, each [B, L, H] fp32, for the token-sequential
+    commit of one block.  The forget gates sit near 1 (sigmoid(7) = 0.9991) so that a block of a
+    few thousand tokens does not erase the state."""
+    gen = _gen(cfg, block, COMMIT_STEP, salt=8)
+    alpha = alpha_mean + torch.randn(cfg.B, cfg.L, cfg.H, generator=gen, dtype=torch.float32)
+    beta = beta_mean + torch.randn(cfg.B, cfg.L, cfg.H, generator=gen, dtype=torch.float32)
+    return alpha, beta
+
+
 def feature_weights(cfg: Config):
     """W_phi_q, W_phi_k, W_phi_v, each [H, D, D] (in, out) = I + 0.02 N(0, 1), config dtype."""
     gen = _gen(cfg, 0, 0, salt=5)

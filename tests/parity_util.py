@@ -116,6 +116,24 @@ class Pair:
             err = err[mask]
         return float(err.max())
 
+    def commit_tokens(self, kc, vc, alpha, beta, heads=None):
+        """Token-sequential commit with per-token gates on both sides; worst per-head error of S."""
+        d = self.dev
+        dv = lambda t: None if t is None else t.to(d)  # noqa: E731
+        self.layer.commit_tokens(kc.to(d), vc.to(d), dv(alpha), dv(beta))
+        got = self.layer.get_state().numpy().astype(np.float64)
+        self.S_ref = self.oracle.commit_tokens(kc, vc, self.S_ref, alpha, beta, self.wk, self.wv,
+                                               self.cos, self.sin, eps=self.eps, heads=heads)
+        assert np.isfinite(got).all()
+        err = head_errors(got, self.S_ref, head_axis_first=True)
+        if heads is not None:
+            mask = np.zeros(err.shape, dtype=bool)
+            for b, h in heads:
+                mask[b, h] = True
+            self.S_ref[~mask] = got[~mask]
+            err = err[mask]
+        return float(err.max())
+
     def reset(self, stream=-1):
         self.layer.reset(stream)
         self.S_ref = self.oracle.reset(self.S_ref, stream)
