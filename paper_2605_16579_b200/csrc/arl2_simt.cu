@@ -568,22 +568,34 @@ __global__ void __launch_bounds__(NT) token_prepare_kernel(TokenCommitArgs a)
     if (tid == 0) a.gc[((size_t)b * H + h) * a.nchunk + chunk] = expf(cl[kTokChunk]);
 }
 
-// The sequential pass: S <- g S + Khat^T (U1 - W S) chunk after chunk, for 16 columns of the
-// state of one (stream, head).  Reads and writes the fp32 state in place and refreshes the
-// bf16 operand copy when one is kept.
-constexpr int kScanCols = 16;
-template <int D>
+// The sequential pass: S <- g S + Khat^T (U1 - W S) chunk after chunk, for kScanCols columns of
+// the state of one (stream, head).  Reads and writes the fp32 state in place and refreshes the
+// bf16 operand copy when one is kept.  The W tile of the next chunk is fetched (cp.async) while
+// the state update of this chunk runs, the Khat tile while the next U is formed.
+__device__ __forceinline__ void cp_async16(float* dst_smem, const float* src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(
+                     (uint32_t)__cvta_generic_to_shared(dst_smem)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+template <int D, int kScanCols>
 __global__ void __launch_bounds__(NT) token_scan_kernel(TokenCommitArgs a)
 {
     extern __shared__ __align__(16) float smem[];
     constexpr int LD = D + PAD;
-    constexpr int CP = D * kScanCols / NT;      // state columns per thread in the update: 8 or 4
+    constexpr int CG = kScanCols / 4;           // float4 column groups
+    constexpr int RPT = kTokChunk * CG / NT;    // U rows per thread: 1 (16 columns) or 2 (32)
+    constexpr int CP = D * kScanCols / NT;      // state columns per thread in the update
     constexpr int TPR = kScanCols / CP;         // threads per state row
+    static_assert(RPT >= 1 && CP % 4 == 0 && TPR >= 1, "thread mapping");
     float* Wt = smem;                           // [64][LD]
     float* Kt = Wt + kTokChunk * LD;            // [64][LD]
-    float* U1t = Kt + kTokChunk * LD;           // [64][16]
-    float* Ut = U1t + kTokChunk * kScanCols;    // [64][16]
-    float* Ss = Ut + kTokChunk * kScanCols;     // [D][16]
+    float* U1t = Kt + kTokChunk * LD;           // [64][kScanCols]
+    float* Ut = U1t + kTokChunk * kScanCols;    // [64][kScanCols]
+    float* Ss = Ut + kTokChunk * kScanCols;     // [D][kScanCols]
 
     const int tid = threadIdx.x;
     const int H = a.s.H;
@@ -591,47 +603,66 @@ __global__ void __launch_bounds__(NT) token_scan_kernel(TokenCommitArgs a)
     const size_t bh = (size_t)b * H + h;
     float* Sg = a.state + bh * D * D;
     const size_t rows_pad = (size_t)a.nchunk * kTokChunk;
+    const float* wbase = a.w + bh * rows_pad * D;
+    const float* kbase = a.kh + bh * rows_pad * D;
+    const float* ubase = a.u1 + bh * rows_pad * D;
 
+    auto fetch_tile = [&](float* dst, const float* src) {   // 64 x D floats, row stride LD in smem
+        for (int idx = tid; idx < kTokChunk * D / 4; idx += NT) {
+            const int j = idx / (D / 4), d4 = idx % (D / 4);
+            cp_async16(dst + j * LD + d4 * 4, src + (size_t)j * D + d4 * 4);
+        }
+    };
+    auto fetch_u1 = [&](const float* src) {                 // 64 x kScanCols floats
+        for (int idx = tid; idx < kTokChunk * CG; idx += NT) {
+            const int j = idx / CG, q = idx % CG;
+            cp_async16(U1t + j * kScanCols + q * 4, src + (size_t)j * D + e0 + q * 4);
+        }
+    };
+
+    // group order per chunk: {W, U1} then {Khat}
+    fetch_tile(Wt, wbase);
+    fetch_u1(ubase);
+    cp_async_commit();
+    fetch_tile(Kt, kbase);
+    cp_async_commit();
     for (int idx = tid; idx < D * kScanCols; idx += NT)
         Ss[idx] = Sg[(size_t)(idx / kScanCols) * D + e0 + idx % kScanCols];
 
-    const int r = tid >> 2, cg = tid & 3;       // U phase: row r, columns cg*4 .. cg*4+3
-    const int sd = tid / TPR, sc = (tid % TPR) * CP;   // update phase: state row sd, columns sc ..
+    const int cg = tid % CG, r_first = tid / CG;            // U phase: rows r_first + k * (NT / CG)
+    const int sd = tid / TPR, sc = (tid % TPR) * CP;        // update phase: state row sd, columns sc ..
     for (int chunk = 0; chunk < a.nchunk; ++chunk) {
-        const size_t base = (bh * rows_pad + (size_t)chunk * kTokChunk) * D;
-        __syncthreads();   // the previous chunk's reads of the tiles and writes of Ss are done
-        for (int idx = tid; idx < kTokChunk * D / 4; idx += NT) {
-            const int j = idx / (D / 4), d4 = idx % (D / 4);
-            *reinterpret_cast<float4*>(Wt + j * LD + d4 * 4) =
-                *reinterpret_cast<const float4*>(a.w + base + (size_t)j * D + d4 * 4);
-            *reinterpret_cast<float4*>(Kt + j * LD + d4 * 4) =
-                *reinterpret_cast<const float4*>(a.kh + base + (size_t)j * D + d4 * 4);
-        }
-        {
-            const int j = tid >> 2, q = tid & 3;   // 64 rows x 4 float4
-            *reinterpret_cast<float4*>(U1t + j * kScanCols + q * 4) =
-                *reinterpret_cast<const float4*>(a.u1 + base + (size_t)j * D + e0 + q * 4);
-        }
         const float g = a.gc[bh * a.nchunk + chunk];
-        __syncthreads();
+        cp_async_wait<1>();     // W and U1 of this chunk have landed (Khat may still be in flight)
+        __syncthreads();        // ... for every thread; the previous update's writes of Ss are visible
 
         // U = U1 - W S
-        float4 u = *reinterpret_cast<const float4*>(U1t + r * kScanCols + cg * 4);
-#pragma unroll 4
-        for (int d4 = 0; d4 < D / 4; ++d4) {
-            const float4 w = *reinterpret_cast<const float4*>(Wt + r * LD + d4 * 4);
-            const float wv[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-            for (int dd = 0; dd < 4; ++dd) {
-                const float4 s4 = *reinterpret_cast<const float4*>(Ss + (d4 * 4 + dd) * kScanCols + cg * 4);
-                u.x -= wv[dd] * s4.x;
-                u.y -= wv[dd] * s4.y;
-                u.z -= wv[dd] * s4.z;
-                u.w -= wv[dd] * s4.w;
+        for (int k = 0; k < RPT; ++k) {
+            const int r = r_first + k * (NT / CG);
+            float4 u = *reinterpret_cast<const float4*>(U1t + r * kScanCols + cg * 4);
+#pragma unroll 4
+            for (int d4 = 0; d4 < D / 4; ++d4) {
+                const float4 w = *reinterpret_cast<const float4*>(Wt + r * LD + d4 * 4);
+                const float wv[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                for (int dd = 0; dd < 4; ++dd) {
+                    const float4 s4 = *reinterpret_cast<const float4*>(Ss + (d4 * 4 + dd) * kScanCols + cg * 4);
+                    u.x -= wv[dd] * s4.x;
+                    u.y -= wv[dd] * s4.y;
+                    u.z -= wv[dd] * s4.z;
+                    u.w -= wv[dd] * s4.w;
+                }
             }
+            *reinterpret_cast<float4*>(Ut + r * kScanCols + cg * 4) = u;
         }
-        *reinterpret_cast<float4*>(Ut + r * kScanCols + cg * 4) = u;
-        __syncthreads();
+        cp_async_wait<0>();     // Khat of this chunk
+        __syncthreads();        // U complete; nobody reads W, U1 or (others' rows of) Ss any more
+        if (chunk + 1 < a.nchunk) {
+            fetch_tile(Wt, wbase + (size_t)(chunk + 1) * kTokChunk * D);
+            fetch_u1(ubase + (size_t)(chunk + 1) * kTokChunk * D);
+        }
+        cp_async_commit();
 
         // S <- g S + Khat^T U   (this thread's CP elements of row sd)
         float s[CP];
@@ -649,11 +680,13 @@ __global__ void __launch_bounds__(NT) token_scan_kernel(TokenCommitArgs a)
                 s[e4 * 4 + 3] += kv * uu.w;
             }
         }
-        // every thread finished reading Ss in the U phase before the barrier above; in this phase
-        // each thread reads and writes only its own elements
 #pragma unroll
         for (int e = 0; e < CP; ++e) Ss[sd * kScanCols + sc + e] = s[e];
+        __syncthreads();        // every thread is done with Khat and U
+        if (chunk + 1 < a.nchunk) fetch_tile(Kt, kbase + (size_t)(chunk + 1) * kTokChunk * D);
+        cp_async_commit();
     }
+    cp_async_wait<0>();
     __syncthreads();
     for (int idx = tid; idx < D * kScanCols; idx += NT) {
         const size_t at = (size_t)(idx / kScanCols) * D + e0 + idx % kScanCols;
@@ -849,10 +882,11 @@ int launch_commit_tokens(const TokenCommitArgs& a, cudaStream_t st)
     dim3 grid1(a.nchunk, a.s.H, a.s.B);
     token_prepare_kernel<D, T><<<grid1, NT, smem1, st>>>(a);
     if (int r = check_launch("token_prepare_kernel")) return r;
+    constexpr int kScanCols = D / 4;   // 4 CTAs per (stream, head)
     size_t smem2 = sizeof(float) * (2 * kTokChunk * (D + PAD) + 2 * kTokChunk * kScanCols + D * kScanCols);
-    if (int r = set_smem(token_scan_kernel<D>, smem2)) return r;
+    if (int r = set_smem(token_scan_kernel<D, kScanCols>, smem2)) return r;
     dim3 grid2(D / kScanCols, a.s.H, a.s.B);
-    token_scan_kernel<D><<<grid2, NT, smem2, st>>>(a);
+    token_scan_kernel<D, kScanCols><<<grid2, NT, smem2, st>>>(a);
     if (int r = check_launch("token_scan_kernel")) return r;
     return 2;
 }
