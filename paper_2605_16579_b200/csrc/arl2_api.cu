@@ -92,7 +92,7 @@ Layout make_layout(const arl2_config& c)
         l.tok_w = off;  off += per;
         l.tok_u1 = off; off += per;
         l.tok_kh = off; off += per;
-        l.tok_gc = off; off += align_up((size_t)c.B * c.H * l.nchunk * sizeof(float));
+        l.tok_gc = off; off += align_up((size_t)c.B * c.H * (l.nchunk + 1) * sizeof(float));   // up to 2 per 128-token tile
     }
     l.total = off;
     return l;
@@ -368,6 +368,16 @@ int arl2_commit_tokens(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_cle
     a.kh = reinterpret_cast<float*>(ctx->ws + ctx->lay.tok_kh);
     a.gc = reinterpret_cast<float*>(ctx->ws + ctx->lay.tok_gc);
     a.nchunk = ctx->lay.nchunk;
+    if ((reinterpret_cast<uintptr_t>(d_k_clean) | reinterpret_cast<uintptr_t>(d_v_clean)) % 16 != 0) {
+        set_error("commit_tokens: k_clean and v_clean must be 16-byte aligned");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    if (ctx->use_tc)
+        return account(ctx, tc_commit_tokens(
+                                a, reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wk_op),
+                                reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wv_op),
+                                ctx->rope_cos != nullptr ? ctx->ws + ctx->lay.rope_h : nullptr,
+                                reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status), as_stream(stream)));
     return account(ctx, simt_commit_tokens(a, ctx->cfg.io_dtype, as_stream(stream)));
 }
 

@@ -105,6 +105,9 @@ int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* 
 int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat16* wv_op,
               cudaStream_t st);   // partial sums on tensor cores, then commit_reduce
 
+int tc_commit_tokens(const TokenCommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat16* wv_op,
+                     const void* rope_h, uint32_t* status, cudaStream_t st);   // prepare + ordered scan
+
 void set_error(const char* fmt, ...);
 
 }  // namespace arl2

@@ -1093,7 +1093,558 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Token-sequential commit with per-token gates (Eq. 4 token by token), chunkwise, tensor cores.
+// Notation as in the plain-FMA version: for a chunk of C = 64 tokens entering with state S_0,
+//   U = U1 - W S_0,  S_C = g S_0 + Khat^T U,  U1 = T diag(beta) V',  W = T diag(beta g_{j-1}) K',
+//   T = (I + A)^-1,  A_ji = beta_j (g_{j-1} / g_i) <K'_j, K'_i> (i < j),  Khat_i = (g / g_i) K'_i.
+// tc_token_prepare_kernel: one CTA (128 threads, thread = token) per 128-token tile = two chunks.
+//   U_k, U_v (MMA) -> K' -> Gram matrix K' K'^T (MMA) -> A (fp32, shared memory) -> T by forward
+//   substitution (thread = column), stored as a bf16 block-diagonal 128 x 128 operand -> W and U1
+//   (MMA, both chunks at once) -> global: W, Khat, U1 in bf16, chunk decays g in fp32.
+// tc_token_scan_kernel: one CTA per (stream, head) walks the chunks in order (further down).
+// ---------------------------------------------------------------------------------------------
+constexpr int kTPOffWk = 0;                        // maps; later the fp32 matrix A (2 x 64 x 65)
+constexpr int kTPOffWv = kTileBytes;
+constexpr int kTPOffK = 2 * kTileBytes;            // raw K tile -> K' (bf16)
+constexpr int kTPOffV = 3 * kTileBytes;            // raw V tile -> diag(beta) V'
+constexpr int kTPOffKs = 4 * kTileBytes;           // diag(beta g_{j-1}) K'
+constexpr int kTPOffT = 5 * kTileBytes;            // block-diagonal T
+constexpr int kTPOffBars = 6 * kTileBytes;
+constexpr int kTPSmemBytes = kTPOffBars + 1024 + 1024;   // barriers, gate scratch, alignment slack
+constexpr int kTokC = 64;                          // tokens per chunk
+constexpr int kLdA = kTokC + 1;
+static_assert(2 * kTokC * kLdA * 4 <= 2 * kTileBytes, "A fits over the two maps");
+
+enum TPBar : int { kTPBarLoad = 0, kTPBarU, kTPBarG, kTPBarW, kTPNumBars };
+
+struct TcTokenParams {
+    Shape s;
+    const uint4* rope_h;
+    const float* alpha;        // [B, L, H] logits or nullptr
+    const float* beta;
+    __nv_bfloat16* w;          // [B, H, rows_pad, 128]
+    __nv_bfloat16* kh;         // [B, H, rows_pad, 128]
+    __nv_bfloat16* u1;         // [B, H, rows_pad, 128]
+    float* gc;                 // [B, H, 2 * ntile]
+    float* state;              // scan kernel only
+    __nv_bfloat16* state_bf16;
+    uint32_t* status;
+    int ntile;                 // 128-token tiles; rows_pad = 128 * ntile
+    int nchunk;                // ceil(L / 64): chunks the scan walks
+};
+
+__device__ __forceinline__ void store_row_bf16_swizzled(uint8_t* tile, int r, const uint32_t (&x)[128], float f)
+{
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+        uint4 v;
+        v.x = pack_bf16(__uint_as_float(x[c * 8 + 0]) * f, __uint_as_float(x[c * 8 + 1]) * f);
+        v.y = pack_bf16(__uint_as_float(x[c * 8 + 2]) * f, __uint_as_float(x[c * 8 + 3]) * f);
+        v.z = pack_bf16(__uint_as_float(x[c * 8 + 4]) * f, __uint_as_float(x[c * 8 + 5]) * f);
+        v.w = pack_bf16(__uint_as_float(x[c * 8 + 6]) * f, __uint_as_float(x[c * 8 + 7]) * f);
+        const int off = (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+        *reinterpret_cast<uint4*>(tile + off) = v;
+    }
+}
+__device__ __forceinline__ void store_row_bf16_global(__nv_bfloat16* dst, const uint32_t (&x)[128], float f)
+{
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+        uint4 v;
+        v.x = pack_bf16(__uint_as_float(x[c * 8 + 0]) * f, __uint_as_float(x[c * 8 + 1]) * f);
+        v.y = pack_bf16(__uint_as_float(x[c * 8 + 2]) * f, __uint_as_float(x[c * 8 + 3]) * f);
+        v.z = pack_bf16(__uint_as_float(x[c * 8 + 4]) * f, __uint_as_float(x[c * 8 + 5]) * f);
+        v.w = pack_bf16(__uint_as_float(x[c * 8 + 6]) * f, __uint_as_float(x[c * 8 + 7]) * f);
+        *reinterpret_cast<uint4*>(dst + c * 8) = v;
+    }
+}
+
+__global__ void __launch_bounds__(128, 1)
+tc_token_prepare_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                        const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv,
+                        const TcTokenParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                               ~static_cast<uintptr_t>(1023));
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t bars = smem_base + kTPOffBars;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kTPOffBars + kTPNumBars * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kTPOffBars + kTPNumBars * 8 + 4);
+    float* cl_s = reinterpret_cast<float*>(smem + kTPOffBars + 64);          // [128] log g_j (inclusive)
+    float* wsum = reinterpret_cast<float*>(smem + kTPOffBars + 64 + 512);    // [4] warp totals
+    const Abort ab{abort_flag, p.status};
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tile = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int L = p.s.L, H = p.s.H;
+    const int row = tile * kTile + tid;          // this thread's token
+    const int chunk = tid >> 6, jj = tid & 63;   // chunk of the tile, index in the chunk
+
+    if (tid == 0) {
+        for (int i = 0; i < kTPNumBars; ++i) mbar_init(bars + 8 * i, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    // the off-diagonal blocks of T stay zero
+    for (int i = tid; i < kTileBytes / 16; i += 128)
+        reinterpret_cast<uint4*>(smem + kTPOffT)[i] = make_uint4(0u, 0u, 0u, 0u);
+    fence_proxy_async_smem();
+    if (warp == 0) {
+        tmem_alloc(smem_u32(tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+
+    bool ok = true;
+    if (tid == 0) {
+        const uint32_t bar = bars + 8 * kTPBarLoad;
+        mbar_expect_tx(bar, 4 * kTileBytes);
+        tma_load_2d(smem_base + kTPOffWk, &tm_wk, bar, 0, h * kTile);
+        tma_load_2d(smem_base + kTPOffWk + kHalfBytes, &tm_wk, bar, 64, h * kTile);
+        tma_load_2d(smem_base + kTPOffWv, &tm_wv, bar, 0, h * kTile);
+        tma_load_2d(smem_base + kTPOffWv + kHalfBytes, &tm_wv, bar, 64, h * kTile);
+        tma_load_4d(smem_base + kTPOffK, &tm_k, bar, 0, h, tile * kTile, b);
+        tma_load_4d(smem_base + kTPOffK + kHalfBytes, &tm_k, bar, 64, h, tile * kTile, b);
+        tma_load_4d(smem_base + kTPOffV, &tm_v, bar, 0, h, tile * kTile, b);
+        tma_load_4d(smem_base + kTPOffV + kHalfBytes, &tm_v, bar, 64, h, tile * kTile, b);
+    }
+
+    // ---- gates: log alpha_j, beta_j, cumulative decay within the chunk (tokens past L: 1 and 0)
+    float la = 0.0f, be = 0.0f;
+    if (row < L) {
+        const size_t gi = ((size_t)b * L + row) * H + h;
+        if (p.alpha != nullptr) {
+            const float x = __ldg(p.alpha + gi);
+            la = x >= 0.0f ? -log1pf(expf(-x)) : x - log1pf(expf(x));
+        }
+        be = p.beta != nullptr ? 1.0f / (1.0f + expf(-__ldg(p.beta + gi))) : 1.0f;
+    }
+    float cl = la;   // inclusive scan over the 64 tokens of the chunk (two warps)
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const float up = __shfl_up_sync(0xffffffffu, cl, off);
+        if (lane >= off) cl += up;
+    }
+    if (lane == 31) wsum[warp] = cl;
+    __syncthreads();
+    if (warp & 1) cl += wsum[warp - 1];
+    cl_s[tid] = cl;
+    __syncthreads();
+    const float cl_total = cl_s[chunk * kTokC + kTokC - 1];
+    const float cl_excl = cl - la;
+
+    constexpr uint32_t kLboK = 1u << 16;
+    constexpr uint32_t kLboMN = (uint32_t)(kHalfBytes >> 4) << 16;
+    const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0, 0) >> 32);
+    auto desc64 = [&](uint32_t lo) {
+        uint64_t d;
+        asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(desc_hi));
+        return d;
+    };
+    constexpr uint32_t idesc_kk = idesc_bf16(kTile, kTile, 0, 0);   // both operands d-major
+    constexpr uint32_t idesc_kn = idesc_bf16(kTile, kTile, 0, 1);   // A K-major, B rows = contraction index
+    auto koff_k = [](int ks) { return (uint32_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4); };
+
+    // ---- U_k = K W_phi_k, U_v = V W_phi_v
+    if (tid == 0) {
+        ok = wait_bar(bars + 8 * kTPBarLoad, 0, ab, 90);
+        if (ok) {
+            tc_fence_after();
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const uint32_t a_lo = ((smem_base + (u ? kTPOffV : kTPOffK)) >> 4) | kLboK;
+                const uint32_t b_lo = ((smem_base + (u ? kTPOffWv : kTPOffWk)) >> 4) | kLboK;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    mma_ss(tmem_base + u * kTile, desc64(a_lo + koff_k(ks)), desc64(b_lo + koff_k(ks)), idesc_kk, ks > 0);
+            }
+            mma_commit(bars + 8 * kTPBarU);
+        }
+    }
+    uint32_t sreg[128];
+    bool alive = wait_bar(bars + 8 * kTPBarU, 0, ab, 91);
+    const size_t grow = (((size_t)b * H + h) * p.ntile + tile) * kTile + tid;   // row of the scratch tensors
+    if (alive) {
+        tc_fence_after();
+        // ---- K' = L2Norm(RoPE(U_k)); three copies: K' (Gram), scaled for W, scaled for the scan
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            tmem_ld32(lane_base + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
+        tmem_wait_ld();
+        if (p.rope_h != nullptr) {
+            const uint4* tab = p.rope_h + ((size_t)(row >> 5) * 16) * 32 + (row & 31);
+            uint4 cs[16];
+#pragma unroll
+            for (int c = 0; c < 16; ++c) cs[c] = __ldg(tab + c * 32);
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+                const uint32_t h2[4] = {cs[c].x, cs[c].y, cs[c].z, cs[c].w};
+#pragma unroll
+                for (int m = 0; m < 4; ++m) {
+                    float cc, s1;
+                    unpack_cs(h2[m], cc, s1);
+                    const float x0 = __uint_as_float(sreg[c * 8 + 2 * m]);
+                    const float x1 = __uint_as_float(sreg[c * 8 + 2 * m + 1]);
+                    sreg[c * 8 + 2 * m] = __float_as_uint(x0 * cc - x1 * s1);
+                    sreg[c * 8 + 2 * m + 1] = __float_as_uint(x0 * s1 + x1 * cc);
+                }
+            }
+        }
+        float ss4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+        for (int c = 0; c < 128; c += 4) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                ss4[k] = fmaf(__uint_as_float(sreg[c + k]), __uint_as_float(sreg[c + k]), ss4[k]);
+        }
+        const float f = rsqrtf((ss4[0] + ss4[1]) + (ss4[2] + ss4[3]) + p.s.eps);
+        store_row_bf16_swizzled(smem + kTPOffK, tid, sreg, f);
+        store_row_bf16_swizzled(smem + kTPOffKs, tid, sreg, f * be * expf(cl_excl));
+        store_row_bf16_global(p.kh + grow * kTile, sreg, f * expf(cl_total - cl));
+        // ---- diag(beta) V'
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            tmem_ld32(lane_base + kTile + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
+        tmem_wait_ld();
+        store_row_bf16_swizzled(smem + kTPOffV, tid, sreg, be);
+    }
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncthreads();
+
+    // ---- Gram matrix K' K'^T -> TMEM columns 256-383 (row = token j, column = token i)
+    if (tid == 0 && ok && !*abort_flag) {
+        tc_fence_after();
+        const uint32_t k_lo = ((smem_base + kTPOffK) >> 4) | kLboK;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+            mma_ss(tmem_base + 2 * kTile, desc64(k_lo + koff_k(ks)), desc64(k_lo + koff_k(ks)), idesc_kk, ks > 0);
+        mma_commit(bars + 8 * kTPBarG);
+    }
+    alive = alive && wait_bar(bars + 8 * kTPBarG, 0, ab, 92);
+    float* As = reinterpret_cast<float*>(smem + kTPOffWk);   // the maps are dead: U_k, U_v are complete
+    if (alive) {
+        tc_fence_after();
+        // this token's row of A: only the columns of its own chunk, strictly below the diagonal
+        uint32_t g[64];
+        tmem_ld32(lane_base + 2 * kTile + chunk * kTokC, *reinterpret_cast<uint32_t(*)[32]>(&g[0]));
+        tmem_ld32(lane_base + 2 * kTile + chunk * kTokC + 32, *reinterpret_cast<uint32_t(*)[32]>(&g[32]));
+        tmem_wait_ld();
+        float* arow = As + (chunk * kTokC + jj) * kLdA;
+#pragma unroll
+        for (int i = 0; i < kTokC; ++i) {
+            const float w = be * expf(cl_excl - cl_s[chunk * kTokC + i]);
+            arow[i] = i < jj ? w * __uint_as_float(g[i]) : 0.0f;
+        }
+    }
+    __syncthreads();
+    // ---- T = (I + A)^-1 by forward substitution; this thread owns column jj of its chunk's T
+    if (alive) {
+        const float* Ac = As + chunk * kTokC * kLdA;
+        float t[kTokC];
+#pragma unroll
+        for (int j = 0; j < kTokC; ++j) {
+            float acc = j == jj ? 1.0f : 0.0f;
+#pragma unroll
+            for (int i = 0; i < j; ++i) acc -= Ac[j * kLdA + i] * t[i];
+            t[j] = acc;
+        }
+        // element (row r = chunk*64 + j, column c = chunk*64 + jj) of the K-major swizzled bf16 tile
+        const int cglob = chunk * kTokC + jj;
+        uint8_t* tt = smem + kTPOffT + (cglob >> 6) * kHalfBytes + (cglob & 7) * 2;
+        const int c16 = (cglob & 63) >> 3;
+#pragma unroll
+        for (int j = 0; j < kTokC; ++j) {
+            const int r = chunk * kTokC + j;
+            *reinterpret_cast<__nv_bfloat16*>(tt + r * 128 + ((c16 ^ (r & 7)) << 4)) = __float2bfloat16_rn(t[j]);
+        }
+    }
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncthreads();
+
+    // ---- W = T diag(beta g_{j-1}) K' -> columns 0-127, U1 = T diag(beta) V' -> columns 128-255
+    if (tid == 0 && ok && !*abort_flag) {
+        tc_fence_after();
+        const uint32_t t_lo = ((smem_base + kTPOffT) >> 4) | kLboK;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const uint32_t b_lo = ((smem_base + (u ? kTPOffV : kTPOffKs)) >> 4) | kLboMN;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks)
+                mma_ss(tmem_base + u * kTile, desc64(t_lo + koff_k(ks)), desc64(b_lo + (uint32_t)(ks * (2048 >> 4))),
+                       idesc_kn, ks > 0);
+        }
+        mma_commit(bars + 8 * kTPBarW);
+    }
+    alive = alive && wait_bar(bars + 8 * kTPBarW, 0, ab, 93);
+    if (alive) {
+        tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            tmem_ld32(lane_base + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
+        tmem_wait_ld();
+        store_row_bf16_global(p.w + grow * kTile, sreg, 1.0f);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            tmem_ld32(lane_base + kTile + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
+        tmem_wait_ld();
+        store_row_bf16_global(p.u1 + grow * kTile, sreg, 1.0f);
+        if (jj == kTokC - 1)
+            p.gc[(((size_t)b * H + h) * p.ntile + tile) * 2 + chunk] = expf(cl_total);
+    }
+    if (tid == 0 && (!ok || *abort_flag)) drain_bar(bars + 8 * kTPBarLoad, 0);   // no bulk copy left in flight
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// tc_token_scan_kernel: one CTA (128 threads) per (stream, head); the fp32 state lives in TMEM
+// (row = key dim d, 128 columns) for the whole walk.  Per chunk:
+//   Y = W_c S            MMA, A = W tile (128 rows fetched, the first 64 are the chunk), B = bf16 copy of S
+//   U = U1_c - Y         threads 0-63 (one per token), written as a bf16 operand tile
+//   S += Khat_c^T U      MMA over the chunk's 64 tokens, accumulating on g_c S (scaled beforehand)
+//   bf16 copy of the new S for the next chunk; S scaled by g_{c+1} in the same pass
+// The tiles of chunk c + 2 are fetched by TMA as soon as chunk c has released its buffers.
+constexpr int kTSOffS = 0;                           // bf16 S, [d][e], 128 rows
+constexpr int kTSOffW = kTileBytes;                  // 2 x 32 KB: W tiles (128 rows)
+constexpr int kTSOffKh = 3 * kTileBytes;             // 2 x 16 KB: Khat chunks (64 rows)
+constexpr int kTSOffU1 = 4 * kTileBytes;             // 2 x 16 KB: U1 chunks
+constexpr int kTSOffU = 5 * kTileBytes;              // 16 KB: U operand
+constexpr int kTSOffBars = 5 * kTileBytes + kHalfBytes;
+constexpr int kTSSmemBytes = kTSOffBars + 128 + 1024;
+constexpr int kChunkHalf = kTokC * 128;              // bytes of a 64-row, 64-column box
+constexpr uint32_t kChunkTx = kTileBytes + 4 * kChunkHalf;   // W tile + Khat + U1 per chunk
+
+enum TSBar : int { kTSBarS0 = 0, kTSBarFull0, kTSBarFull1, kTSBarY, kTSBarS2, kTSNumBars };
+
+__global__ void __launch_bounds__(128, 1)
+tc_token_scan_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_kh,
+                     const __grid_constant__ CUtensorMap tm_u1, const __grid_constant__ CUtensorMap tm_s,
+                     const TcTokenParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                               ~static_cast<uintptr_t>(1023));
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t bars = smem_base + kTSOffBars;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kTSOffBars + kTSNumBars * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kTSOffBars + kTSNumBars * 8 + 4);
+    const Abort ab{abort_flag, p.status};
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int h = blockIdx.x, b = blockIdx.y;
+    const size_t bh = (size_t)b * p.s.H + h;
+    const int rows_pad = p.ntile * kTile;
+    const int nchunk = p.nchunk;
+    const float* gc = p.gc + bh * 2 * p.ntile;
+
+    if (tid == 0) {
+        for (int i = 0; i < kTSNumBars; ++i) mbar_init(bars + 8 * i, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+        fence_proxy_async_smem();
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(tmem_slot), 256);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+
+    int loads_issued = 0;
+    auto load_chunk = [&](int c) {
+        const uint32_t bar = bars + 8 * (kTSBarFull0 + (c & 1));
+        const int r0 = (int)(bh * rows_pad) + c * kTokC;
+        mbar_expect_tx(bar, kChunkTx);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            tma_load_2d(smem_base + kTSOffW + (c & 1) * kTileBytes + half * kHalfBytes, &tm_w, bar, half * 64, r0);
+            tma_load_2d(smem_base + kTSOffKh + (c & 1) * kHalfBytes + half * kChunkHalf, &tm_kh, bar, half * 64, r0);
+            tma_load_2d(smem_base + kTSOffU1 + (c & 1) * kHalfBytes + half * kChunkHalf, &tm_u1, bar, half * 64, r0);
+        }
+        ++loads_issued;
+    };
+    if (tid == 0) {
+        mbar_expect_tx(bars + 8 * kTSBarS0, kTileBytes);
+        tma_load_2d(smem_base + kTSOffS, &tm_s, bars + 8 * kTSBarS0, 0, (int)bh * kTile);
+        tma_load_2d(smem_base + kTSOffS + kHalfBytes, &tm_s, bars + 8 * kTSBarS0, 64, (int)bh * kTile);
+        load_chunk(0);
+        if (nchunk > 1) load_chunk(1);
+    }
+
+    // fp32 state row d = tid into TMEM columns 128-255, already scaled by the first chunk's decay
+    float* srow = p.state + (bh * kTile + tid) * kTile;
+    {
+        const float g0 = __ldg(gc);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t x[32];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float4 v = *reinterpret_cast<const float4*>(srow + c * 32 + e * 4);
+                x[e * 4 + 0] = __float_as_uint(v.x * g0);
+                x[e * 4 + 1] = __float_as_uint(v.y * g0);
+                x[e * 4 + 2] = __float_as_uint(v.z * g0);
+                x[e * 4 + 3] = __float_as_uint(v.w * g0);
+            }
+            tmem_st32(lane_base + kTile + c * 32, x);
+        }
+        tmem_wait_st();
+    }
+    tc_fence_before();
+    __syncthreads();
+
+    constexpr uint32_t kLboK = 1u << 16;
+    constexpr uint32_t kLboMN = (uint32_t)(kHalfBytes >> 4) << 16;     // 128-row tiles
+    constexpr uint32_t kLboMN64 = (uint32_t)(kChunkHalf >> 4) << 16;   // 64-row tiles
+    const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0, 0) >> 32);
+    auto desc64 = [&](uint32_t lo) {
+        uint64_t d;
+        asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(desc_hi));
+        return d;
+    };
+    constexpr uint32_t idesc_kn = idesc_bf16(kTile, kTile, 0, 1);
+    constexpr uint32_t idesc_nn = idesc_bf16(kTile, kTile, 1, 1);
+
+    bool ok = true, alive = true;
+    for (int c = 0; c < nchunk; ++c) {
+        const int s = c & 1;
+        const uint32_t par = (uint32_t)((c >> 1) & 1);
+        // ---- Y = W_c S
+        if (tid == 0) {
+            if (c == 0) ok = wait_bar(bars + 8 * kTSBarS0, 0, ab, 100);
+            if (ok) ok = wait_bar(bars + 8 * (kTSBarFull0 + s), par, ab, 101);
+            if (ok) {
+                tc_fence_after();
+                const uint32_t a_lo = ((smem_base + kTSOffW + s * kTileBytes) >> 4) | kLboK;
+                const uint32_t b_lo = ((smem_base + kTSOffS) >> 4) | kLboMN;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t koff = (uint32_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
+                    mma_ss(tmem_base, desc64(a_lo + koff), desc64(b_lo + (uint32_t)(ks * (2048 >> 4))), idesc_kn, ks > 0);
+                }
+                mma_commit(bars + 8 * kTSBarY);
+            }
+        }
+        alive = wait_bar(bars + 8 * kTSBarY, (uint32_t)(c & 1), ab, 102);
+        // the chunk's tiles landed before the MMA above was issued; waiting here as well makes
+        // the bulk copy's writes visible to this thread
+        if (alive) alive = wait_bar(bars + 8 * (kTSBarFull0 + s), par, ab, 103);
+        tc_fence_after();
+        // ---- U = U1_c - Y for the chunk's 64 tokens (threads 0-63), as a bf16 operand tile
+        if (alive && tid < kTokC) {
+            const uint8_t* u1t = smem + kTSOffU1 + s * kHalfBytes;
+            uint8_t* ut = smem + kTSOffU;
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+                uint32_t y[32];
+                tmem_ld32(lane_base + cc * 32, y);
+                tmem_wait_ld();
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    const int q = cc * 4 + q4;   // 16-byte chunk of the row: columns 8q .. 8q+7
+                    const int off = (q >> 3) * kChunkHalf + tid * 128 + (((q & 7) ^ (tid & 7)) << 4);
+                    const uint4 u1 = *reinterpret_cast<const uint4*>(u1t + off);
+                    const uint32_t uw[4] = {u1.x, u1.y, u1.z, u1.w};
+                    uint32_t o[4];
+#pragma unroll
+                    for (int m = 0; m < 4; ++m) {
+                        const float lo = __uint_as_float(uw[m] << 16) - __uint_as_float(y[q4 * 8 + 2 * m]);
+                        const float hi = __uint_as_float(uw[m] & 0xFFFF0000u) - __uint_as_float(y[q4 * 8 + 2 * m + 1]);
+                        o[m] = pack_bf16(lo, hi);
+                    }
+                    *reinterpret_cast<uint4*>(ut + off) = make_uint4(o[0], o[1], o[2], o[3]);
+                }
+            }
+        }
+        fence_proxy_async_smem();
+        tc_fence_before();
+        if (__syncthreads_or(!alive)) break;   // every thread leaves together
+        // ---- S += Khat_c^T U
+        if (tid == 0 && ok) {
+            tc_fence_after();
+            const uint32_t a_lo = ((smem_base + kTSOffKh + s * kHalfBytes) >> 4) | kLboMN64;
+            const uint32_t b_lo = ((smem_base + kTSOffU) >> 4) | kLboMN64;
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+                mma_ss(tmem_base + kTile, desc64(a_lo + (uint32_t)(ks * (2048 >> 4))),
+                       desc64(b_lo + (uint32_t)(ks * (2048 >> 4))), idesc_nn, 1u);
+            mma_commit(bars + 8 * kTSBarS2);
+        }
+        alive = wait_bar(bars + 8 * kTSBarS2, (uint32_t)(c & 1), ab, 104);
+        tc_fence_after();
+        if (alive && tid == 0 && c + 2 < nchunk) load_chunk(c + 2);   // both MMAs that read slot s are done
+        // ---- the new S: bf16 operand copy, and the fp32 rows scaled for the next chunk (or stored)
+        const bool last = c + 1 == nchunk;
+        const float gn = last ? 1.0f : __ldg(gc + c + 1);
+#pragma unroll
+        for (int cc = 0; cc < 4 && alive; ++cc) {
+            uint32_t x[32];
+            tmem_ld32(lane_base + kTile + cc * 32, x);
+            tmem_wait_ld();
+            if (!last) {
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    const int q = cc * 4 + q4;
+                    const int off = (q >> 3) * kHalfBytes + tid * 128 + (((q & 7) ^ (tid & 7)) << 4);
+                    *reinterpret_cast<uint4*>(smem + kTSOffS + off) =
+                        make_uint4(pack_bf16(__uint_as_float(x[q4 * 8 + 0]), __uint_as_float(x[q4 * 8 + 1])),
+                                   pack_bf16(__uint_as_float(x[q4 * 8 + 2]), __uint_as_float(x[q4 * 8 + 3])),
+                                   pack_bf16(__uint_as_float(x[q4 * 8 + 4]), __uint_as_float(x[q4 * 8 + 5])),
+                                   pack_bf16(__uint_as_float(x[q4 * 8 + 6]), __uint_as_float(x[q4 * 8 + 7])));
+                }
+#pragma unroll
+                for (int e = 0; e < 32; ++e) x[e] = __float_as_uint(__uint_as_float(x[e]) * gn);
+                tmem_st32(lane_base + kTile + cc * 32, x);
+            } else {
+                __nv_bfloat16* mrow = p.state_bf16 + (bh * kTile + tid) * kTile;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    *reinterpret_cast<uint4*>(srow + cc * 32 + e * 4) = make_uint4(x[e * 4], x[e * 4 + 1], x[e * 4 + 2], x[e * 4 + 3]);
+                }
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4)
+                    *reinterpret_cast<uint4*>(mrow + cc * 32 + q4 * 8) =
+                        make_uint4(pack_bf16(__uint_as_float(x[q4 * 8 + 0]), __uint_as_float(x[q4 * 8 + 1])),
+                                   pack_bf16(__uint_as_float(x[q4 * 8 + 2]), __uint_as_float(x[q4 * 8 + 3])),
+                                   pack_bf16(__uint_as_float(x[q4 * 8 + 4]), __uint_as_float(x[q4 * 8 + 5])),
+                                   pack_bf16(__uint_as_float(x[q4 * 8 + 6]), __uint_as_float(x[q4 * 8 + 7])));
+            }
+        }
+        tmem_wait_st();
+        fence_proxy_async_smem();
+        tc_fence_before();
+        if (__syncthreads_or(!alive)) break;
+    }
+    if (tid == 0 && (!ok || *abort_flag)) {
+        // leave no bulk copy in flight into this CTA's shared memory
+        drain_bar(bars + 8 * kTSBarS0, 0);
+        for (int m = (loads_issued > 2 ? loads_issued - 2 : 0); m < loads_issued; ++m)
+            drain_bar(bars + 8 * (kTSBarFull0 + (m & 1)), (uint32_t)((m >> 1) & 1));
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 256);
+    }
+}
+
 // The rotation table in the form the step kernel reads: half2 (cos, sin) per pair, 16 vectors of
+
 // 4 pairs per token, stored so that the 32 tokens a warp owns are interleaved -- vector c of
 // token l sits at uint4 index ((l / 32) * 16 + c) * 32 + l % 32 -- and each of a warp's 16 loads is
 // one contiguous 512-byte segment.  Tokens past L (padding up to a whole tile) read as zero.
@@ -1160,13 +1711,13 @@ int make_map_blhd(CUtensorMap* m, const void* base, const Shape& s)
 }
 
 // [rows, 128] bf16 row-major; box = 64 columns x 128 rows.
-int make_map_rows(CUtensorMap* m, const void* base, size_t rows)
+int make_map_rows(CUtensorMap* m, const void* base, size_t rows, int box_rows = kTile)
 {
     EncodeTiledFn fn = encode_fn();
     if (fn == nullptr) { set_error("cuTensorMapEncodeTiled is not available from the driver"); return ARL2_ERR_CUDA; }
     cuuint64_t dims[2] = {(cuuint64_t)kTile, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)kTile * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)kTile};
+    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -1288,6 +1839,57 @@ int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat
     int m = commit_reduce(a, st);
     if (m < 0) return m;
     return 1 + m;
+}
+
+// Eq. 4 token by token with per-token gates on the tensor-core path (bf16 I/O, D = 128).  The
+// scratch tensors of `a` (sized for the fp32 plain-FMA version) are used as bf16 here.
+int tc_commit_tokens(const TokenCommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat16* wv_op,
+                     const void* rope_h, uint32_t* status, cudaStream_t st)
+{
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_token_prepare_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kTPSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(tc_token_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSSmemBytes);
+        if (e != cudaSuccess) { set_error("cudaFuncSetAttribute(token kernels): %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
+        attr_set = true;
+    }
+    if (a.state_bf16 == nullptr) { set_error("tc_commit_tokens: needs the bf16 copy of the state"); return ARL2_ERR_INVALID_ARG; }
+    TcTokenParams p;
+    p.s = a.s;
+    p.rope_h = static_cast<const uint4*>(rope_h);
+    p.alpha = a.alpha;
+    p.beta = a.beta;
+    p.w = reinterpret_cast<__nv_bfloat16*>(a.w);
+    p.kh = reinterpret_cast<__nv_bfloat16*>(a.kh);
+    p.u1 = reinterpret_cast<__nv_bfloat16*>(a.u1);
+    p.gc = a.gc;
+    p.state = a.state;
+    p.state_bf16 = a.state_bf16;
+    p.status = status;
+    p.ntile = (a.s.L + kTile - 1) / kTile;
+    p.nchunk = (a.s.L + kTokC - 1) / kTokC;
+    const size_t rows = (size_t)a.s.B * a.s.H * p.ntile * kTile;
+    if (rows >= ((size_t)1 << 31)) { set_error("tc_commit_tokens: too many rows"); return ARL2_ERR_UNSUPPORTED; }
+    CUtensorMap tm_k, tm_v, tm_wk, tm_wv, tm_w, tm_kh, tm_u1, tm_s;
+    if (int r = make_map_blhd(&tm_k, a.k, a.s)) return r;
+    if (int r = make_map_blhd(&tm_v, a.v, a.s)) return r;
+    if (int r = make_map_rows(&tm_wk, wk_op, (size_t)a.s.H * kTile)) return r;
+    if (int r = make_map_rows(&tm_wv, wv_op, (size_t)a.s.H * kTile)) return r;
+    if (int r = make_map_rows(&tm_w, p.w, rows)) return r;
+    if (int r = make_map_rows(&tm_kh, p.kh, rows, kTokC)) return r;
+    if (int r = make_map_rows(&tm_u1, p.u1, rows, kTokC)) return r;
+    if (int r = make_map_rows(&tm_s, a.state_bf16, (size_t)a.s.B * a.s.H * kTile)) return r;
+    dim3 grid1(p.ntile, a.s.H, a.s.B);
+    tc_token_prepare_kernel<<<grid1, 128, kTPSmemBytes, st>>>(tm_k, tm_v, tm_wk, tm_wv, p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_error("launch of tc_token_prepare_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
+    dim3 grid2(a.s.H, a.s.B);
+    tc_token_scan_kernel<<<grid2, 128, kTSSmemBytes, st>>>(tm_w, tm_kh, tm_u1, tm_s, p);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { set_error("launch of tc_token_scan_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
+    return 2;
 }
 
 }  // namespace arl2
