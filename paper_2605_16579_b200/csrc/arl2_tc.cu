@@ -1113,7 +1113,7 @@ constexpr int kTPOffT = 5 * kTileBytes;            // block-diagonal T
 constexpr int kTPOffBars = 6 * kTileBytes;
 constexpr int kTPSmemBytes = kTPOffBars + 1024 + 1024;   // barriers, gate scratch, alignment slack
 constexpr int kTokC = 64;                          // tokens per chunk
-constexpr int kLdA = kTokC + 1;
+constexpr int kLdA = kTokC + 4;   // 16-byte aligned rows, conflict-free 16-byte stores
 static_assert(2 * kTokC * kLdA * 4 <= 2 * kTileBytes, "A fits over the two maps");
 
 enum TPBar : int { kTPBarLoad = 0, kTPBarU, kTPBarG, kTPBarW, kTPNumBars };
@@ -1338,9 +1338,15 @@ tc_token_prepare_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
         tmem_wait_ld();
         float* arow = As + (chunk * kTokC + jj) * kLdA;
 #pragma unroll
-        for (int i = 0; i < kTokC; ++i) {
-            const float w = be * expf(cl_excl - cl_s[chunk * kTokC + i]);
-            arow[i] = i < jj ? w * __uint_as_float(g[i]) : 0.0f;
+        for (int i4 = 0; i4 < kTokC / 4; ++i4) {
+            float v[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int i = i4 * 4 + k;
+                const float w = be * __expf(cl_excl - cl_s[chunk * kTokC + i]);
+                v[k] = i < jj ? w * __uint_as_float(g[i]) : 0.0f;
+            }
+            *reinterpret_cast<float4*>(arow + i4 * 4) = make_float4(v[0], v[1], v[2], v[3]);
         }
     }
     __syncthreads();
@@ -1350,10 +1356,18 @@ tc_token_prepare_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
         float t[kTokC];
 #pragma unroll
         for (int j = 0; j < kTokC; ++j) {
-            float acc = j == jj ? 1.0f : 0.0f;
+            // row j of A in 16-byte pieces (the same address for the whole chunk: a broadcast),
+            // four independent partial sums
+            float acc[4] = {j == jj ? 1.0f : 0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-            for (int i = 0; i < j; ++i) acc -= Ac[j * kLdA + i] * t[i];
-            t[j] = acc;
+            for (int i4 = 0; i4 < (j + 3) / 4; ++i4) {
+                const float4 a4 = *reinterpret_cast<const float4*>(Ac + j * kLdA + i4 * 4);
+                const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if (i4 * 4 + k < j) acc[k] -= av[k] * t[i4 * 4 + k];
+            }
+            t[j] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
         }
         // element (row r = chunk*64 + j, column c = chunk*64 + jj) of the K-major swizzled bf16 tile
         const int cglob = chunk * kTokC + jj;
