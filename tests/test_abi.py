@@ -65,6 +65,13 @@ def test_workspace_bytes_and_argument_errors(lib):
     # NULL context
     assert lib.arl2_reset(None, -1, None) == -1
     assert lib.arl2_commit(None, None, None, None, None) == -1
+    assert lib.arl2_commit_delta(None, None, None, None, None, None) == -1
+    assert lib.arl2_commit_tokens(None, None, None, None, None, None) == -1
+    # the token-gate scratch is reserved only on request: three [B, H, ceil(L/128)*128, D] fp32 tensors
+    c0 = arl2.make_config(1, 12, 4680, 128, "bf16")
+    c1 = arl2.make_config(1, 12, 4680, 128, "bf16", flags=arl2.ARL2_FLAG_TOKEN_GATES)
+    extra = arl2.arl2_workspace_bytes(c1) - arl2.arl2_workspace_bytes(c0)
+    assert 3 * 12 * 4680 * 128 * 4 <= extra <= 3 * 12 * (4680 + 128) * 128 * 4 + (1 << 20)
     assert lib.arl2_launch_count(None) == 0
     assert lib.arl2_version().startswith(b"arl2")
 
