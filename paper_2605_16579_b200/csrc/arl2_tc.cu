@@ -1422,12 +1422,13 @@ tc_token_prepare_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
     }
 }
 
-// tc_token_scan_kernel: one CTA (128 threads) per (stream, head); the fp32 state lives in TMEM
+// tc_token_scan_kernel: one CTA (256 threads) per (stream, head); the fp32 state lives in TMEM
 // (row = key dim d, 128 columns) for the whole walk.  Per chunk:
 //   Y = W_c S            MMA, A = W tile (128 rows fetched, the first 64 are the chunk), B = bf16 copy of S
-//   U = U1_c - Y         threads 0-63 (one per token), written as a bf16 operand tile
+//   U = U1_c - Y         two threads per token (64 columns each), written as a bf16 operand tile
 //   S += Khat_c^T U      MMA over the chunk's 64 tokens, accumulating on g_c S (scaled beforehand)
-//   bf16 copy of the new S for the next chunk; S scaled by g_{c+1} in the same pass
+//   bf16 copy of the new S for the next chunk; S scaled by g_{c+1} in the same pass (two threads
+//                        per state row, 64 columns each)
 // The tiles of chunk c + 2 are fetched by TMA as soon as chunk c has released its buffers.
 constexpr int kTSOffS = 0;                           // bf16 S, [d][e], 128 rows
 constexpr int kTSOffW = kTileBytes;                  // 2 x 32 KB: W tiles (128 rows)
@@ -1441,7 +1442,8 @@ constexpr uint32_t kChunkTx = kTileBytes + 4 * kChunkHalf;   // W tile + Khat + 
 
 enum TSBar : int { kTSBarS0 = 0, kTSBarFull0, kTSBarFull1, kTSBarY, kTSBarS2, kTSNumBars };
 
-__global__ void __launch_bounds__(128, 1)
+constexpr int kTSThreads = 256;
+__global__ void __launch_bounds__(kTSThreads, 1)
 tc_token_scan_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_kh,
                      const __grid_constant__ CUtensorMap tm_u1, const __grid_constant__ CUtensorMap tm_s,
                      const TcTokenParams p)
@@ -1476,7 +1478,10 @@ tc_token_scan_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+    // warps w and w + 4 own the same 32 TMEM lanes (rows) and split the 128 columns in two
+    const int rowid = (warp & 3) * 32 + (tid & 31);
+    const int chalf = warp >> 2;
+    const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(chalf * 64);
 
     int loads_issued = 0;
     auto load_chunk = [&](int c) {
@@ -1499,12 +1504,13 @@ tc_token_scan_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
         if (nchunk > 1) load_chunk(1);
     }
 
-    // fp32 state row d = tid into TMEM columns 128-255, already scaled by the first chunk's decay
-    float* srow = p.state + (bh * kTile + tid) * kTile;
+    // fp32 state row d = rowid (this thread's 64 columns) into TMEM columns 128-255, already scaled
+    // by the first chunk's decay
+    float* srow = p.state + (bh * kTile + rowid) * kTile + chalf * 64;
     {
         const float g0 = __ldg(gc);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 2; ++c) {
             uint32_t x[32];
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
@@ -1559,29 +1565,26 @@ tc_token_scan_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
         if (alive) alive = wait_bar(bars + 8 * (kTSBarFull0 + s), par, ab, 103);
         tc_fence_after();
         // ---- U = U1_c - Y for the chunk's 64 tokens (threads 0-63), as a bf16 operand tile
-        if (alive && tid < kTokC) {
-            const uint8_t* u1t = smem + kTSOffU1 + s * kHalfBytes;
-            uint8_t* ut = smem + kTSOffU;
+        if (alive && rowid < kTokC) {
+            const uint8_t* u1t = smem + kTSOffU1 + s * kHalfBytes + chalf * kChunkHalf;
+            uint8_t* ut = smem + kTSOffU + chalf * kChunkHalf;
+            uint32_t y[64];
+            tmem_ld32(lane_base, *reinterpret_cast<uint32_t(*)[32]>(&y[0]));
+            tmem_ld32(lane_base + 32, *reinterpret_cast<uint32_t(*)[32]>(&y[32]));
+            tmem_wait_ld();
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-                uint32_t y[32];
-                tmem_ld32(lane_base + cc * 32, y);
-                tmem_wait_ld();
+            for (int q = 0; q < 8; ++q) {   // 16-byte chunk of this thread's 64-column half
+                const int off = rowid * 128 + ((q ^ (rowid & 7)) << 4);
+                const uint4 u1 = *reinterpret_cast<const uint4*>(u1t + off);
+                const uint32_t uw[4] = {u1.x, u1.y, u1.z, u1.w};
+                uint32_t o[4];
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    const int q = cc * 4 + q4;   // 16-byte chunk of the row: columns 8q .. 8q+7
-                    const int off = (q >> 3) * kChunkHalf + tid * 128 + (((q & 7) ^ (tid & 7)) << 4);
-                    const uint4 u1 = *reinterpret_cast<const uint4*>(u1t + off);
-                    const uint32_t uw[4] = {u1.x, u1.y, u1.z, u1.w};
-                    uint32_t o[4];
-#pragma unroll
-                    for (int m = 0; m < 4; ++m) {
-                        const float lo = __uint_as_float(uw[m] << 16) - __uint_as_float(y[q4 * 8 + 2 * m]);
-                        const float hi = __uint_as_float(uw[m] & 0xFFFF0000u) - __uint_as_float(y[q4 * 8 + 2 * m + 1]);
-                        o[m] = pack_bf16(lo, hi);
-                    }
-                    *reinterpret_cast<uint4*>(ut + off) = make_uint4(o[0], o[1], o[2], o[3]);
+                for (int m = 0; m < 4; ++m) {
+                    const float lo = __uint_as_float(uw[m] << 16) - __uint_as_float(y[q * 8 + 2 * m]);
+                    const float hi = __uint_as_float(uw[m] & 0xFFFF0000u) - __uint_as_float(y[q * 8 + 2 * m + 1]);
+                    o[m] = pack_bf16(lo, hi);
                 }
+                *reinterpret_cast<uint4*>(ut + off) = make_uint4(o[0], o[1], o[2], o[3]);
             }
         }
         fence_proxy_async_smem();
@@ -1604,38 +1607,36 @@ tc_token_scan_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
         // ---- the new S: bf16 operand copy, and the fp32 rows scaled for the next chunk (or stored)
         const bool last = c + 1 == nchunk;
         const float gn = last ? 1.0f : __ldg(gc + c + 1);
-#pragma unroll
-        for (int cc = 0; cc < 4 && alive; ++cc) {
-            uint32_t x[32];
-            tmem_ld32(lane_base + kTile + cc * 32, x);
+        if (alive) {
+            uint32_t x[64];
+            tmem_ld32(lane_base + kTile, *reinterpret_cast<uint32_t(*)[32]>(&x[0]));
+            tmem_ld32(lane_base + kTile + 32, *reinterpret_cast<uint32_t(*)[32]>(&x[32]));
             tmem_wait_ld();
             if (!last) {
+                uint8_t* sb = smem + kTSOffS + chalf * kHalfBytes + rowid * 128;
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    const int q = cc * 4 + q4;
-                    const int off = (q >> 3) * kHalfBytes + tid * 128 + (((q & 7) ^ (tid & 7)) << 4);
-                    *reinterpret_cast<uint4*>(smem + kTSOffS + off) =
-                        make_uint4(pack_bf16(__uint_as_float(x[q4 * 8 + 0]), __uint_as_float(x[q4 * 8 + 1])),
-                                   pack_bf16(__uint_as_float(x[q4 * 8 + 2]), __uint_as_float(x[q4 * 8 + 3])),
-                                   pack_bf16(__uint_as_float(x[q4 * 8 + 4]), __uint_as_float(x[q4 * 8 + 5])),
-                                   pack_bf16(__uint_as_float(x[q4 * 8 + 6]), __uint_as_float(x[q4 * 8 + 7])));
-                }
+                for (int q = 0; q < 8; ++q)
+                    *reinterpret_cast<uint4*>(sb + ((q ^ (rowid & 7)) << 4)) =
+                        make_uint4(pack_bf16(__uint_as_float(x[q * 8 + 0]), __uint_as_float(x[q * 8 + 1])),
+                                   pack_bf16(__uint_as_float(x[q * 8 + 2]), __uint_as_float(x[q * 8 + 3])),
+                                   pack_bf16(__uint_as_float(x[q * 8 + 4]), __uint_as_float(x[q * 8 + 5])),
+                                   pack_bf16(__uint_as_float(x[q * 8 + 6]), __uint_as_float(x[q * 8 + 7])));
 #pragma unroll
-                for (int e = 0; e < 32; ++e) x[e] = __float_as_uint(__uint_as_float(x[e]) * gn);
-                tmem_st32(lane_base + kTile + cc * 32, x);
+                for (int e = 0; e < 64; ++e) x[e] = __float_as_uint(__uint_as_float(x[e]) * gn);
+                tmem_st32(lane_base + kTile, *reinterpret_cast<uint32_t(*)[32]>(&x[0]));
+                tmem_st32(lane_base + kTile + 32, *reinterpret_cast<uint32_t(*)[32]>(&x[32]));
             } else {
-                __nv_bfloat16* mrow = p.state_bf16 + (bh * kTile + tid) * kTile;
+                __nv_bfloat16* mrow = p.state_bf16 + (bh * kTile + rowid) * kTile + chalf * 64;
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    *reinterpret_cast<uint4*>(srow + cc * 32 + e * 4) = make_uint4(x[e * 4], x[e * 4 + 1], x[e * 4 + 2], x[e * 4 + 3]);
-                }
+                for (int e = 0; e < 16; ++e)
+                    *reinterpret_cast<uint4*>(srow + e * 4) = make_uint4(x[e * 4], x[e * 4 + 1], x[e * 4 + 2], x[e * 4 + 3]);
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4)
-                    *reinterpret_cast<uint4*>(mrow + cc * 32 + q4 * 8) =
-                        make_uint4(pack_bf16(__uint_as_float(x[q4 * 8 + 0]), __uint_as_float(x[q4 * 8 + 1])),
-                                   pack_bf16(__uint_as_float(x[q4 * 8 + 2]), __uint_as_float(x[q4 * 8 + 3])),
-                                   pack_bf16(__uint_as_float(x[q4 * 8 + 4]), __uint_as_float(x[q4 * 8 + 5])),
-                                   pack_bf16(__uint_as_float(x[q4 * 8 + 6]), __uint_as_float(x[q4 * 8 + 7])));
+                for (int q = 0; q < 8; ++q)
+                    *reinterpret_cast<uint4*>(mrow + q * 8) =
+                        make_uint4(pack_bf16(__uint_as_float(x[q * 8 + 0]), __uint_as_float(x[q * 8 + 1])),
+                                   pack_bf16(__uint_as_float(x[q * 8 + 2]), __uint_as_float(x[q * 8 + 3])),
+                                   pack_bf16(__uint_as_float(x[q * 8 + 4]), __uint_as_float(x[q * 8 + 5])),
+                                   pack_bf16(__uint_as_float(x[q * 8 + 6]), __uint_as_float(x[q * 8 + 7])));
             }
         }
         tmem_wait_st();
@@ -1900,7 +1901,7 @@ int tc_commit_tokens(const TokenCommitArgs& a, const __nv_bfloat16* wk_op, const
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_error("launch of tc_token_prepare_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
     dim3 grid2(a.s.H, a.s.B);
-    tc_token_scan_kernel<<<grid2, 128, kTSSmemBytes, st>>>(tm_w, tm_kh, tm_u1, tm_s, p);
+    tc_token_scan_kernel<<<grid2, kTSThreads, kTSSmemBytes, st>>>(tm_w, tm_kh, tm_u1, tm_s, p);
     e = cudaGetLastError();
     if (e != cudaSuccess) { set_error("launch of tc_token_scan_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
     return 2;
