@@ -391,6 +391,27 @@ def run_ours(args):
     tok.sync_status()
     del tok
 
+    # the teacher's layer on the same kernels (Eq. 1 over a key/value cache that grows by one block
+    # per generated block) against the horizon: its cost per denoise pass grows, the layer's does not
+    teacher = None
+    if layer.step_kernel == "tcgen05" and not args.no_teacher:
+        teacher = {"cache_blocks": [], "ms_per_pass": []}
+        q0, k0, v0, _ = dev_sets[0]
+        for nb in (1, 2, 4, 8, 16):
+            kcache, vcache = k0.repeat(1, nb, 1, 1), v0.repeat(1, nb, 1, 1)
+            ts = []
+            for it in range(5):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                layer.set_profile_events(e0, e1)
+                layer.teacher_step(q0, kcache, vcache, out=out)
+                torch.cuda.synchronize()
+                if it >= 2:
+                    ts.append(e0.elapsed_time(e1))
+            teacher["cache_blocks"].append(nb)
+            teacher["ms_per_pass"].append(statistics.mean(ts))
+            del kcache, vcache
+        layer.sync_status()
+
     ms_total, ms_e2e, kern_mean = max_over_ranks([ms_total, ms_e2e, statistics.mean(kern_ms)], world, dev)
 
     if rank == 0:
@@ -441,6 +462,7 @@ def run_ours(args):
             "clocks": clocks,
             "horizon": horizon_report(block_ms, mem_marks, layer.workspace_bytes + layer.state.numel() * 4),
             "commit_ms": commit_ms,
+            "teacher_horizon": teacher,
         }
         if world == 1 and not args.no_cpu_baseline:
             s = CpuSample(cfg)
@@ -471,6 +493,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="long", choices=["tiny", "small", "chunked", "batched", "long"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-teacher", action="store_true", help="skip the teacher-attention horizon leg")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

@@ -115,6 +115,20 @@ int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const voi
                       const float* d_gate_logits, void* d_out, void* stream);
 
 /*
+ * The teacher's layer for comparison (Eq. 1): plain softmax attention of the current block's L
+ * queries over a key/value cache of `cache_tokens` tokens (the blocks generated so far plus the
+ * current one), all visible to every query:
+ *   d_out[b,i,h,:] = softmax_j(<q_i, k_j> scale) v_j,   j = 0 .. cache_tokens-1.
+ * d_q, d_out: [B, L, H, D]; d_k_cache, d_v_cache: [B, cache_tokens, H, D], io_dtype.  No rotation
+ * is applied (a cache holds rotated keys; pass rotated queries), the feature maps, the gate and
+ * the recurrent state play no part.  Its cost grows with cache_tokens where arl2_denoise_step's
+ * does not: this entry point exists to measure that on the same kernels.  Contexts with bf16 I/O
+ * and D = 128 only (ARL2_ERR_UNSUPPORTED otherwise).  Honours arl2_set_profile_events.
+ */
+int arl2_teacher_step(arl2_ctx* ctx, const void* d_q, const void* d_k_cache, const void* d_v_cache,
+                      int32_t cache_tokens, void* d_out, void* stream);
+
+/*
  * State commit, once per block, from the clean pass's K and V (Algorithm 1, clean-pass
  * branch; Eq. 4 in its gated-linear form):
  *   S[b,h] <- sigmoid(a[b,h]) S[b,h] + sum_l K'_l^T V'_l,

@@ -208,6 +208,46 @@ void arl2_oracle_step_rows(int B, int H, int L, int D,
 }
 
 /*
+ * Eq. 1: the teacher's softmax attention of L queries over a key/value cache of Lk tokens,
+ * every cached token visible to every query (the cache holds the blocks so far and the current
+ * one).  q, out: [B, L, H, D]; k, v: [B, Lk, H, D].  No rotation, no state.
+ *   out_i = sum_j softmax_j(<q_i, k_j> scale) v_j
+ */
+void arl2_oracle_attend_cache(int B, int H, int L, int Lk, int D,
+                              const double *q, const double *k, const double *v,
+                              double scale, double *out)
+{
+#pragma omp parallel
+    {
+        double *w = (double *)malloc(sizeof(double) * (size_t)Lk);
+#pragma omp for collapse(2) schedule(dynamic, 8)
+        for (int bh = 0; bh < B * H; ++bh)
+            for (int i = 0; i < L; ++i) {
+                int b = bh / H, h = bh % H;
+                const double *qi = q + (((size_t)b * L + i) * H + h) * D;
+                double mx = -INFINITY;
+                for (int j = 0; j < Lk; ++j) {
+                    const double *kj = k + (((size_t)b * Lk + j) * H + h) * D;
+                    double sc = 0.0;
+                    for (int d = 0; d < D; ++d) sc += qi[d] * kj[d];
+                    w[j] = sc * scale;
+                    if (w[j] > mx) mx = w[j];
+                }
+                double sum = 0.0;
+                for (int j = 0; j < Lk; ++j) { w[j] = exp(w[j] - mx); sum += w[j]; }
+                double *o = out + (((size_t)b * L + i) * H + h) * D;
+                for (int e = 0; e < D; ++e) o[e] = 0.0;
+                for (int j = 0; j < Lk; ++j) {
+                    const double *vj = v + (((size_t)b * Lk + j) * H + h) * D;
+                    double pj = w[j] / sum;
+                    for (int e = 0; e < D; ++e) o[e] += pj * vj[e];
+                }
+            }
+        free(w);
+    }
+}
+
+/*
  * State commit for one (b, h), run once per block from the clean pass's K, V
  * (Algorithm 1, clean-pass branch).  K' = L2Norm(RoPE(phi_k(K))), V' = phi_v(V).
  *

@@ -119,6 +119,19 @@ def step_rows(q, k, v, g, S, rows, wq=None, rope_cos=None, rope_sin=None, scale=
     return out
 
 
+def attend_cache(q, k_cache, v_cache, scale=None):
+    """Eq. 1: softmax attention of q [B, L, H, D] over a cache [B, Lk, H, D]; scale None = 1/sqrt(D)."""
+    q, k_cache, v_cache = _f64(q), _f64(k_cache), _f64(v_cache)
+    B, L, H, D = q.shape
+    Lk = k_cache.shape[1]
+    assert k_cache.shape == (B, Lk, H, D) and v_cache.shape == (B, Lk, H, D)
+    out = np.empty((B, L, H, D), dtype=np.float64)
+    sc = (1.0 / np.sqrt(D)) if scale is None else float(scale)
+    _load().arl2_oracle_attend_cache(B, H, L, Lk, D, _p(q), _p(k_cache), _p(v_cache),
+                                     ctypes.c_double(sc), _p(out))
+    return out
+
+
 def commit(kc, vc, a, S, wk=None, wv=None, rope_cos=None, rope_sin=None, eps=1e-6, rule=0,
            beta_logit=None, heads=None):
     """State commit, once per block.  Returns the new S (the argument is not modified).

@@ -22,7 +22,7 @@ ARL2_FLAG_TOKEN_GATES = 2
 EXPORTS = (
     "arl2_workspace_bytes", "arl2_create", "arl2_set_params", "arl2_denoise_step", "arl2_commit",
     "arl2_reset", "arl2_get_state", "arl2_set_state", "arl2_sync_status", "arl2_launch_count",
-    "arl2_set_profile_events", "arl2_commit_static_scratch", "arl2_commit_delta", "arl2_commit_tokens",
+    "arl2_set_profile_events", "arl2_commit_static_scratch", "arl2_commit_delta", "arl2_commit_tokens", "arl2_teacher_step",
     "arl2_step_kernel_name", "arl2_destroy", "arl2_last_error", "arl2_version",
 )
 
@@ -70,6 +70,8 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     lib.arl2_denoise_step.argtypes = [vp] * 7
     lib.arl2_commit.restype = ctypes.c_int
     lib.arl2_commit.argtypes = [vp] * 5
+    lib.arl2_teacher_step.restype = ctypes.c_int
+    lib.arl2_teacher_step.argtypes = [vp, vp, vp, vp, ctypes.c_int32, vp, vp]
     lib.arl2_commit_delta.restype = ctypes.c_int
     lib.arl2_commit_delta.argtypes = [vp] * 6
     lib.arl2_commit_tokens.restype = ctypes.c_int
@@ -178,6 +180,22 @@ class Layer:
         with torch.cuda.device(self.device):
             _check(load().arl2_denoise_step(self._ctx, _ptr(q), _ptr(k), _ptr(v), _ptr(gate_logits),
                                             _ptr(out), _stream()), "arl2_denoise_step")
+        return out
+
+    def teacher_step(self, q, k_cache, v_cache, out=None):
+        """Eq. 1: softmax attention of q [B, L, H, D] over a cache [B, Lk, H, D] (no rotation, no state)."""
+        shape = (self.B, self.L, self.H, self.D)
+        self._want(q, shape, self.dtype, "q")
+        lk = int(k_cache.shape[1])
+        self._want(k_cache, (self.B, lk, self.H, self.D), self.dtype, "k_cache")
+        self._want(v_cache, (self.B, lk, self.H, self.D), self.dtype, "v_cache")
+        if out is None:
+            out = torch.empty(shape, dtype=self.dtype, device=self.device)
+        else:
+            self._want(out, shape, self.dtype, "out")
+        with torch.cuda.device(self.device):
+            _check(load().arl2_teacher_step(self._ctx, _ptr(q), _ptr(k_cache), _ptr(v_cache), lk,
+                                            _ptr(out), _stream()), "arl2_teacher_step")
         return out
 
     def commit(self, k_clean, v_clean, decay_logits):

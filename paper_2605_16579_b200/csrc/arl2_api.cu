@@ -289,6 +289,56 @@ int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const voi
     return r;
 }
 
+int arl2_teacher_step(arl2_ctx* ctx, const void* d_q, const void* d_k_cache, const void* d_v_cache,
+                      int32_t cache_tokens, void* d_out, void* stream)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    if (!d_q || !d_k_cache || !d_v_cache || !d_out) {
+        set_error("teacher_step: q, k_cache, v_cache and out must not be NULL");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    if (cache_tokens < 1) {
+        set_error("teacher_step: cache_tokens must be >= 1 (got %d)", cache_tokens);
+        return ARL2_ERR_INVALID_ARG;
+    }
+    if (d_out == d_q || d_out == d_k_cache || d_out == d_v_cache) {
+        set_error("teacher_step: out must not alias an input");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    if ((reinterpret_cast<uintptr_t>(d_q) | reinterpret_cast<uintptr_t>(d_k_cache) |
+         reinterpret_cast<uintptr_t>(d_v_cache) | reinterpret_cast<uintptr_t>(d_out)) % 16 != 0) {
+        set_error("teacher_step: q, k_cache, v_cache and out must be 16-byte aligned");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    if (!ctx->use_tc) {
+        set_error("teacher_step: built for bf16 I/O with D = 128 (the tensor-core context) only");
+        return ARL2_ERR_UNSUPPORTED;
+    }
+    if ((size_t)ctx->cfg.B * cache_tokens * ctx->cfg.H * ctx->cfg.D >= ((size_t)1 << 40)) {
+        set_error("teacher_step: cache too large");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    StepArgs a;
+    a.s = ctx->shape;
+    a.q = d_q; a.k_rot = d_k_cache; a.v = d_v_cache;
+    a.gate = nullptr;                      // closed gate: the state contributes nothing
+    a.state = ctx->state; a.wq = ctx->wq;
+    a.rope_cos = nullptr; a.rope_sin = nullptr;
+    a.out = d_out;
+    a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status);
+    a.launch_parity = (int)(ctx->step_calls++ & 1u);
+    a.rope_h = nullptr;                    // the caller's Q and cache are already rotated
+    a.Lk = cache_tokens;
+    cudaStream_t st = as_stream(stream);
+    cudaEvent_t e0 = ctx->ev_before, e1 = ctx->ev_after;
+    ctx->ev_before = ctx->ev_after = nullptr;
+    if (e0 != nullptr) cudaEventRecord(e0, st);
+    int r = account(ctx, tc_step(a, reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wq_op),
+                                 reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.state_bf16), st));
+    if (e1 != nullptr) cudaEventRecord(e1, st);
+    return r;
+}
+
 int arl2_set_profile_events(arl2_ctx* ctx, void* ev_before, void* ev_after)
 {
     if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;

@@ -41,6 +41,7 @@ struct StepArgs {
     uint32_t* status;
     int launch_parity;      // step launches so far on this context, mod 2 (scheduler counters)
     const void* rope_h;     // [L, D/2] half2 (cos, sin) copy of the tables (tensor-core path), or nullptr
+    int Lk = 0;             // > 0: K and V hold Lk tokens (a cache), [B, Lk, H, D]; 0: L
 };
 
 struct CommitArgs {

@@ -80,9 +80,11 @@ struct TcStepParams {
     uint32_t* status;
     uint32_t* sched_counter;   // this launch's item counter (zero on entry)
     uint32_t* sched_next;      // the next launch's counter: cleared by this launch
-    int n_kv;                  // key tiles per head = query tiles per head
-    int n_pair_items;          // B * H * (n_kv / 2): items with two query tiles
-    int n_items;               // + ceil(B * H / 2) items of ragged last tiles when n_kv is odd
+    int Lk;                    // keys per head: L, or the length of a key/value cache (Eq. 1)
+    int n_q;                   // query tiles per head
+    int n_kv;                  // key tiles per head
+    int n_pair_items;          // B * H * (n_q / 2): items with two query tiles
+    int n_items;               // + ceil(B * H / 2) items of ragged last tiles when n_q is odd
 };
 
 struct Abort {
@@ -204,7 +206,7 @@ struct Item {
 __device__ __forceinline__ Item decode_item(int id, const TcStepParams& p)
 {
     Item it;
-    const int full_pairs = p.n_kv >> 1;
+    const int full_pairs = p.n_q >> 1;
     const int units = p.s.B * p.s.H;
     if (id < p.n_pair_items) {
         const int bh = id / full_pairs;
@@ -353,7 +355,7 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                 tmem_wait_ld();
                 ARL2_STAMP(tr, ts + 2);
 
-                const int n_valid = L - j * kTile;  // keys of this tile that exist
+                const int n_valid = p.Lk - j * kTile;  // keys of this tile that exist
                 if (n_valid < kTile) {   // ragged last tile: zero-filled key rows must not count
 #pragma unroll
                     for (int c = 0; c < 128; ++c)
@@ -447,7 +449,8 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
             // ---- inter branch: U = Q W_phi_q arrives in the S columns                  (Eq. 3)
             // the row's rotation table is fetched while the MMA is still running
             uint4 cs[16];
-            const float gate_logit = valid_row ? __ldg(p.gate + ((size_t)b * L + row) * H + h) : 0.0f;   // fetched early too
+            // fetched early too; no gate tensor = closed gate (plain softmax attention, Eq. 1)
+            const float gate_logit = (valid_row && p.gate != nullptr) ? __ldg(p.gate + ((size_t)b * L + row) * H + h) : -INFINITY;
             const bool rotate_u = p.rope_h != nullptr && valid_row;
             if (rotate_u) {
                 const uint4* tab = p.rope_h + ((size_t)(row >> 5) * 16) * 32 + (row & 31);
@@ -1785,8 +1788,10 @@ int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* 
     }
     CUtensorMap tm_q, tm_k, tm_v, tm_w, tm_s;
     if (int r = make_map_blhd(&tm_q, a.q, a.s)) return r;
-    if (int r = make_map_blhd(&tm_k, a.k_rot, a.s)) return r;
-    if (int r = make_map_blhd(&tm_v, a.v, a.s)) return r;
+    Shape ks = a.s;
+    ks.L = a.Lk > 0 ? a.Lk : a.s.L;   // K and V may be a longer cache
+    if (int r = make_map_blhd(&tm_k, a.k_rot, ks)) return r;
+    if (int r = make_map_blhd(&tm_v, a.v, ks)) return r;
     if (int r = make_map_rows(&tm_w, wq_op, (size_t)a.s.H * kTile)) return r;
     if (int r = make_map_rows(&tm_s, state_bf16, (size_t)a.s.B * a.s.H * kTile)) return r;
     TcStepParams p;
@@ -1797,10 +1802,12 @@ int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* 
     p.rope_h = static_cast<const uint4*>(a.rope_h);
     p.out = static_cast<__nv_bfloat16*>(a.out);
     p.status = a.status;
-    p.n_kv = (a.s.L + kTile - 1) / kTile;
+    p.Lk = ks.L;
+    p.n_q = (a.s.L + kTile - 1) / kTile;
+    p.n_kv = (ks.L + kTile - 1) / kTile;
     const int bh = a.s.B * a.s.H;
-    p.n_pair_items = bh * (p.n_kv / 2);
-    p.n_items = p.n_pair_items + ((p.n_kv & 1) ? (bh + 1) / 2 : 0);   // ragged tiles go two by two
+    p.n_pair_items = bh * (p.n_q / 2);
+    p.n_items = p.n_pair_items + ((p.n_q & 1) ? (bh + 1) / 2 : 0);   // ragged tiles go two by two
     // two item counters alternate between launches: a launch consumes one and clears the other
     p.sched_counter = a.status + kStatusSched + (a.launch_parity & 1);
     p.sched_next = a.status + kStatusSched + ((a.launch_parity + 1) & 1);

@@ -344,6 +344,30 @@ def sig(x):
     return 1.0 / (1.0 + np.exp(-x))
 
 
+def test_cache_attention_against_library_and_the_layer(oracle):
+    """Eq. 1 over a longer cache: the library's attention routine; with a cache of exactly the
+    block and a closed gate it is the layer's intra branch without rotation; a cache of one token
+    returns that token's value; explicit softmax weights with a custom scale."""
+    B, L, Lk, H, D = 2, 5, 13, 2, 8
+    q, k, v = rnd(B, L, H, D), rnd(B, Lk, H, D), rnd(B, Lk, H, D)
+    got = oracle.attend_cache(q, k, v)
+    tq, tk, tv = (torch.from_numpy(t).permute(0, 2, 1, 3) for t in (q, k, v))
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv).permute(0, 2, 1, 3).numpy()
+    np.testing.assert_allclose(got, ref, rtol=1e-10, atol=1e-12)
+    same = oracle.step(q, k[:, :L], v[:, :L], np.full((B, L, H), -800.0), rnd(B, H, D, D))
+    np.testing.assert_allclose(oracle.attend_cache(q, k[:, :L], v[:, :L]), same, rtol=1e-12, atol=1e-14)
+    one = oracle.attend_cache(q, k[:, :1], v[:, :1])
+    np.testing.assert_allclose(one, np.broadcast_to(v[:, :1], one.shape), rtol=1e-12)
+    # explicit weights (einsum + exp) with an extra zero key and a custom scale
+    far = np.concatenate([k, np.zeros_like(k[:, :1])], axis=1)
+    v2 = np.concatenate([v, 1e3 * np.ones_like(v[:, :1])], axis=1)
+    big = oracle.attend_cache(q, far, v2, scale=1.0)
+    sc = np.einsum("blhd,bjhd->bhlj", q, far)
+    w = np.exp(sc - sc.max(-1, keepdims=True))
+    w /= w.sum(-1, keepdims=True)
+    np.testing.assert_allclose(big, np.einsum("bhlj,bjhe->blhe", w, v2), rtol=1e-10, atol=1e-10)
+
+
 def test_token_gates_matrix_product_form(oracle):
     """Per-token Eq. 4 rewritten as S_j = (alpha_j I - beta_j k_j^T k_j) S_{j-1} + beta_j k_j^T v_j
     and evaluated with explicit D x D transition matrices (library matmul), with feature maps,
