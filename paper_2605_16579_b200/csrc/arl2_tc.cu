@@ -38,6 +38,10 @@ constexpr int kStages = 5;
 constexpr int kThreads = 384;              // 3 warpgroups: softmax 0, softmax 1, {TMA, MMA, 2 idle}
 constexpr int kRegsSoftmax = 232;          // per-thread registers after the warpgroups rebalance
 constexpr int kRegsOther = 40;
+// setmaxnreg.inc waits (without a bound) for registers of the CTA's own launch allocation
+// (threads x the launch register count): the rebalanced total must fit in it
+constexpr int kLaunchRegs = (65536 / kThreads) / 8 * 8;
+static_assert(256 * kRegsSoftmax + (kThreads - 256) * kRegsOther <= kThreads * kLaunchRegs, "register pool");
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units of slack before O is rescaled
 #ifndef ARL2_POLY_COUNT
