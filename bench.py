@@ -63,6 +63,16 @@ def step_bytes(cfg):
     return cfg.B * cfg.H * (4.0 * cfg.L * cfg.D * e + 4.0 * cfg.L + cfg.D * cfg.D * (4 + e))
 
 
+def sfu_bound(cfg, kern_ms, sm_mhz, per_clk_per_sm=16, sms=148):
+    """Exponentials of one denoise pass against the special-function unit's rate."""
+    n_exp = float(cfg.B * cfg.H) * cfg.L * cfg.L
+    if not sm_mhz:
+        return {"exp_per_launch": n_exp, "min_ms": None, "frac": None}
+    min_ms = n_exp / (per_clk_per_sm * sms * sm_mhz * 1e6) * 1e3
+    return {"exp_per_launch": n_exp, "min_ms": min_ms, "frac": min_ms / kern_ms,
+            "rate": f"{per_clk_per_sm}/clk/SM x {sms} SMs at {sm_mhz:.0f} MHz"}
+
+
 class ClockSampler:
     """nvidia-smi in the background during the timed region (read-only queries)."""
 
@@ -454,6 +464,9 @@ def run_ours(args):
                 "algorithmic_flops_per_launch": step_flops(cfg),
                 "algorithmic_bytes_per_launch": step_bytes(cfg),
                 "hbm_frac": step_bytes(cfg) / (kern_mean * 1e-3) / 1e9 / pk["hbm_gbs"],
+                # secondary bound: one exponential per score element on the special-function unit
+                # (16 per clock per SM, 148 SMs, at the SM clock sampled during the run)
+                "sfu": sfu_bound(cfg, kern_mean, (clocks or {}).get("sm_mhz")),
             },
             "e2e": {"value": world * cfg.B * cfg.L * cfg.steps * e2e_blocks / (ms_e2e * 1e-3),
                     "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
