@@ -371,8 +371,10 @@ def run_ours(args):
     # the block uses, and the delta rule of Eq. 4 at block level
     beta = workload.beta_logits(cfg, commit_block).to(dev)
     commit_ms = {}
+    alpha_tok = workload.token_gate_logits(cfg, commit_block)[0].to(dev)
     for name, call in (("gated_linear", lambda: layer.commit(*dev_commit)),
-                       ("delta", lambda: layer.commit_delta(*dev_commit, beta))):
+                       ("delta", lambda: layer.commit_delta(*dev_commit, beta)),
+                       ("decay_tokens", lambda: layer.commit_decay_tokens(dev_commit[0], dev_commit[1], alpha_tok))):
         layer.reset()
         for _ in range(3):
             call()

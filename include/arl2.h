@@ -154,6 +154,17 @@ int arl2_commit_delta(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clea
                       const float* d_decay_logits, const float* d_beta_logits, void* stream);
 
 /*
+ * The gated-linear commit with one forget gate per token (the gate granularity the paper states;
+ * Eq. 4 without its correction term, token by token): for l = 0..L-1
+ *   S[b,h] <- alpha_l S[b,h] + K'_l^T V'_l,   alpha_l = sigmoid(d_alpha_logits[b,l,h]),
+ * computed in closed form as (prod_l alpha_l) S + sum_l (prod_{i>l} alpha_i) K'_l^T V'_l: a small
+ * kernel forms the suffix products, then arl2_commit's kernels run with weighted value rows.
+ * d_alpha_logits: [B, L, H] fp32.  Other arguments, reproducibility and errors as arl2_commit.
+ */
+int arl2_commit_decay_tokens(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
+                             const float* d_alpha_logits, void* stream);
+
+/*
  * State commit with Eq. 4 applied token by token, in order, with per-token gates (the sentence
  * after Eq. 4): for l = 0..L-1
  *   S[b,h] <- alpha_l S[b,h] + beta_l K'_l^T (V'_l - K'_l S[b,h]),

@@ -386,6 +386,40 @@ void arl2_oracle_commit_tokens(int B, int H, int L, int D,
     }
 }
 
+/*
+ * The gated-linear update (Eq. 4 without the correction term) with the per-token forget gates
+ * the paper states, token by token:  for j = 0..L-1:  S <- alpha_j S + K'_j^T V'_j,
+ * alpha_j = sigmoid(alpha_logit[b,j,h]).
+ */
+void arl2_oracle_commit_decay_tokens(int B, int H, int L, int D,
+                                     const double *kc, const double *vc, const double *alpha_logit,
+                                     const double *wk, const double *wv,
+                                     const double *rope_cos, const double *rope_sin, double eps,
+                                     int n_heads, const int *bs, const int *hs, double *S)
+{
+    int total = bs ? n_heads : B * H;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int t = 0; t < total; ++t) {
+        int b = bs ? bs[t] : t / H;
+        int h = bs ? hs[t] : t % H;
+        double *Sh = S + ((size_t)b * H + h) * D * D;
+        double *kf = (double *)malloc(sizeof(double) * D);
+        double *vf = (double *)malloc(sizeof(double) * D);
+        for (int j = 0; j < L; ++j) {
+            size_t off = (((size_t)b * L + j) * H + h) * D;
+            phi(kc + off, wk, h, D, kf);
+            rope(kf, D, rope_cos, rope_sin, j);
+            l2norm(kf, D, eps);
+            phi(vc + off, wv, h, D, vf);
+            double alpha = sigmoid(alpha_logit[((size_t)b * L + j) * H + h]);
+            for (int d = 0; d < D; ++d)
+                for (int e = 0; e < D; ++e)
+                    Sh[(size_t)d * D + e] = alpha * Sh[(size_t)d * D + e] + kf[d] * vf[e];
+        }
+        free(vf); free(kf);
+    }
+}
+
 /* S <- 0 for stream `stream` (or all streams when stream < 0): Algorithm 1, first line. */
 void arl2_oracle_reset(int B, int H, int D, int stream, double *S)
 {

@@ -183,6 +183,28 @@ def commit_tokens(kc, vc, S, alpha_logit=None, beta_logit=None, wk=None, wv=None
     return S
 
 
+def commit_decay_tokens(kc, vc, S, alpha_logit, wk=None, wv=None, rope_cos=None, rope_sin=None,
+                        eps=1e-6, heads=None):
+    """Gated-linear update with per-token forget gates [B, L, H], token by token.  Returns the new S."""
+    kc, vc, alpha_logit = _f64(kc), _f64(vc), _f64(alpha_logit)
+    wk, wv, rope_cos, rope_sin = _f64(wk), _f64(wv), _f64(rope_cos), _f64(rope_sin)
+    S = _f64(S).copy()
+    B, L, H, D = kc.shape
+    assert S.shape == (B, H, D, D) and alpha_logit.shape == (B, L, H)
+    if heads is None:
+        n, bs, hs = 0, None, None
+    else:
+        heads = np.asarray(heads, dtype=np.int32).reshape(-1, 2)
+        n = heads.shape[0]
+        bs = np.ascontiguousarray(heads[:, 0])
+        hs = np.ascontiguousarray(heads[:, 1])
+    _load().arl2_oracle_commit_decay_tokens(
+        B, H, L, D, _p(kc), _p(vc), _p(alpha_logit), _p(wk), _p(wv), _p(rope_cos), _p(rope_sin),
+        ctypes.c_double(eps), n, _p(bs), _p(hs), _p(S),
+    )
+    return S
+
+
 def reset(S, stream: int = -1):
     """S <- 0 for one stream or all (stream < 0).  Returns a new array."""
     S = _f64(S).copy()

@@ -22,7 +22,7 @@ ARL2_FLAG_TOKEN_GATES = 2
 EXPORTS = (
     "arl2_workspace_bytes", "arl2_create", "arl2_set_params", "arl2_denoise_step", "arl2_commit",
     "arl2_reset", "arl2_get_state", "arl2_set_state", "arl2_sync_status", "arl2_launch_count",
-    "arl2_set_profile_events", "arl2_commit_static_scratch", "arl2_commit_delta", "arl2_commit_tokens", "arl2_teacher_step",
+    "arl2_set_profile_events", "arl2_commit_static_scratch", "arl2_commit_delta", "arl2_commit_tokens", "arl2_teacher_step", "arl2_commit_decay_tokens",
     "arl2_step_kernel_name", "arl2_destroy", "arl2_last_error", "arl2_version",
 )
 
@@ -74,6 +74,8 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     lib.arl2_teacher_step.argtypes = [vp, vp, vp, vp, ctypes.c_int32, vp, vp]
     lib.arl2_commit_delta.restype = ctypes.c_int
     lib.arl2_commit_delta.argtypes = [vp] * 6
+    lib.arl2_commit_decay_tokens.restype = ctypes.c_int
+    lib.arl2_commit_decay_tokens.argtypes = [vp] * 5
     lib.arl2_commit_tokens.restype = ctypes.c_int
     lib.arl2_commit_tokens.argtypes = [vp] * 6
     lib.arl2_reset.restype = ctypes.c_int
@@ -218,6 +220,16 @@ class Layer:
         with torch.cuda.device(self.device):
             _check(load().arl2_commit_delta(self._ctx, _ptr(k_clean), _ptr(v_clean), _ptr(decay_logits),
                                             _ptr(beta_logits), _stream()), "arl2_commit_delta")
+
+    def commit_decay_tokens(self, k_clean, v_clean, alpha_logits):
+        """Gated-linear commit with one forget gate per token: S <- alpha_l S + K'_l^T V'_l in order."""
+        shape = (self.B, self.L, self.H, self.D)
+        self._want(k_clean, shape, self.dtype, "k_clean")
+        self._want(v_clean, shape, self.dtype, "v_clean")
+        self._want(alpha_logits, (self.B, self.L, self.H), torch.float32, "alpha_logits")
+        with torch.cuda.device(self.device):
+            _check(load().arl2_commit_decay_tokens(self._ctx, _ptr(k_clean), _ptr(v_clean),
+                                                   _ptr(alpha_logits), _stream()), "arl2_commit_decay_tokens")
 
     def commit_tokens(self, k_clean, v_clean, alpha_logits=None, beta_logits=None):
         """Eq. 4 token by token with per-token gates [B, L, H] (None = gate 1); the layer must have

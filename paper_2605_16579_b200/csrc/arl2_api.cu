@@ -27,7 +27,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, k_rot, partials, state_bf16, wq_op, wk_op, wv_op, rope_h, tok_w, tok_u1, tok_kh, tok_gc, total;
+    size_t status, k_rot, partials, state_bf16, wq_op, wk_op, wv_op, rope_h, dec_w, dec_total, tok_w, tok_u1, tok_kh, tok_gc, total;
     int nsplit, nchunk;
 };
 
@@ -84,6 +84,9 @@ Layout make_layout(const arl2_config& c)
     l.wk_op = off;      off += align_up((size_t)c.H * dd * 2);
     l.wv_op = off;      off += align_up((size_t)c.H * dd * 2);
     l.rope_h = off;     off += align_up((size_t)((c.L + 127) / 128) * 128 * (c.D / 2) * 4);
+    // per-token decay weights of arl2_commit_decay_tokens (small)
+    l.dec_w = off;      off += align_up((size_t)c.B * c.L * c.H * sizeof(float));
+    l.dec_total = off;  off += align_up((size_t)c.B * c.H * sizeof(float));
     // scratch of arl2_commit_tokens, only when the context asks for it
     l.nchunk = (c.L + kTokenChunk - 1) / kTokenChunk;
     l.tok_w = l.tok_u1 = l.tok_kh = l.tok_gc = 0;
@@ -351,7 +354,7 @@ namespace {
 
 // Shared by arl2_commit (delta = false) and arl2_commit_delta.
 int commit_impl(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
-                const float* d_decay_logits, bool delta, const float* d_beta_logits, void* stream)
+                const float* d_decay_logits, int mode, const float* d_beta, bool decay_direct, void* stream)
 {
     if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
     if (!d_k_clean || !d_v_clean || !d_decay_logits) {
@@ -370,8 +373,9 @@ int commit_impl(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
     a.nsplit = ctx->lay.nsplit;
     a.rope_h = (ctx->use_tc && ctx->rope_cos != nullptr) ? ctx->ws + ctx->lay.rope_h : nullptr;
     a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status);
-    a.delta = delta;
-    a.beta = d_beta_logits;
+    a.mode = mode;
+    a.beta = d_beta;
+    a.decay_direct = decay_direct;
     if ((reinterpret_cast<uintptr_t>(d_k_clean) | reinterpret_cast<uintptr_t>(d_v_clean)) % 16 != 0) {
         set_error("commit: k_clean and v_clean must be 16-byte aligned");
         return ARL2_ERR_INVALID_ARG;
@@ -388,7 +392,7 @@ int commit_impl(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
 int arl2_commit(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
                 const float* d_decay_logits, void* stream)
 {
-    return commit_impl(ctx, d_k_clean, d_v_clean, d_decay_logits, false, nullptr, stream);
+    return commit_impl(ctx, d_k_clean, d_v_clean, d_decay_logits, 0, nullptr, false, stream);
 }
 
 int arl2_commit_tokens(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
@@ -434,7 +438,22 @@ int arl2_commit_tokens(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_cle
 int arl2_commit_delta(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
                       const float* d_decay_logits, const float* d_beta_logits, void* stream)
 {
-    return commit_impl(ctx, d_k_clean, d_v_clean, d_decay_logits, true, d_beta_logits, stream);
+    return commit_impl(ctx, d_k_clean, d_v_clean, d_decay_logits, 1, d_beta_logits, false, stream);
+}
+
+int arl2_commit_decay_tokens(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
+                             const float* d_alpha_logits, void* stream)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    if (!d_alpha_logits) {
+        set_error("commit_decay_tokens: alpha_logits must not be NULL");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    float* w = reinterpret_cast<float*>(ctx->ws + ctx->lay.dec_w);
+    float* total = reinterpret_cast<float*>(ctx->ws + ctx->lay.dec_total);
+    int r = account(ctx, decay_weights(ctx->shape, d_alpha_logits, w, total, as_stream(stream)));
+    if (r != ARL2_OK) return r;
+    return commit_impl(ctx, d_k_clean, d_v_clean, total, 2, w, true, stream);
 }
 
 int arl2_reset(arl2_ctx* ctx, int32_t stream_index, void* stream)

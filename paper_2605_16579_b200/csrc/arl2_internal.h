@@ -59,8 +59,11 @@ struct CommitArgs {
     int nsplit;
     const void* rope_h;     // half2 (cos, sin) copy of the tables (tensor-core path), or nullptr
     uint32_t* status;
-    bool delta = false;     // Eq. 4 as printed: value operand diag(beta) (V' - K' S_old)
-    const float* beta = nullptr;   // [B, L, H] learning-rate logits, or nullptr = 1 (delta only)
+    // 0: value rows V'; 1: Eq. 4 as printed, diag(sigmoid(beta)) (V' - K' S_old); 2: diag(beta) V'
+    // with beta given directly (per-token decay weights)
+    int mode = 0;
+    const float* beta = nullptr;   // [B, L, H]: logits (mode 1) or weights (mode 2); nullptr = 1
+    bool decay_direct = false;     // `decay` holds the factors themselves, not logits
 };
 
 // Eq. 4 token by token with per-token gates (chunkwise form): the two launches share these.
@@ -91,6 +94,8 @@ int simt_rope_k(const Shape& s, int dtype, const void* k, const float* cos_t, co
 int simt_step(const StepArgs& a, int dtype, cudaStream_t st);
 int simt_commit(const CommitArgs& a, int dtype, cudaStream_t st);
 int commit_reduce(const CommitArgs& a, cudaStream_t st);  // fixed-order sum + gated decay
+// w[b,l,h] = prod_{i>l} sigmoid(alpha[b,i,h]), total[b,h] = prod_l sigmoid(alpha[b,l,h])
+int decay_weights(const Shape& s, const float* alpha_logits, float* w, float* total, cudaStream_t st);
 int simt_commit_tokens(const TokenCommitArgs& a, int dtype, cudaStream_t st);
 int fill_zero(void* p, size_t bytes, cudaStream_t st);
 int state_to_bf16(const float* state, __nv_bfloat16* dst, size_t n, cudaStream_t st);

@@ -360,7 +360,24 @@ __global__ void __launch_bounds__(NT) simt_commit_partial_kernel(CommitArgs a)
         __syncthreads();
         feature_tile<D, T>(Ks, Ws, wk, r0, lim, a.rope_cos, a.rope_sin, a.s.eps, true, tx, ty, tid);
         feature_tile<D, T>(Vs2, Ws, wv, r0, lim, nullptr, nullptr, a.s.eps, false, tx, ty, tid);
-        if (a.delta) {
+        if (a.mode == 2) {
+            // per-token decay weights: the value rows are scaled by w_l = prod_{i>l} alpha_i
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int row = r0 + ty * 4 + i;
+                const float wgt = (a.beta != nullptr && row < lim) ? a.beta[((size_t)b * L + row) * H + h]
+                                                                   : (row < lim ? 1.0f : 0.0f);
+#pragma unroll
+                for (int c = 0; c < D / 64; ++c) {
+                    float4* pv = reinterpret_cast<float4*>(Vs2 + (ty * 4 + i) * LD + c * 64 + tx * 4);
+                    float4 v = *pv;
+                    v.x *= wgt; v.y *= wgt; v.z *= wgt; v.w *= wgt;
+                    *pv = v;
+                }
+            }
+            __syncthreads();
+        }
+        if (a.mode == 1) {
             // Eq. 4 as printed: the value rows become beta (V' - K' S_old); S_old is the state as
             // it stands (the reduce kernel, a later launch, is the only writer)
             float x[4][D / 16];
@@ -701,7 +718,7 @@ __global__ void __launch_bounds__(NT) token_scan_kernel(TokenCommitArgs a)
 // order so that the result does not depend on scheduling.  Also refreshes the bf16 operand
 // copy of S when one is kept.  One thread per 4 state elements.
 __global__ void commit_reduce_kernel(float* __restrict__ state, const float* __restrict__ partials,
-                                     const float* __restrict__ decay,
+                                     const float* __restrict__ decay, int decay_direct,
                                      __nv_bfloat16* __restrict__ state_bf16, int nsplit, int DD,
                                      size_t total4)
 {
@@ -710,7 +727,7 @@ __global__ void commit_reduce_kernel(float* __restrict__ state, const float* __r
     size_t e = t * 4;
     size_t bh = e / DD;
     size_t within = e % DD;
-    float alpha = 1.0f / (1.0f + __expf(-decay[bh]));
+    float alpha = decay_direct ? decay[bh] : 1.0f / (1.0f + __expf(-decay[bh]));
     float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
     const float* p = partials + bh * (size_t)nsplit * DD + within;
     for (int s = 0; s < nsplit; ++s) {
@@ -838,12 +855,47 @@ int launch_commit(const CommitArgs& a, cudaStream_t st)
 
 }  // namespace
 
+// Suffix products of the per-token forget gates of one (stream, head): each thread takes a
+// contiguous run of tokens, the runs are combined through shared memory, everything in log space.
+__global__ void __launch_bounds__(256) decay_weights_kernel(const float* __restrict__ alpha,
+                                                            float* __restrict__ w, float* __restrict__ total,
+                                                            int L, int H)
+{
+    __shared__ float seg_sum[256];
+    const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+    const int seg = (L + 255) / 256;
+    const int l0 = min(L, tid * seg), l1 = min(L, l0 + seg);
+    auto log_alpha = [&](int l) {
+        const float x = alpha[((size_t)b * L + l) * H + h];
+        return x >= 0.0f ? -log1pf(expf(-x)) : x - log1pf(expf(x));
+    };
+    float s = 0.0f;
+    for (int l = l0; l < l1; ++l) s += log_alpha(l);
+    seg_sum[tid] = s;
+    __syncthreads();
+    float after = 0.0f;   // log of the product over every later run
+    for (int t = tid + 1; t < 256; ++t) after += seg_sum[t];
+    float run = after;
+    for (int l = l1 - 1; l >= l0; --l) {
+        w[((size_t)b * L + l) * H + h] = expf(run);
+        run += log_alpha(l);
+    }
+    if (tid == 0) total[(size_t)b * H + h] = expf(run);   // run now covers every token
+}
+
+int decay_weights(const Shape& s, const float* alpha_logits, float* w, float* total, cudaStream_t st)
+{
+    decay_weights_kernel<<<dim3(s.H, s.B), 256, 0, st>>>(alpha_logits, w, total, s.L, s.H);
+    if (int r = check_launch("decay_weights_kernel")) return r;
+    return 1;
+}
+
 int commit_reduce(const CommitArgs& a, cudaStream_t st)
 {
     int DD = a.s.D * a.s.D;
     size_t total4 = (size_t)a.s.B * a.s.H * DD / 4;
     commit_reduce_kernel<<<(unsigned)((total4 + 255) / 256), 256, 0, st>>>(
-        a.state, a.partials, a.decay, a.state_bf16, a.nsplit, DD, total4);
+        a.state, a.partials, a.decay, a.decay_direct ? 1 : 0, a.state_bf16, a.nsplit, DD, total4);
     if (int r = check_launch("commit_reduce_kernel")) return r;
     return 1;
 }

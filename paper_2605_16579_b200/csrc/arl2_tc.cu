@@ -848,10 +848,11 @@ struct TcCommitParams {
     int nsplit;
 };
 
-// kDelta (Eq. 4 as printed, at block level): the value operand of the last MMA is
+// kMode 1 (Eq. 4 as printed, at block level): the value operand of the last MMA is
 // R = diag(beta) (V' - K' S_old) instead of V'; K' S_old is one more MMA per tile (A = K' as
 // written for the last MMA, read d-major; B = the bf16 copy of the state) into TMEM columns 384-511.
-template <bool kDelta>
+// kMode 2 (per-token decay in the gated-linear form): the value rows are scaled by given weights.
+template <int kMode>   // 0: V'; 1: delta rule; 2: per-token weights
 __global__ void __launch_bounds__(kCommitThreads, 1)
 tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                  const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv,
@@ -905,8 +906,8 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         prefetch_tensormap(&tm_k);
         prefetch_tensormap(&tm_v);
         const uint32_t bar_w = bars + 8 * kCBarW;
-        mbar_expect_tx(bar_w, (kDelta ? 3 : 2) * kTileBytes);
-        if (kDelta) {
+        mbar_expect_tx(bar_w, (kMode == 1 ? 3 : 2) * kTileBytes);
+        if (kMode == 1) {
             tma_load_2d(smem_base + kCOffState, &tm_s, bar_w, 0, (b * H + h) * kTile);
             tma_load_2d(smem_base + kCOffState + kHalfBytes, &tm_s, bar_w, 64, (b * H + h) * kTile);
         }
@@ -1002,7 +1003,7 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 *reinterpret_cast<uint4*>(pair + off) = v;
             }
         }
-        if (kDelta) {
+        if (kMode == 1) {
             // ---- prediction K' S_old                                                   (Eq. 4)
             fence_proxy_async_smem();
             tc_fence_before();
@@ -1027,7 +1028,13 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         for (int c = 0; c < 4; ++c)
             tmem_ld32(lane_base + kTile + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
         tmem_wait_ld();
-        if (kDelta) {
+        if (kMode == 2) {
+            const float wgt = (p.beta != nullptr && row < L) ? __ldg(p.beta + ((size_t)b * L + row) * H + h)
+                                                             : (row < L ? 1.0f : 0.0f);
+#pragma unroll
+            for (int e = 0; e < 128; ++e) sreg[e] = __float_as_uint(wgt * __uint_as_float(sreg[e]));
+        }
+        if (kMode == 1) {
             float beta = 1.0f;
             if (p.beta != nullptr) beta = row < L ? sigmoid_fast(__ldg(p.beta + ((size_t)b * L + row) * H + h)) : 0.0f;
 #pragma unroll
@@ -1826,15 +1833,18 @@ int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat
 {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc_commit_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(tc_commit_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kCommitSmemBytes);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(tc_commit_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            e = cudaFuncSetAttribute(tc_commit_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kCommitSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(tc_commit_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      kCommitSmemBytes);
         if (e != cudaSuccess) { set_error("cudaFuncSetAttribute(tc_commit_kernel, %d): %s", kCommitSmemBytes, cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
         attr_set = true;
     }
-    if (a.delta && a.state_bf16 == nullptr) {
+    if (a.mode == 1 && a.state_bf16 == nullptr) {
         set_error("tc_commit: the delta rule needs the bf16 copy of the state");
         return ARL2_ERR_INVALID_ARG;
     }
@@ -1843,7 +1853,7 @@ int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat
     if (int r = make_map_blhd(&tm_v, a.v, a.s)) return r;
     if (int r = make_map_rows(&tm_wk, wk_op, (size_t)a.s.H * kTile)) return r;
     if (int r = make_map_rows(&tm_wv, wv_op, (size_t)a.s.H * kTile)) return r;
-    if (a.delta) {
+    if (a.mode == 1) {
         if (int r = make_map_rows(&tm_s, a.state_bf16, (size_t)a.s.B * a.s.H * kTile)) return r;
     } else {
         tm_s = tm_wk;   // not read
@@ -1856,10 +1866,12 @@ int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat
     p.status = a.status;
     p.nsplit = a.nsplit;
     dim3 grid(a.nsplit, a.s.H, a.s.B);
-    if (a.delta)
-        tc_commit_kernel<true><<<grid, kCommitThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, tm_wv, tm_s, p);
+    if (a.mode == 1)
+        tc_commit_kernel<1><<<grid, kCommitThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, tm_wv, tm_s, p);
+    else if (a.mode == 2)
+        tc_commit_kernel<2><<<grid, kCommitThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, tm_wv, tm_s, p);
     else
-        tc_commit_kernel<false><<<grid, kCommitThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, tm_wv, tm_s, p);
+        tc_commit_kernel<0><<<grid, kCommitThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, tm_wv, tm_s, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_error("launch of tc_commit_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
     int m = commit_reduce(a, st);

@@ -116,6 +116,23 @@ class Pair:
             err = err[mask]
         return float(err.max())
 
+    def commit_decay_tokens(self, kc, vc, alpha, heads=None):
+        """Gated-linear commit with per-token forget gates on both sides; worst per-head error of S."""
+        d = self.dev
+        self.layer.commit_decay_tokens(kc.to(d), vc.to(d), alpha.to(d))
+        got = self.layer.get_state().numpy().astype(np.float64)
+        self.S_ref = self.oracle.commit_decay_tokens(kc, vc, self.S_ref, alpha, self.wk, self.wv,
+                                                     self.cos, self.sin, eps=self.eps, heads=heads)
+        assert np.isfinite(got).all()
+        err = head_errors(got, self.S_ref, head_axis_first=True)
+        if heads is not None:
+            mask = np.zeros(err.shape, dtype=bool)
+            for b, h in heads:
+                mask[b, h] = True
+            self.S_ref[~mask] = got[~mask]
+            err = err[mask]
+        return float(err.max())
+
     def commit_tokens(self, kc, vc, alpha, beta, heads=None):
         """Token-sequential commit with per-token gates on both sides; worst per-head error of S."""
         d = self.dev

@@ -441,6 +441,30 @@ def test_token_gates_special_cases(oracle):
     assert not np.allclose(got[0, 1], S0[0, 1])
 
 
+def test_per_token_decay_closed_form(oracle):
+    """S <- alpha_j S + k_j^T v_j in order equals (prod alpha) S_0 + sum_j (prod_{i>j} alpha_i) k_j^T v_j
+    (library cumulative products and einsum); with every gate open it is the block-level commit."""
+    B, L, H, D = 2, 11, 2, 8
+    k, v, S0 = rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, H, D, D)
+    al = rnd(B, L, H) + 1.0
+    wk, wv = np.eye(D) + 0.1 * rnd(H, D, D), np.eye(D) + 0.1 * rnd(H, D, D)
+    cos, sin = tables(L, D)
+    got = oracle.commit_decay_tokens(k, v, S0, al, wk, wv, cos, sin)
+    kf = torch.from_numpy(oracle.feature(k, wk, cos, sin, 1e-6, 0))
+    vf = torch.from_numpy(oracle.feature(v, wv, None, None, 1e-6, 1))
+    a = torch.from_numpy(sig(al))
+    suffix = torch.flip(torch.cumprod(torch.flip(a, dims=[1]), dim=1), dims=[1])      # prod_{i>=j}
+    w = suffix / a                                                                    # prod_{i>j}
+    ref = suffix[:, 0][..., None, None] * torch.from_numpy(S0) \
+        + torch.einsum("blhd,blhe->bhde", kf * w[..., None], vf)
+    np.testing.assert_allclose(got, ref.numpy(), rtol=1e-11, atol=1e-13)
+    ones = oracle.commit_decay_tokens(k, v, S0, np.full((B, L, H), 800.0), wk, wv, cos, sin)
+    block = oracle.commit(k, v, np.full((B, H), 800.0), S0, wk, wv, cos, sin)
+    np.testing.assert_allclose(ones, block, rtol=1e-12, atol=1e-14)
+    part = oracle.commit_decay_tokens(k, v, S0, al, heads=[(1, 0)])
+    np.testing.assert_array_equal(part[0], S0[0])
+
+
 def test_state_norm_stays_bounded(oracle):
     """Unit-norm keys and alpha <= alpha_max < 1: |S_T|_F <= max_t |K'^T V'|_F / (1 - alpha_max)."""
     B, L, H, D, T = 1, 12, 2, 8, 60
