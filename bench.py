@@ -336,30 +336,64 @@ def run_ours(args):
     layer.sync_status()
 
     # end to end through the same entry points with HOST buffers: every pass copies its inputs
-    # from pinned host memory and its output back inside the timed region
+    # from pinned host memory and its output back inside the timed region.  Copies run on their own
+    # streams with double-buffered staging, as a caller would: the upload of the next pass and the
+    # download of the previous one overlap the kernels (PCIe carries both directions at once).
     e2e_blocks = max(1, min(args.steps, 5))
     pin_sets = [tuple(t.pin_memory() for t in hs) for hs in host_sets]
     pin_commit = tuple(t.pin_memory() for t in host_commit)
-    pin_out = torch.empty(out.shape, dtype=out.dtype).pin_memory()
-    stage = tuple(torch.empty_like(t) for t in dev_sets[0])
+    pin_outs = [torch.empty(out.shape, dtype=out.dtype).pin_memory() for _ in range(2)]
+    stages = [tuple(torch.empty_like(t) for t in dev_sets[0]) for _ in range(2)]
+    outs = [torch.empty_like(out) for _ in range(2)]
     stage_c = tuple(torch.empty_like(t) for t in dev_commit)
+    s_main = torch.cuda.current_stream()
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    ev_in = [torch.cuda.Event() for _ in range(2)]        # staging slot filled
+    ev_done = [torch.cuda.Event() for _ in range(2)]      # kernels of the slot finished
+    ev_out = [torch.cuda.Event() for _ in range(2)]       # output slot downloaded
+    ev_c_in, ev_c_done = torch.cuda.Event(), torch.cuda.Event()
+    for e in ev_done + ev_out + [ev_c_done]:
+        e.record(s_main)
+    n_pass = [0]
 
     def block_host(i):
         for s in range(cfg.steps):
-            for d, h in zip(stage, pin_sets[(i * cfg.steps + s) % RING]):
+            slot = n_pass[0] & 1
+            n_pass[0] += 1
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(ev_done[slot])            # the kernels that read this slot are done
+                for d, h in zip(stages[slot], pin_sets[(i * cfg.steps + s) % RING]):
+                    d.copy_(h, non_blocking=True)
+                ev_in[slot].record(s_in)
+            s_main.wait_event(ev_in[slot])
+            s_main.wait_event(ev_out[slot])               # the previous output of this slot is on the host
+            layer.denoise_step(*stages[slot], out=outs[slot])
+            ev_done[slot].record(s_main)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_done[slot])
+                pin_outs[slot].copy_(outs[slot], non_blocking=True)
+                ev_out[slot].record(s_out)
+        with torch.cuda.stream(s_in):
+            s_in.wait_event(ev_c_done)
+            for d, h in zip(stage_c, pin_commit):
                 d.copy_(h, non_blocking=True)
-            layer.denoise_step(*stage, out=out)
-            pin_out.copy_(out, non_blocking=True)
-        for d, h in zip(stage_c, pin_commit):
-            d.copy_(h, non_blocking=True)
+            ev_c_in.record(s_in)
+        s_main.wait_event(ev_c_in)
         layer.commit(*stage_c)
+        ev_c_done.record(s_main)
+
+    def drain():
+        s_main.wait_stream(s_in)
+        s_main.wait_stream(s_out)
 
     block_host(0)
+    drain()
     barrier()
     h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     h0.record()
     for i in range(e2e_blocks):
         block_host(i)
+    drain()                                               # every download has landed before the clock stops
     h1.record()
     barrier()
     ms_e2e = h0.elapsed_time(h1)
