@@ -265,8 +265,10 @@ int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const voi
     const void* k_rot = d_k;
     if (ctx->rope_cos != nullptr) {
         void* buf = ctx->ws + ctx->lay.k_rot;
-        int r = account(ctx, simt_rope_k(ctx->shape, ctx->cfg.io_dtype, d_k, ctx->rope_cos,
-                                         ctx->rope_sin, buf, st));
+        int r = ctx->use_tc
+                    ? account(ctx, tc_rope_k(ctx->shape, d_k, ctx->ws + ctx->lay.rope_h, buf, st))
+                    : account(ctx, simt_rope_k(ctx->shape, ctx->cfg.io_dtype, d_k, ctx->rope_cos,
+                                               ctx->rope_sin, buf, st));
         if (r != ARL2_OK) return r;
         k_rot = buf;
     }

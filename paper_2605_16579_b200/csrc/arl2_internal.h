@@ -106,6 +106,8 @@ bool tc_supported(const arl2_config& c);
 int tc_prepare_map(const void* w, __nv_bfloat16* w_op, int H, cudaStream_t st);
 // cos, sin [L, 64] fp32 -> out [L, 64] half2 (cos, sin): one 256-byte row per token
 int tc_prepare_rope(const float* cos_t, const float* sin_t, void* out, int L, cudaStream_t st);
+// k_rot = RoPE(k), bf16 [B, L, H, 128], from the packed table tc_prepare_rope wrote
+int tc_rope_k(const Shape& s, const void* k, const void* rope_h, void* k_rot, cudaStream_t st);
 int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* state_bf16,
             cudaStream_t st);
 int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat16* wv_op,

@@ -1689,6 +1689,30 @@ __global__ void pack_rope_kernel(const float* __restrict__ cos_t, const float* _
     out[dst] = l < L ? __floats2half2_rn(cos_t[t], sin_t[t]) : __floats2half2_rn(0.0f, 0.0f);
 }
 
+// k_rot = RoPE(k) for bf16 [B, L, H, 128] from the packed half2 table: 8 elements (4 rotation pairs,
+// one 16-byte table vector) per thread.  The same table rotates Q inside the step kernel.
+__global__ void tc_rope_k_kernel(const uint4* __restrict__ k, const uint4* __restrict__ rope_h,
+                                 uint4* __restrict__ out, int L, int H, size_t total8)
+{
+    const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= total8) return;
+    const int c = (int)(t & 15);                     // vector of the 128-element row
+    const int l = (int)((t >> 4) / H % L);           // token
+    const uint4 raw = __ldg(k + t);
+    const uint4 cs = __ldg(rope_h + ((size_t)(l >> 5) * 16 + c) * 32 + (l & 31));
+    uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+    const uint32_t h2[4] = {cs.x, cs.y, cs.z, cs.w};
+#pragma unroll
+    for (int m = 0; m < 4; ++m) {
+        float cc, ss;
+        unpack_cs(h2[m], cc, ss);
+        const float x0 = __uint_as_float(w[m] << 16);
+        const float x1 = __uint_as_float(w[m] & 0xFFFF0000u);
+        w[m] = pack_bf16(x0 * cc - x1 * ss, x0 * ss + x1 * cc);
+    }
+    out[t] = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
 // out[h][o][i] = w[h][i][o] (bf16), or the identity when w is null: the K-major B operand of
 // U = Q W_phi (B[n][k] = W[k][n]).
 __global__ void transpose_map_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ out,
@@ -1769,6 +1793,16 @@ int tc_prepare_map(const void* w, __nv_bfloat16* w_op, int H, cudaStream_t st)
         static_cast<const __nv_bfloat16*>(w), w_op, kTile, total);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_error("launch of transpose_map_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
+    return 1;
+}
+
+int tc_rope_k(const Shape& s, const void* k, const void* rope_h, void* k_rot, cudaStream_t st)
+{
+    const size_t total8 = (size_t)s.B * s.L * s.H * kTile / 8;
+    tc_rope_k_kernel<<<(unsigned)((total8 + 255) / 256), 256, 0, st>>>(
+        static_cast<const uint4*>(k), static_cast<const uint4*>(rope_h), static_cast<uint4*>(k_rot), s.L, s.H, total8);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_error("launch of tc_rope_k_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
     return 1;
 }
 
