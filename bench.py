@@ -57,6 +57,15 @@ def step_flops(cfg):
     return cfg.B * cfg.H * (4.0 * cfg.L * cfg.L * cfg.D + 4.0 * cfg.L * cfg.D * cfg.D)
 
 
+def commit_bytes_flops(cfg):
+    """Algorithmic HBM bytes and tensor flops of one gated-linear commit: K_c, V_c in, S read and
+    written, the two maps; U_k, U_v and K'^T V' contractions."""
+    e = cfg.elem_bytes
+    byts = cfg.B * cfg.H * (2.0 * cfg.L * cfg.D * e + 8.0 * cfg.D * cfg.D + 2.0 * cfg.D * cfg.D * e)
+    flops = cfg.B * cfg.H * 6.0 * cfg.L * cfg.D * cfg.D
+    return byts, flops
+
+
 def step_bytes(cfg):
     """Algorithmic HBM bytes of one denoise pass: Q, K, V in, O out, gate logits, S and W_phi_q."""
     e = cfg.elem_bytes
@@ -511,6 +520,14 @@ def run_ours(args):
             "clocks": clocks,
             "horizon": horizon_report(block_ms, mem_marks, layer.workspace_bytes + layer.state.numel() * 4),
             "commit_ms": commit_ms,
+            # the commit is HBM-bound by its arithmetic intensity (about 175 flop/B); the same bytes
+            # serve the delta and per-token-decay variants, whose extra work is on-chip
+            "commit_roofline": {
+                "bound": "hbm", "unit": "GB/s", "peak": pk["hbm_gbs"],
+                "algorithmic_bytes": commit_bytes_flops(cfg)[0], "algorithmic_flops": commit_bytes_flops(cfg)[1],
+                "achieved": {k: commit_bytes_flops(cfg)[0] / (v * 1e-3) / 1e9 for k, v in commit_ms.items()},
+                "frac": {k: commit_bytes_flops(cfg)[0] / (v * 1e-3) / 1e9 / pk["hbm_gbs"] for k, v in commit_ms.items()},
+            },
             "teacher_horizon": teacher,
         }
         if world == 1 and not args.no_cpu_baseline:

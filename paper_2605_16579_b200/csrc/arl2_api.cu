@@ -78,7 +78,7 @@ Layout make_layout(const arl2_config& c)
     size_t off = 0;
     l.status = off;     off += align_up(kStatusWords * sizeof(uint32_t));
     l.k_rot = off;      off += align_up(tensor);
-    l.partials = off;   off += align_up((size_t)c.B * c.H * l.nsplit * dd * sizeof(float));
+    l.partials = off;   off += align_up((size_t)c.B * c.H * (l.nsplit + 1) * dd * sizeof(float));
     l.state_bf16 = off; off += align_up((size_t)c.B * c.H * dd * 2);
     l.wq_op = off;      off += align_up((size_t)c.H * dd * 2);
     l.wk_op = off;      off += align_up((size_t)c.H * dd * 2);

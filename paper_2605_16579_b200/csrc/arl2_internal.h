@@ -64,6 +64,12 @@ struct CommitArgs {
     int mode = 0;
     const float* beta = nullptr;   // [B, L, H]: logits (mode 1) or weights (mode 2); nullptr = 1
     bool decay_direct = false;     // `decay` holds the factors themselves, not logits
+    // How the partial sums of a head are laid out for the reduce kernel: nsplit slots of fixed
+    // 512-token chunks (run_share == 0), or the tensor-core kernel's runs of run_share tiles over
+    // the flattened tile sequence (a head's slots are the CTAs its run_ntile tiles fall into)
+    int run_share = 0;
+    int run_ntile = 0;
+    int nslot = 0;                 // slots per head in `partials` (0: nsplit)
 };
 
 // Eq. 4 token by token with per-token gates (chunkwise form): the two launches share these.

@@ -720,7 +720,7 @@ __global__ void __launch_bounds__(NT) token_scan_kernel(TokenCommitArgs a)
 __global__ void commit_reduce_kernel(float* __restrict__ state, const float* __restrict__ partials,
                                      const float* __restrict__ decay, int decay_direct,
                                      __nv_bfloat16* __restrict__ state_bf16, int nsplit, int DD,
-                                     size_t total4)
+                                     size_t total4, int run_share, int run_ntile, int nslot)
 {
     size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= total4) return;
@@ -729,8 +729,15 @@ __global__ void commit_reduce_kernel(float* __restrict__ state, const float* __r
     size_t within = e % DD;
     float alpha = decay_direct ? decay[bh] : 1.0f / (1.0f + __expf(-decay[bh]));
     float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-    const float* p = partials + bh * (size_t)nsplit * DD + within;
-    for (int s = 0; s < nsplit; ++s) {
+    int nparts = nsplit, stride = nsplit;
+    if (run_share > 0) {   // the slots are the runs this head's tiles fall into
+        const int first = (int)((bh * run_ntile) / run_share);
+        const int last = (int)((bh * run_ntile + run_ntile - 1) / run_share);
+        nparts = last - first + 1;
+        stride = nslot;
+    }
+    const float* p = partials + bh * (size_t)stride * DD + within;
+    for (int s = 0; s < nparts; ++s) {
         float4 x = *reinterpret_cast<const float4*>(p + (size_t)s * DD);
         sum.x += x.x; sum.y += x.y; sum.z += x.z; sum.w += x.w;
     }
@@ -895,7 +902,8 @@ int commit_reduce(const CommitArgs& a, cudaStream_t st)
     int DD = a.s.D * a.s.D;
     size_t total4 = (size_t)a.s.B * a.s.H * DD / 4;
     commit_reduce_kernel<<<(unsigned)((total4 + 255) / 256), 256, 0, st>>>(
-        a.state, a.partials, a.decay, a.decay_direct ? 1 : 0, a.state_bf16, a.nsplit, DD, total4);
+        a.state, a.partials, a.decay, a.decay_direct ? 1 : 0, a.state_bf16, a.nsplit, DD, total4,
+        a.run_share, a.run_ntile, a.nslot);
     if (int r = check_launch("commit_reduce_kernel")) return r;
     return 1;
 }

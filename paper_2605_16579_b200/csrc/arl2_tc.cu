@@ -819,15 +819,18 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 }
 
 // ---------------------------------------------------------------------------------------------
-// Commit kernel (Eq. 3, Eq. 4 in its gated-linear form): one CTA per (stream b, head h, chunk of
-// 512 tokens), 128 threads.  Per 128-token tile:
+// Commit kernel (Eq. 3, Eq. 4 in its gated-linear form): 128 threads per CTA; the 128-token tiles of
+// all (stream, head) units form one flattened sequence that is cut into equal runs, one run per CTA
+// (one CTA per SM when there is enough work), so a run may cross from one head into the next.
+// Per tile:
 //   U_k = K_c W_phi_k, U_v = V_c W_phi_v            two MMAs into TMEM (columns 0-127, 128-255)
 //   K'  = L2Norm(RoPE(U_k)), V' = U_v               one thread per token; written as bf16 over
 //                                                   the raw tiles, in the swizzled tile layout
 //   dS += K'^T V'                                   MMA with both operands token-major (the
 //                                                   contraction runs over the tile's tokens)
-// dS (TMEM columns 256-383, fp32) is written to this chunk's slot of the partial-sum buffer; the
-// reduce kernel adds the chunks in a fixed order and applies the gated decay.
+// dS (TMEM columns 256-383, fp32) accumulates over the tiles of one head inside a run and is then
+// written to that (head, CTA) slot of the partial-sum buffer; the assignment of tiles to CTAs and
+// slots is static, and the reduce kernel adds a head's slots in index order and applies the decay.
 // ---------------------------------------------------------------------------------------------
 constexpr int kCOffWk = 0;
 constexpr int kCOffWv = kTileBytes;
@@ -843,15 +846,44 @@ struct TcCommitParams {
     Shape s;
     const uint4* rope_h;   // warp-interleaved half2 (cos, sin) table, or nullptr
     const float* beta;     // [B, L, H] learning-rate logits (delta rule), or nullptr = 1
-    float* partials;     // [B, H, nsplit, 128, 128] fp32
+    float* partials;     // [B * H, nslot, 128, 128] fp32
     uint32_t* status;
-    int nsplit;
+    int ntile;           // 128-token tiles per (stream, head)
+    int total_tiles;     // B * H * ntile
+    int share;           // tiles per CTA: CTA c takes tiles [c * share, (c + 1) * share) of the flattened order
+    int nslot;           // partial-sum slots per (stream, head)
 };
 
 // kMode 1 (Eq. 4 as printed, at block level): the value operand of the last MMA is
 // R = diag(beta) (V' - K' S_old) instead of V'; K' S_old is one more MMA per tile (A = K' as
 // written for the last MMA, read d-major; B = the bf16 copy of the state) into TMEM columns 384-511.
 // kMode 2 (per-token decay in the gated-linear form): the value rows are scaled by given weights.
+__device__ __forceinline__ void store_row_bf16_swizzled(uint8_t* tile, int r, const uint32_t (&x)[128], float f)
+{
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+        uint4 v;
+        v.x = pack_bf16(__uint_as_float(x[c * 8 + 0]) * f, __uint_as_float(x[c * 8 + 1]) * f);
+        v.y = pack_bf16(__uint_as_float(x[c * 8 + 2]) * f, __uint_as_float(x[c * 8 + 3]) * f);
+        v.z = pack_bf16(__uint_as_float(x[c * 8 + 4]) * f, __uint_as_float(x[c * 8 + 5]) * f);
+        v.w = pack_bf16(__uint_as_float(x[c * 8 + 6]) * f, __uint_as_float(x[c * 8 + 7]) * f);
+        const int off = (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+        *reinterpret_cast<uint4*>(tile + off) = v;
+    }
+}
+__device__ __forceinline__ void store_row_bf16_global(__nv_bfloat16* dst, const uint32_t (&x)[128], float f)
+{
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+        uint4 v;
+        v.x = pack_bf16(__uint_as_float(x[c * 8 + 0]) * f, __uint_as_float(x[c * 8 + 1]) * f);
+        v.y = pack_bf16(__uint_as_float(x[c * 8 + 2]) * f, __uint_as_float(x[c * 8 + 3]) * f);
+        v.z = pack_bf16(__uint_as_float(x[c * 8 + 4]) * f, __uint_as_float(x[c * 8 + 5]) * f);
+        v.w = pack_bf16(__uint_as_float(x[c * 8 + 6]) * f, __uint_as_float(x[c * 8 + 7]) * f);
+        *reinterpret_cast<uint4*>(dst + c * 8) = v;
+    }
+}
+
 template <int kMode>   // 0: V'; 1: delta rule; 2: per-token weights
 __global__ void __launch_bounds__(kCommitThreads, 1)
 tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -868,11 +900,10 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     const Abort ab{abort_flag, p.status};
 
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
     const int L = p.s.L, H = p.s.H;
-    const int l0 = split * kCommitChunk;
-    const int l1 = min(L, l0 + kCommitChunk);
-    const int ntiles = (l1 - l0 + kTile - 1) / kTile;
+    // this CTA's run of tiles in the flattened (stream, head, tile) order; it may cross heads
+    const int g_begin = (int)blockIdx.x * p.share;
+    const int n_my = min(p.total_tiles, g_begin + p.share) - g_begin;
 
     if (tid == 0) {
         for (int i = 0; i < kCNumBars; ++i) mbar_init(bars + 8 * i, 1);
@@ -890,34 +921,30 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
 
-    auto load_pair = [&](int i) {   // tile i of the chunk into pair i & 1
-        const uint32_t bar = bars + 8 * (kCBarFull0 + (i & 1));
-        const uint32_t dst = smem_base + kCOffPair + (i & 1) * 2 * kTileBytes;
+    auto load_pair = [&](int k) {   // k-th tile of the run into pair k & 1
+        const int g = g_begin + k, bh = g / p.ntile, tl = g - bh * p.ntile;
+        const int hb = bh / H, hh = bh - hb * H;
+        const uint32_t bar = bars + 8 * (kCBarFull0 + (k & 1));
+        const uint32_t dst = smem_base + kCOffPair + (k & 1) * 2 * kTileBytes;
         mbar_expect_tx(bar, 2 * kTileBytes);
-        tma_load_4d(dst, &tm_k, bar, 0, h, l0 + i * kTile, b);
-        tma_load_4d(dst + kHalfBytes, &tm_k, bar, 64, h, l0 + i * kTile, b);
-        tma_load_4d(dst + kTileBytes, &tm_v, bar, 0, h, l0 + i * kTile, b);
-        tma_load_4d(dst + kTileBytes + kHalfBytes, &tm_v, bar, 64, h, l0 + i * kTile, b);
+        tma_load_4d(dst, &tm_k, bar, 0, hh, tl * kTile, hb);
+        tma_load_4d(dst + kHalfBytes, &tm_k, bar, 64, hh, tl * kTile, hb);
+        tma_load_4d(dst + kTileBytes, &tm_v, bar, 0, hh, tl * kTile, hb);
+        tma_load_4d(dst + kTileBytes + kHalfBytes, &tm_v, bar, 64, hh, tl * kTile, hb);
     };
-
-    bool ok = true;
-    int loads_issued = 0;
-    if (tid == 0) {
-        prefetch_tensormap(&tm_k);
-        prefetch_tensormap(&tm_v);
+    auto load_head = [&](int bh) {   // the maps (and the bf16 state) of one (stream, head)
+        const int hh = bh % H;
         const uint32_t bar_w = bars + 8 * kCBarW;
         mbar_expect_tx(bar_w, (kMode == 1 ? 3 : 2) * kTileBytes);
         if (kMode == 1) {
-            tma_load_2d(smem_base + kCOffState, &tm_s, bar_w, 0, (b * H + h) * kTile);
-            tma_load_2d(smem_base + kCOffState + kHalfBytes, &tm_s, bar_w, 64, (b * H + h) * kTile);
+            tma_load_2d(smem_base + kCOffState, &tm_s, bar_w, 0, bh * kTile);
+            tma_load_2d(smem_base + kCOffState + kHalfBytes, &tm_s, bar_w, 64, bh * kTile);
         }
-        tma_load_2d(smem_base + kCOffWk, &tm_wk, bar_w, 0, h * kTile);
-        tma_load_2d(smem_base + kCOffWk + kHalfBytes, &tm_wk, bar_w, 64, h * kTile);
-        tma_load_2d(smem_base + kCOffWv, &tm_wv, bar_w, 0, h * kTile);
-        tma_load_2d(smem_base + kCOffWv + kHalfBytes, &tm_wv, bar_w, 64, h * kTile);
-        for (int i = 0; i < 2 && i < ntiles; ++i, ++loads_issued) load_pair(i);
-        ok = wait_bar(bar_w, 0, ab, 80);
-    }
+        tma_load_2d(smem_base + kCOffWk, &tm_wk, bar_w, 0, hh * kTile);
+        tma_load_2d(smem_base + kCOffWk + kHalfBytes, &tm_wk, bar_w, 64, hh * kTile);
+        tma_load_2d(smem_base + kCOffWv, &tm_wv, bar_w, 0, hh * kTile);
+        tma_load_2d(smem_base + kCOffWv + kHalfBytes, &tm_wv, bar_w, 64, hh * kTile);
+    };
 
     const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0, 0) >> 32);
     constexpr uint32_t kLboK = 1u << 16;
@@ -931,33 +958,61 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     constexpr uint32_t idesc_ds = idesc_bf16(kTile, kTile, 1, 1);   // K'^T V': both token-major
     constexpr uint32_t idesc_ps = idesc_bf16(kTile, kTile, 0, 1);   // K' S_old: A d-major, B = S rows
 
-    uint32_t sreg[128];
-    for (int i = 0; i < ntiles; ++i) {
-        const int s = i & 1;
-        uint8_t* pair = smem + kCOffPair + s * 2 * kTileBytes;
-        const uint32_t pair_addr = smem_base + kCOffPair + s * 2 * kTileBytes;
-        if (tid == 0 && ok) {
-            ok = wait_bar(bars + 8 * (kCBarFull0 + s), (uint32_t)((i >> 1) & 1), ab, 81);
-            if (ok) {
-                tc_fence_after();
+    bool ok = true;
+    int loads_issued = 0;
+    uint32_t w_loads = 0;   // head loads issued so far (issuing thread)
+    uint32_t w_seen = 0;    // head loads the issuing thread has waited for
+    // U_k = K_c W_phi_k, U_v = V_c W_phi_v of the run's k-th tile into TMEM columns 0-255
+    auto issue_u = [&](int k) {
+        if (w_seen < w_loads) {   // the tile belongs to a head whose maps were requested since
+            if (!wait_bar(bars + 8 * kCBarW, (w_loads - 1) & 1, ab, 80)) return false;
+            w_seen = w_loads;
+        }
+        const uint32_t pa = smem_base + kCOffPair + (k & 1) * 2 * kTileBytes;
+        if (!wait_bar(bars + 8 * (kCBarFull0 + (k & 1)), (uint32_t)((k >> 1) & 1), ab, 81)) return false;
+        tc_fence_after();
 #pragma unroll
-                for (int u = 0; u < 2; ++u) {   // U_k then U_v
-                    const uint32_t a_lo = ((pair_addr + u * kTileBytes) >> 4) | kLboK;
-                    const uint32_t b_lo = ((smem_base + (u ? kCOffWv : kCOffWk)) >> 4) | kLboK;
+        for (int u = 0; u < 2; ++u) {   // U_k then U_v
+            const uint32_t a_lo = ((pa + u * kTileBytes) >> 4) | kLboK;
+            const uint32_t b_lo = ((smem_base + (u ? kCOffWv : kCOffWk)) >> 4) | kLboK;
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint32_t koff = (uint32_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
-                        mma_ss(tmem_base + u * kTile, desc64(a_lo + koff), desc64(b_lo + koff), idesc_u, ks > 0);
-                    }
-                }
-                mma_commit(bars + 8 * kCBarU);
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint32_t koff = (uint32_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
+                mma_ss(tmem_base + u * kTile, desc64(a_lo + koff), desc64(b_lo + koff), idesc_u, ks > 0);
             }
         }
-        if (!wait_bar(bars + 8 * kCBarU, (uint32_t)(i & 1), ab, 82)) break;
+        mma_commit(bars + 8 * kCBarU);
+        return true;
+    };
+    if (tid == 0 && n_my > 0) {
+        prefetch_tensormap(&tm_k);
+        prefetch_tensormap(&tm_v);
+        load_head(g_begin / p.ntile);
+        ++w_loads;
+        for (int k = 0; k < 2 && k < n_my; ++k, ++loads_issued) load_pair(k);
+        ok = issue_u(0);
+    }
+
+    uint32_t sreg[128];
+    for (int k = 0; k < n_my; ++k) {
+        const int g = g_begin + k, bh = g / p.ntile, tl = g - bh * p.ntile;
+        const int b = bh / H, h = bh - b * H;
+        const bool seg_first = k == 0 || tl == 0;                    // first tile of this head in my run
+        const bool seg_last = k + 1 == n_my || tl + 1 == p.ntile;    // last one
+        const bool next_new_head = k + 1 < n_my && tl + 1 == p.ntile;
+        uint8_t* pair = smem + kCOffPair + (k & 1) * 2 * kTileBytes;
+        const uint32_t pair_addr = smem_base + kCOffPair + (k & 1) * 2 * kTileBytes;
+        if (!wait_bar(bars + 8 * kCBarU, (uint32_t)(k & 1), ab, 82)) break;
         tc_fence_after();
+        // U(k) is complete: nothing reads this head's maps any more (the delta rule still needs its
+        // state tile for the prediction below)
+        if (kMode != 1 && tid == 0 && ok && next_new_head) {
+            load_head(bh + 1);
+            ++w_loads;
+        }
 
         const int r = tid;                       // token row of the tile
-        const int row = l0 + i * kTile + r;
+        const int row = tl * kTile + r;
         // ---- K' = L2Norm(RoPE(U_k))
 #pragma unroll
         for (int c = 0; c < 4; ++c)
@@ -988,20 +1043,11 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 #pragma unroll
             for (int c = 0; c < 128; c += 4) {
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    ss4[k] = fmaf(__uint_as_float(sreg[c + k]), __uint_as_float(sreg[c + k]), ss4[k]);
+                for (int q = 0; q < 4; ++q)
+                    ss4[q] = fmaf(__uint_as_float(sreg[c + q]), __uint_as_float(sreg[c + q]), ss4[q]);
             }
             const float f = rsqrtf((ss4[0] + ss4[1]) + (ss4[2] + ss4[3]) + p.s.eps);
-#pragma unroll
-            for (int c = 0; c < 16; ++c) {
-                uint4 v;
-                v.x = pack_bf16(__uint_as_float(sreg[c * 8 + 0]) * f, __uint_as_float(sreg[c * 8 + 1]) * f);
-                v.y = pack_bf16(__uint_as_float(sreg[c * 8 + 2]) * f, __uint_as_float(sreg[c * 8 + 3]) * f);
-                v.z = pack_bf16(__uint_as_float(sreg[c * 8 + 4]) * f, __uint_as_float(sreg[c * 8 + 5]) * f);
-                v.w = pack_bf16(__uint_as_float(sreg[c * 8 + 6]) * f, __uint_as_float(sreg[c * 8 + 7]) * f);
-                const int off = (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
-                *reinterpret_cast<uint4*>(pair + off) = v;
-            }
+            store_row_bf16_swizzled(pair, r, sreg, f);
         }
         if (kMode == 1) {
             // ---- prediction K' S_old                                                   (Eq. 4)
@@ -1020,23 +1066,24 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 }
                 mma_commit(bars + 8 * kCBarP);
             }
-            if (!wait_bar(bars + 8 * kCBarP, (uint32_t)(i & 1), ab, 85)) break;
+            if (!wait_bar(bars + 8 * kCBarP, (uint32_t)(k & 1), ab, 85)) break;
             tc_fence_after();
+            if (tid == 0 && ok && next_new_head) {   // the prediction was the last reader of the state tile
+                load_head(bh + 1);
+                ++w_loads;
+            }
         }
-        // ---- V' = U_v, or R = beta (V' - K' S_old)
+        // ---- V' = U_v, or R = beta (V' - K' S_old), or w V'
 #pragma unroll
         for (int c = 0; c < 4; ++c)
             tmem_ld32(lane_base + kTile + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
         tmem_wait_ld();
-        if (kMode == 2) {
-            const float wgt = (p.beta != nullptr && row < L) ? __ldg(p.beta + ((size_t)b * L + row) * H + h)
-                                                             : (row < L ? 1.0f : 0.0f);
-#pragma unroll
-            for (int e = 0; e < 128; ++e) sreg[e] = __float_as_uint(wgt * __uint_as_float(sreg[e]));
-        }
+        float vscale = 1.0f;
+        if (kMode == 2)
+            vscale = (p.beta != nullptr && row < L) ? __ldg(p.beta + ((size_t)b * L + row) * H + h)
+                                                    : (row < L ? 1.0f : 0.0f);
         if (kMode == 1) {
-            float beta = 1.0f;
-            if (p.beta != nullptr) beta = row < L ? sigmoid_fast(__ldg(p.beta + ((size_t)b * L + row) * H + h)) : 0.0f;
+            if (p.beta != nullptr) vscale = row < L ? sigmoid_fast(__ldg(p.beta + ((size_t)b * L + row) * H + h)) : 0.0f;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t pr[32];
@@ -1044,19 +1091,10 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 tmem_wait_ld();
 #pragma unroll
                 for (int e = 0; e < 32; ++e)
-                    sreg[c * 32 + e] = __float_as_uint(beta * (__uint_as_float(sreg[c * 32 + e]) - __uint_as_float(pr[e])));
+                    sreg[c * 32 + e] = __float_as_uint(__uint_as_float(sreg[c * 32 + e]) - __uint_as_float(pr[e]));
             }
         }
-#pragma unroll
-        for (int c = 0; c < 16; ++c) {
-            uint4 v;
-            v.x = pack_bf16(__uint_as_float(sreg[c * 8 + 0]), __uint_as_float(sreg[c * 8 + 1]));
-            v.y = pack_bf16(__uint_as_float(sreg[c * 8 + 2]), __uint_as_float(sreg[c * 8 + 3]));
-            v.z = pack_bf16(__uint_as_float(sreg[c * 8 + 4]), __uint_as_float(sreg[c * 8 + 5]));
-            v.w = pack_bf16(__uint_as_float(sreg[c * 8 + 6]), __uint_as_float(sreg[c * 8 + 7]));
-            const int off = (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
-            *reinterpret_cast<uint4*>(pair + kTileBytes + off) = v;
-        }
+        store_row_bf16_swizzled(pair + kTileBytes, r, sreg, vscale);
         fence_proxy_async_smem();
         tc_fence_before();
         __syncthreads();
@@ -1068,34 +1106,43 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)   // 16 tokens per step
                 mma_ss(tmem_base + 2 * kTile, desc64(a_lo + (uint32_t)(ks * (2048 >> 4))),
-                       desc64(b_lo + (uint32_t)(ks * (2048 >> 4))), idesc_ds, (i > 0 || ks > 0) ? 1u : 0u);
+                       desc64(b_lo + (uint32_t)(ks * (2048 >> 4))), idesc_ds, (!seg_first || ks > 0) ? 1u : 0u);
             mma_commit(bars + 8 * kCBarS);
-            // the pair may be overwritten (and TMEM columns 0-255 reused) once this MMA is done
-            ok = wait_bar(bars + 8 * kCBarS, (uint32_t)(i & 1), ab, 83);
-            if (ok && i + 2 < ntiles) {
-                load_pair(i + 2);
+            // the next tile's U MMAs queue up behind it: every thread has read columns 0-255 (the
+            // barrier above), and they touch the other pair of shared-memory tiles
+            if (k + 1 < n_my) ok = issue_u(k + 1);
+            // this pair may be overwritten once the dS MMA is done
+            if (ok) ok = wait_bar(bars + 8 * kCBarS, (uint32_t)(k & 1), ab, 83);
+            if (ok && k + 2 < n_my) {
+                load_pair(k + 2);
                 ++loads_issued;
             }
         }
-    }
-
-    // ---- epilogue: dS row d_k = tid -> this chunk's partial
-    if (ntiles > 0 && wait_bar(bars + 8 * kCBarS, (uint32_t)((ntiles - 1) & 1), ab, 84)) {
-        tc_fence_after();
-        float* dst = p.partials + ((((size_t)b * H + h) * p.nsplit + split) * kTile + tid) * kTile;
+        if (seg_last) {
+            // ---- this head's share of dS (row d_k = tid) -> its slot of the partial sums
+            if (!wait_bar(bars + 8 * kCBarS, (uint32_t)(k & 1), ab, 84)) break;
+            tc_fence_after();
+            const int part = (int)blockIdx.x - (bh * p.ntile) / p.share;
+            float* dst = p.partials + (((size_t)bh * p.nslot + part) * kTile + tid) * kTile;
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-            uint32_t o[32];
-            tmem_ld32(lane_base + 2 * kTile + c * 32, o);
-            tmem_wait_ld();
+            for (int c = 0; c < 4; ++c) {
+                uint32_t o[32];
+                tmem_ld32(lane_base + 2 * kTile + c * 32, o);
+                tmem_wait_ld();
 #pragma unroll
-            for (int e = 0; e < 8; ++e)
-                *reinterpret_cast<uint4*>(dst + c * 32 + e * 4) = make_uint4(o[e * 4], o[e * 4 + 1], o[e * 4 + 2], o[e * 4 + 3]);
+                for (int e = 0; e < 4; ++e)   // 32-byte stores: whole sectors
+                    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + c * 32 + e * 8),
+                                 "r"(o[e * 8]), "r"(o[e * 8 + 1]), "r"(o[e * 8 + 2]), "r"(o[e * 8 + 3]), "r"(o[e * 8 + 4]),
+                                 "r"(o[e * 8 + 5]), "r"(o[e * 8 + 6]), "r"(o[e * 8 + 7])
+                                 : "memory");
+            }
+            tc_fence_before();
         }
     }
+
     if (tid == 0 && (!ok || *abort_flag)) {
         // leave no bulk copy in flight into this CTA's shared memory
-        drain_bar(bars + 8 * kCBarW, 0);
+        if (w_loads > 0) drain_bar(bars + 8 * kCBarW, (w_loads - 1) & 1);
         for (int m = (loads_issued > 2 ? loads_issued - 2 : 0); m < loads_issued; ++m)
             drain_bar(bars + 8 * (kCBarFull0 + (m & 1)), (uint32_t)((m >> 1) & 1));
     }
@@ -1147,32 +1194,6 @@ struct TcTokenParams {
     int ntile;                 // 128-token tiles; rows_pad = 128 * ntile
     int nchunk;                // ceil(L / 64): chunks the scan walks
 };
-
-__device__ __forceinline__ void store_row_bf16_swizzled(uint8_t* tile, int r, const uint32_t (&x)[128], float f)
-{
-#pragma unroll
-    for (int c = 0; c < 16; ++c) {
-        uint4 v;
-        v.x = pack_bf16(__uint_as_float(x[c * 8 + 0]) * f, __uint_as_float(x[c * 8 + 1]) * f);
-        v.y = pack_bf16(__uint_as_float(x[c * 8 + 2]) * f, __uint_as_float(x[c * 8 + 3]) * f);
-        v.z = pack_bf16(__uint_as_float(x[c * 8 + 4]) * f, __uint_as_float(x[c * 8 + 5]) * f);
-        v.w = pack_bf16(__uint_as_float(x[c * 8 + 6]) * f, __uint_as_float(x[c * 8 + 7]) * f);
-        const int off = (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
-        *reinterpret_cast<uint4*>(tile + off) = v;
-    }
-}
-__device__ __forceinline__ void store_row_bf16_global(__nv_bfloat16* dst, const uint32_t (&x)[128], float f)
-{
-#pragma unroll
-    for (int c = 0; c < 16; ++c) {
-        uint4 v;
-        v.x = pack_bf16(__uint_as_float(x[c * 8 + 0]) * f, __uint_as_float(x[c * 8 + 1]) * f);
-        v.y = pack_bf16(__uint_as_float(x[c * 8 + 2]) * f, __uint_as_float(x[c * 8 + 3]) * f);
-        v.z = pack_bf16(__uint_as_float(x[c * 8 + 4]) * f, __uint_as_float(x[c * 8 + 5]) * f);
-        v.w = pack_bf16(__uint_as_float(x[c * 8 + 6]) * f, __uint_as_float(x[c * 8 + 7]) * f);
-        *reinterpret_cast<uint4*>(dst + c * 8) = v;
-    }
-}
 
 __global__ void __launch_bounds__(128, 1)
 tc_token_prepare_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -1898,8 +1919,28 @@ int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat
     p.beta = a.beta;
     p.partials = a.partials;
     p.status = a.status;
-    p.nsplit = a.nsplit;
-    dim3 grid(a.nsplit, a.s.H, a.s.B);
+    static int num_sms = 0;
+    if (num_sms == 0) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0) {
+            num_sms = 0;
+            set_error("cannot read the SM count");
+            return ARL2_ERR_CUDA;
+        }
+    }
+    // equal runs of the flattened tile sequence, at least 4 tiles each (a head then has at most
+    // ceil(ntile / 4) + 1 partial sums, which is what the workspace holds)
+    p.ntile = (a.s.L + kTile - 1) / kTile;
+    p.total_tiles = a.s.B * a.s.H * p.ntile;
+    p.share = (p.total_tiles + num_sms - 1) / num_sms;
+    if (p.share < 4) p.share = 4;
+    p.nslot = a.nsplit + 1;
+    if ((p.ntile + p.share - 1) / p.share + 1 > p.nslot) {
+        set_error("tc_commit: partial-sum slots (%d) do not cover %d tiles in runs of %d", p.nslot, p.ntile, p.share);
+        return ARL2_ERR_WORKSPACE;
+    }
+    const unsigned grid = (unsigned)((p.total_tiles + p.share - 1) / p.share);
     if (a.mode == 1)
         tc_commit_kernel<1><<<grid, kCommitThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, tm_wv, tm_s, p);
     else if (a.mode == 2)
@@ -1908,7 +1949,11 @@ int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat
         tc_commit_kernel<0><<<grid, kCommitThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, tm_wv, tm_s, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_error("launch of tc_commit_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
-    int m = commit_reduce(a, st);
+    CommitArgs ra = a;
+    ra.run_share = p.share;
+    ra.run_ntile = p.ntile;
+    ra.nslot = p.nslot;
+    int m = commit_reduce(ra, st);
     if (m < 0) return m;
     return 1 + m;
 }
