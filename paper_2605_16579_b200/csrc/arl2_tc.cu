@@ -837,8 +837,8 @@ constexpr int kCOffWv = kTileBytes;
 constexpr int kCOffPair = 2 * kTileBytes;                  // 2 pairs of (K tile, V tile)
 constexpr int kCOffState = kCOffPair + 4 * kTileBytes;     // bf16 copy of S_old (delta rule only)
 constexpr int kCOffBars = kCOffState + kTileBytes;
-constexpr int kCommitSmemBytes = kCOffBars + 128 + 1024;
-constexpr int kCommitThreads = 128;
+constexpr int kCommitSmemBytes = kCOffBars + 128 + 1024 + 1024;   // barriers, row-norm exchange, alignment slack
+constexpr int kCommitThreads = 256;
 
 enum CBar : int { kCBarW = 0, kCBarFull0, kCBarFull1, kCBarU, kCBarS, kCBarP, kCNumBars };
 
@@ -869,6 +869,19 @@ __device__ __forceinline__ void store_row_bf16_swizzled(uint8_t* tile, int r, co
         v.w = pack_bf16(__uint_as_float(x[c * 8 + 6]) * f, __uint_as_float(x[c * 8 + 7]) * f);
         const int off = (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
         *reinterpret_cast<uint4*>(tile + off) = v;
+    }
+}
+// my half (64 columns = one 64-column box) of row r
+__device__ __forceinline__ void store_half_row_bf16_swizzled(uint8_t* tile, int r, int half, const uint32_t (&x)[64], float f)
+{
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        uint4 v;
+        v.x = pack_bf16(__uint_as_float(x[c * 8 + 0]) * f, __uint_as_float(x[c * 8 + 1]) * f);
+        v.y = pack_bf16(__uint_as_float(x[c * 8 + 2]) * f, __uint_as_float(x[c * 8 + 3]) * f);
+        v.z = pack_bf16(__uint_as_float(x[c * 8 + 4]) * f, __uint_as_float(x[c * 8 + 5]) * f);
+        v.w = pack_bf16(__uint_as_float(x[c * 8 + 6]) * f, __uint_as_float(x[c * 8 + 7]) * f);
+        *reinterpret_cast<uint4*>(tile + half * kHalfBytes + r * 128 + ((c ^ (r & 7)) << 4)) = v;
     }
 }
 __device__ __forceinline__ void store_row_bf16_global(__nv_bfloat16* dst, const uint32_t (&x)[128], float f)
@@ -919,7 +932,11 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+    // two threads per token row (warps w and w + 4 own the same TMEM lanes), 64 columns each
+    const int r = (warp & 3) * 32 + (tid & 31);
+    const int chalf = warp >> 2;
+    const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(chalf * 64);
+    float* ssx = reinterpret_cast<float*>(smem + kCOffBars + 128);   // [2][128] partial sums of squares
 
     auto load_pair = [&](int k) {   // k-th tile of the run into pair k & 1
         const int g = g_begin + k, bh = g / p.ntile, tl = g - bh * p.ntile;
@@ -993,7 +1010,7 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         ok = issue_u(0);
     }
 
-    uint32_t sreg[128];
+    uint32_t sreg[64];
     for (int k = 0; k < n_my; ++k) {
         const int g = g_begin + k, bh = g / p.ntile, tl = g - bh * p.ntile;
         const int b = bh / H, h = bh - b * H;
@@ -1011,21 +1028,19 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             ++w_loads;
         }
 
-        const int r = tid;                       // token row of the tile
-        const int row = tl * kTile + r;
-        // ---- K' = L2Norm(RoPE(U_k))
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-            tmem_ld32(lane_base + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
+        const int row = tl * kTile + r;          // this thread's token
+        // ---- K' = L2Norm(RoPE(U_k)): my 64 columns of the row
+        tmem_ld32(lane_base, *reinterpret_cast<uint32_t(*)[32]>(&sreg[0]));
+        tmem_ld32(lane_base + 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[32]));
         tmem_wait_ld();
         if (p.rope_h != nullptr) {
             // rows of the warp-interleaved table: padding rows past L read as zero
-            const uint4* tab = p.rope_h + ((size_t)(row >> 5) * 16) * 32 + (row & 31);
-            uint4 cs[16];
+            const uint4* tab = p.rope_h + ((size_t)(row >> 5) * 16 + chalf * 8) * 32 + (row & 31);
+            uint4 cs[8];
 #pragma unroll
-            for (int c = 0; c < 16; ++c) cs[c] = __ldg(tab + c * 32);
+            for (int c = 0; c < 8; ++c) cs[c] = __ldg(tab + c * 32);
 #pragma unroll
-            for (int c = 0; c < 16; ++c) {
+            for (int c = 0; c < 8; ++c) {
                 const uint32_t h2[4] = {cs[c].x, cs[c].y, cs[c].z, cs[c].w};
 #pragma unroll
                 for (int m = 0; m < 4; ++m) {
@@ -1041,13 +1056,16 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         {
             float ss4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-            for (int c = 0; c < 128; c += 4) {
+            for (int c = 0; c < 64; c += 4) {
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
                     ss4[q] = fmaf(__uint_as_float(sreg[c + q]), __uint_as_float(sreg[c + q]), ss4[q]);
             }
-            const float f = rsqrtf((ss4[0] + ss4[1]) + (ss4[2] + ss4[3]) + p.s.eps);
-            store_row_bf16_swizzled(pair, r, sreg, f);
+            ssx[chalf * kTile + r] = (ss4[0] + ss4[1]) + (ss4[2] + ss4[3]);
+            __syncthreads();   // the other half of the row has posted its sum (slots are rewritten
+                               // only after the next barrier of this loop)
+            const float f = rsqrtf(ssx[r] + ssx[kTile + r] + p.s.eps);
+            store_half_row_bf16_swizzled(pair, r, chalf, sreg, f);
         }
         if (kMode == 1) {
             // ---- prediction K' S_old                                                   (Eq. 4)
@@ -1074,9 +1092,8 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             }
         }
         // ---- V' = U_v, or R = beta (V' - K' S_old), or w V'
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-            tmem_ld32(lane_base + kTile + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
+        tmem_ld32(lane_base + kTile, *reinterpret_cast<uint32_t(*)[32]>(&sreg[0]));
+        tmem_ld32(lane_base + kTile + 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[32]));
         tmem_wait_ld();
         float vscale = 1.0f;
         if (kMode == 2)
@@ -1085,7 +1102,7 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         if (kMode == 1) {
             if (p.beta != nullptr) vscale = row < L ? sigmoid_fast(__ldg(p.beta + ((size_t)b * L + row) * H + h)) : 0.0f;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < 2; ++c) {
                 uint32_t pr[32];
                 tmem_ld32(lane_base + 3 * kTile + c * 32, pr);
                 tmem_wait_ld();
@@ -1094,7 +1111,7 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     sreg[c * 32 + e] = __float_as_uint(__uint_as_float(sreg[c * 32 + e]) - __uint_as_float(pr[e]));
             }
         }
-        store_row_bf16_swizzled(pair + kTileBytes, r, sreg, vscale);
+        store_half_row_bf16_swizzled(pair + kTileBytes, r, chalf, sreg, vscale);
         fence_proxy_async_smem();
         tc_fence_before();
         __syncthreads();
@@ -1123,9 +1140,9 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             if (!wait_bar(bars + 8 * kCBarS, (uint32_t)(k & 1), ab, 84)) break;
             tc_fence_after();
             const int part = (int)blockIdx.x - (bh * p.ntile) / p.share;
-            float* dst = p.partials + (((size_t)bh * p.nslot + part) * kTile + tid) * kTile;
+            float* dst = p.partials + (((size_t)bh * p.nslot + part) * kTile + r) * kTile + chalf * 64;
 #pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < 2; ++c) {
                 uint32_t o[32];
                 tmem_ld32(lane_base + 2 * kTile + c * 32, o);
                 tmem_wait_ld();
