@@ -71,8 +71,9 @@ typedef struct {
 /*
  * Bytes of device scratch a context of this shape needs (256-byte aligned base).  It
  * holds a status word, the rotated copy of K made once per step, tensor-core operand
- * copies of S and of the feature maps, and the partial sums of the commit reduction.
- * Returns 0 for an invalid configuration.
+ * copies of S and of the feature maps, the packed rotation table, the partial sums of the
+ * commit reduction, the per-token decay weights and, with ARL2_FLAG_TOKEN_GATES, the chunk
+ * factors of arl2_commit_tokens.  Returns 0 for an invalid configuration.
  */
 size_t arl2_workspace_bytes(const arl2_config* cfg);
 
