@@ -110,9 +110,12 @@ void arl2_oracle_feature(int B, int H, int L, int D, const double *x, const doub
  *   O_inter = Q'_i S                                            (Eq. 5 / Eq. 8)
  *   O_i     = O_intra + sigmoid(g_i) * O_inter                  (Eq. 6-7, Algorithm 1)
  * S is read, never written (clean-pass-only update, Sec. 3.3).
+ * gate_mode selects the granularity of the combine gate (the paper's layer is headwise; the other
+ * two are the variants of its gate ablation): 0 headwise g [B, L, H]; 1 scalar g [B, L], one gate
+ * per token shared by all heads; 2 elementwise g [B, L, H, D], one gate per output channel.
  * scratch: at least L + 3*D doubles.
  */
-static void step_row(int b, int h, int i, int H, int L, int D,
+static void step_row(int b, int h, int i, int H, int L, int D, int gate_mode,
                      const double *q, const double *k, const double *v, const double *g,
                      const double *S, const double *wq,
                      const double *rope_cos, const double *rope_sin,
@@ -153,8 +156,11 @@ static void step_row(int b, int h, int i, int H, int L, int D,
     rope(qf, D, rope_cos, rope_sin, i);
     l2norm(qf, D, eps);
     const double *Sh = S + ((size_t)b * H + h) * D * D;
-    double gate = sigmoid(g[((size_t)b * L + i) * H + h]);
     for (int e = 0; e < D; ++e) {
+        size_t gi = gate_mode == 1 ? (size_t)b * L + i
+                  : gate_mode == 2 ? (((size_t)b * L + i) * H + h) * D + e
+                                   : ((size_t)b * L + i) * H + h;
+        double gate = sigmoid(g[gi]);
         double acc = 0.0;
         for (int d = 0; d < D; ++d) acc += qf[d] * Sh[(size_t)d * D + e];
         o[e] += gate * acc;
@@ -177,7 +183,30 @@ void arl2_oracle_step(int B, int H, int L, int D,
             int i = (int)(t % L);
             int h = (int)((t / L) % H);
             int b = (int)(t / ((long)L * H));
-            step_row(b, h, i, H, L, D, q, k, v, g, S, wq, rope_cos, rope_sin, scale, eps,
+            step_row(b, h, i, H, L, D, 0, q, k, v, g, S, wq, rope_cos, rope_sin, scale, eps,
+                     out + (((size_t)b * L + i) * H + h) * D, scratch);
+        }
+        free(scratch);
+    }
+}
+
+/* The same with the combine gate at another granularity (see step_row): the gate ablation's variants. */
+void arl2_oracle_step_gate_mode(int B, int H, int L, int D, int gate_mode,
+                                const double *q, const double *k, const double *v, const double *g,
+                                const double *S, const double *wq,
+                                const double *rope_cos, const double *rope_sin,
+                                double scale, double eps, double *out)
+{
+    long total = (long)B * H * L;
+#pragma omp parallel
+    {
+        double *scratch = (double *)malloc(sizeof(double) * ((size_t)L + 3 * (size_t)D));
+#pragma omp for schedule(dynamic, 16)
+        for (long t = 0; t < total; ++t) {
+            int i = (int)(t % L);
+            int h = (int)((t / L) % H);
+            int b = (int)(t / ((long)L * H));
+            step_row(b, h, i, H, L, D, gate_mode, q, k, v, g, S, wq, rope_cos, rope_sin, scale, eps,
                      out + (((size_t)b * L + i) * H + h) * D, scratch);
         }
         free(scratch);
@@ -201,7 +230,7 @@ void arl2_oracle_step_rows(int B, int H, int L, int D,
         double *scratch = (double *)malloc(sizeof(double) * ((size_t)L + 3 * (size_t)D));
 #pragma omp for schedule(dynamic, 4)
         for (int t = 0; t < n; ++t)
-            step_row(bs[t], hs[t], is[t], H, L, D, q, k, v, g, S, wq, rope_cos, rope_sin,
+            step_row(bs[t], hs[t], is[t], H, L, D, 0, q, k, v, g, S, wq, rope_cos, rope_sin,
                      scale, eps, out_rows + (size_t)t * D, scratch);
         free(scratch);
     }

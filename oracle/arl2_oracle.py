@@ -96,6 +96,23 @@ def step(q, k, v, g, S, wq=None, rope_cos=None, rope_sin=None, scale=None, eps=1
     return out
 
 
+def step_gate_mode(q, k, v, g, S, gate_mode, wq=None, rope_cos=None, rope_sin=None, scale=None, eps=1e-6):
+    """The layer with the combine gate at another granularity: gate_mode 0 headwise g [B, L, H],
+    1 scalar g [B, L], 2 elementwise g [B, L, H, D]."""
+    q, k, v, g, S = _f64(q), _f64(k), _f64(v), _f64(g), _f64(S)
+    wq, rope_cos, rope_sin = _f64(wq), _f64(rope_cos), _f64(rope_sin)
+    B, L, H, D = q.shape
+    assert g.shape == {0: (B, L, H), 1: (B, L), 2: (B, L, H, D)}[gate_mode]
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    out = np.empty_like(q)
+    _load().arl2_oracle_step_gate_mode(
+        B, H, L, D, gate_mode, _p(q), _p(k), _p(v), _p(g), _p(S), _p(wq), _p(rope_cos), _p(rope_sin),
+        ctypes.c_double(scale), ctypes.c_double(eps), _p(out),
+    )
+    return out
+
+
 def step_rows(q, k, v, g, S, rows, wq=None, rope_cos=None, rope_sin=None, scale=None,
               eps=1e-6):
     """Outputs of the sampled (b, h, i) triples in ``rows`` ([n, 3] ints): returns [n, D]."""

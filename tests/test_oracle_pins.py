@@ -344,6 +344,28 @@ def sig(x):
     return 1.0 / (1.0 + np.exp(-x))
 
 
+def test_gate_granularities(oracle):
+    """Scalar and elementwise combine gates: with the same logit repeated they are the headwise
+    layer; an elementwise gate closed on some channels leaves exactly the intra branch there and
+    the fully open layer elsewhere."""
+    B, L, H, D = 2, 6, 3, 8
+    q, k, v, S = rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, H, D, D)
+    cos, sin = tables(L, D)
+    g_tok = rnd(B, L)
+    head = oracle.step(q, k, v, np.repeat(g_tok[..., None], H, axis=2), S, None, cos, sin)
+    np.testing.assert_allclose(oracle.step_gate_mode(q, k, v, g_tok, S, 1, None, cos, sin), head, rtol=1e-13)
+    g_head = rnd(B, L, H)
+    ref = oracle.step(q, k, v, g_head, S, None, cos, sin)
+    elem = oracle.step_gate_mode(q, k, v, np.repeat(g_head[..., None], D, axis=3), S, 2, None, cos, sin)
+    np.testing.assert_allclose(elem, ref, rtol=1e-13)
+    np.testing.assert_allclose(oracle.step_gate_mode(q, k, v, g_head, S, 0, None, cos, sin), ref, rtol=0)
+    closed = oracle.step(q, k, v, np.full((B, L, H), -800.0), S, None, cos, sin)
+    opened = oracle.step(q, k, v, np.full((B, L, H), 800.0), S, None, cos, sin)
+    mask = np.random.default_rng(5).random((B, L, H, D)) < 0.5
+    mixed = oracle.step_gate_mode(q, k, v, np.where(mask, 800.0, -800.0), S, 2, None, cos, sin)
+    np.testing.assert_allclose(mixed, np.where(mask, opened, closed), rtol=1e-13, atol=1e-15)
+
+
 def test_cache_attention_against_library_and_the_layer(oracle):
     """Eq. 1 over a longer cache: the library's attention routine; with a cache of exactly the
     block and a closed gate it is the layer's intra branch without rotation; a cache of one token
