@@ -52,6 +52,10 @@ typedef enum {
 
 /* arl2_config.flags */
 #define ARL2_FLAG_FORCE_SIMT 1u /* bf16 I/O through the plain-FMA kernels (debug / A-B checks) */
+/* Granularity of the combine gate of arl2_denoise_step (Eq. 6-7 take one gate per token and head;
+   the other two are the variants of the paper's gate ablation, offered for comparison):          */
+#define ARL2_FLAG_GATE_SCALAR 4u      /* d_gate_logits is [B, L]: one gate per token, all heads     */
+#define ARL2_FLAG_GATE_ELEMENTWISE 8u /* d_gate_logits is [B, L, H, D]: one gate per output channel */
 #define ARL2_FLAG_TOKEN_GATES 2u /* reserve workspace for arl2_commit_tokens (3 fp32 copies of a
                                     [B, H, ceil(L/64)*64, D] tensor)                             */
 
@@ -109,8 +113,9 @@ int arl2_set_params(arl2_ctx* ctx, const void* d_wphi_q, const void* d_wphi_k,
  *                    + sigmoid(g[b,i,h]) * L2Norm(RoPE(q_i Wphi_q[h])) S[b,h]
  * READS the state, never writes it (clean-pass-only update, Sec. 3.3): S is bitwise
  * unchanged after any number of calls.  d_q, d_k, d_v, d_out: [B, L, H, D] io_dtype;
- * d_gate_logits: [B, L, H] fp32 (the projection x W_g of Eq. 6).  d_out must not
- * alias an input.
+ * d_gate_logits: [B, L, H] fp32 (the projection x W_g of Eq. 6), or [B, L] / [B, L, H, D] when
+ * the context was created with ARL2_FLAG_GATE_SCALAR / ARL2_FLAG_GATE_ELEMENTWISE.  d_out must
+ * not alias an input.
  */
 int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const void* d_v,
                       const float* d_gate_logits, void* d_out, void* stream);

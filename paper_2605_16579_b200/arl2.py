@@ -18,6 +18,8 @@ LIB_PATH = os.path.join(_PKG, "libarl2.so")
 ARL2_BF16, ARL2_FP32 = 0, 1
 ARL2_FLAG_FORCE_SIMT = 1
 ARL2_FLAG_TOKEN_GATES = 2
+ARL2_FLAG_GATE_SCALAR = 4
+ARL2_FLAG_GATE_ELEMENTWISE = 8
 
 EXPORTS = (
     "arl2_workspace_bytes", "arl2_create", "arl2_set_params", "arl2_denoise_step", "arl2_commit",
@@ -142,6 +144,7 @@ class Layer:
         lib = load()
         self.cfg = make_config(B, H, L, D, dtype, softmax_scale, l2_eps, 0, flags)
         self.B, self.H, self.L, self.D = B, H, L, D
+        self.flags = flags
         self.device = torch.device(device)
         self.dtype = torch.bfloat16 if self.cfg.io_dtype == ARL2_BF16 else torch.float32
         self.workspace_bytes = arl2_workspace_bytes(self.cfg)
@@ -174,7 +177,10 @@ class Layer:
         shape = (self.B, self.L, self.H, self.D)
         for t in (q, k, v):
             self._want(t, shape, self.dtype, "q/k/v")
-        self._want(gate_logits, (self.B, self.L, self.H), torch.float32, "gate_logits")
+        gshape = ((self.B, self.L) if self.flags & ARL2_FLAG_GATE_SCALAR else
+                  (self.B, self.L, self.H, self.D) if self.flags & ARL2_FLAG_GATE_ELEMENTWISE else
+                  (self.B, self.L, self.H))
+        self._want(gate_logits, gshape, torch.float32, "gate_logits")
         if out is None:
             out = torch.empty(shape, dtype=self.dtype, device=self.device)
         else:

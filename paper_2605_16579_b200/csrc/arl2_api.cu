@@ -52,6 +52,10 @@ bool valid_config(const arl2_config* c)
         set_error("io_dtype must be ARL2_BF16 or ARL2_FP32 (got %d)", c->io_dtype);
         return false;
     }
+    if ((c->flags & ARL2_FLAG_GATE_SCALAR) && (c->flags & ARL2_FLAG_GATE_ELEMENTWISE)) {
+        set_error("ARL2_FLAG_GATE_SCALAR and ARL2_FLAG_GATE_ELEMENTWISE exclude each other");
+        return false;
+    }
     if (c->commit_rule != 0) {
         set_error("commit_rule %d is reserved; only 0 (gated linear) is built", c->commit_rule);
         return false;
@@ -275,6 +279,7 @@ int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const voi
     StepArgs a;
     a.s = ctx->shape;
     a.q = d_q; a.k_rot = k_rot; a.v = d_v; a.gate = d_gate_logits;
+    a.gate_mode = (ctx->cfg.flags & ARL2_FLAG_GATE_ELEMENTWISE) ? 2 : (ctx->cfg.flags & ARL2_FLAG_GATE_SCALAR) ? 1 : 0;
     a.state = ctx->state; a.wq = ctx->wq;
     a.rope_cos = ctx->rope_cos; a.rope_sin = ctx->rope_sin;
     a.out = d_out;

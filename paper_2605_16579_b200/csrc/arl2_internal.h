@@ -42,6 +42,7 @@ struct StepArgs {
     int launch_parity;      // step launches so far on this context, mod 2 (scheduler counters)
     const void* rope_h;     // [L, D/2] half2 (cos, sin) copy of the tables (tensor-core path), or nullptr
     int Lk = 0;             // > 0: K and V hold Lk tokens (a cache), [B, Lk, H, D]; 0: L
+    int gate_mode = 0;      // 0: gate [B, L, H]; 1: [B, L]; 2: [B, L, H, D]
 };
 
 struct CommitArgs {

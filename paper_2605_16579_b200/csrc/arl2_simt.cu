@@ -314,13 +314,18 @@ __global__ void __launch_bounds__(NT) simt_step_kernel(StepArgs a)
     for (int i = 0; i < 4; ++i) {
         int row = i0 + ty * 4 + i;
         if (row >= L) continue;
-        float gate = sigmoidf_(a.gate[((size_t)b * L + row) * H + h]);
+        // combine gate: one per (token, head), one per token, or one per output channel
+        const size_t rh = ((size_t)b * L + row) * H + h;
+        float gate = a.gate_mode == 2 ? 0.0f : sigmoidf_(a.gate[a.gate_mode == 1 ? (size_t)b * L + row : rh]);
         float inv = 1.0f / lrun[i];
 #pragma unroll
         for (int c = 0; c < D / 64; ++c) {
-            T* p = out + (((size_t)b * L + row) * H + h) * D + c * 64 + tx * 4;
+            T* p = out + rh * D + c * 64 + tx * 4;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) from_f(p[e], o[i][c * 4 + e] * inv + gate * x[i][c * 4 + e]);
+            for (int e = 0; e < 4; ++e) {
+                if (a.gate_mode == 2) gate = sigmoidf_(a.gate[rh * D + c * 64 + tx * 4 + e]);
+                from_f(p[e], o[i][c * 4 + e] * inv + gate * x[i][c * 4 + e]);
+            }
         }
     }
 }

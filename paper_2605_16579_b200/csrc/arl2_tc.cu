@@ -84,6 +84,7 @@ struct TcStepParams {
     uint32_t* status;
     uint32_t* sched_counter;   // this launch's item counter (zero on entry)
     uint32_t* sched_next;      // the next launch's counter: cleared by this launch
+    int gate_mode;             // 0: gate logits [B, L, H]; 1: [B, L] (one per token); 2: [B, L, H, D] (per channel)
     int Lk;                    // keys per head: L, or the length of a key/value cache (Eq. 1)
     int n_q;                   // query tiles per head
     int n_kv;                  // key tiles per head
@@ -277,7 +278,9 @@ __device__ __forceinline__ Entry item_entry(const Item& it, int n_kv, int e)
     return en;
 }
 
-// One softmax group thread: owns query row `r` of tile `t` of every item.
+// One softmax group thread: owns query row `r` of tile `t` of every item.  kElemGate compiles the
+// per-channel gate variant in (a separate kernel instantiation, so the default path is unchanged).
+template <bool kElemGate>
 __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* smem, uint32_t bars,
                                              uint32_t tmem_base, const Abort& ab,
                                              const volatile int* item_slots, int t, int r,
@@ -454,7 +457,10 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
             // the row's rotation table is fetched while the MMA is still running
             uint4 cs[16];
             // fetched early too; no gate tensor = closed gate (plain softmax attention, Eq. 1)
-            const float gate_logit = (valid_row && p.gate != nullptr) ? __ldg(p.gate + ((size_t)b * L + row) * H + h) : -INFINITY;
+            const bool elem_gate = kElemGate && p.gate_mode == 2 && p.gate != nullptr;   // one gate per output channel
+            const float gate_logit = (valid_row && p.gate != nullptr && !elem_gate)
+                                         ? __ldg(p.gate + (p.gate_mode == 1 ? (size_t)b * L + row : ((size_t)b * L + row) * H + h))
+                                         : -INFINITY;
             const bool rotate_u = p.rope_h != nullptr && valid_row;
             if (rotate_u) {
                 const uint4* tab = p.rope_h + ((size_t)(row >> 5) * 16) * 32 + (row & 31);
@@ -495,8 +501,9 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                 }
                 const float ss = (ss4[0] + ss4[1]) + (ss4[2] + ss4[3]);
                 const float gate = valid_row ? sigmoid_fast(gate_logit) : 0.0f;
-                // scaled by the row sum so that the common 1/l of the epilogue leaves gate * Q' S
-                const float f = rsqrtf(ss + p.s.eps) * gate * l_sum;
+                // scaled by the row sum so that the common 1/l of the epilogue leaves gate * Q' S;
+                // with per-channel gates the readout is kept apart and gated in the epilogue
+                const float f = elem_gate ? rsqrtf(ss + p.s.eps) : rsqrtf(ss + p.s.eps) * gate * l_sum;
 #pragma unroll
                 for (int c = 0; c < 64; ++c)
                     sreg[c] = pack_bf16(__uint_as_float(sreg[2 * c]) * f, __uint_as_float(sreg[2 * c + 1]) * f);
@@ -507,6 +514,53 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
             tc_fence_before();
             mbar_arrive(bar_p);
 
+            if (elem_gate) {
+                // ---- per-channel gates: X = Q' S arrives 64 channels at a time in columns 64-127 of
+                // S_t; out = O_t / l + sigmoid(G) X.  O_t is final: its last MMA preceded U's.
+                const float inv_l = 1.0f / l_sum;
+                const size_t rbase = ((size_t)b * L + (valid_row ? row : 0)) * H + h;
+                __nv_bfloat16* orow = p.out + rbase * kTile;
+                const float* grow = p.gate + rbase * kTile;
+#pragma unroll 1
+                for (int hv = 0; hv < 2; ++hv) {
+                    if (!wait_bar(bar_s, s_cnt & 1, ab, 32 + t)) return;
+                    ++s_cnt;
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t x[32], o[32];
+                        tmem_ld32(s_addr + 64 + c * 32, x);
+                        tmem_ld32(o_addr + hv * 64 + c * 32, o);
+                        tmem_wait_ld();
+                        if (valid_row) {
+#pragma unroll
+                            for (int e = 0; e < 2; ++e) {
+                                uint32_t w[8];
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    const float4 gl = __ldg(reinterpret_cast<const float4*>(grow + hv * 64 + c * 32 + e * 16 + i * 4));
+                                    const float gv[4] = {gl.x, gl.y, gl.z, gl.w};
+                                    float y[4];
+#pragma unroll
+                                    for (int u = 0; u < 4; ++u) {
+                                        const int n = e * 16 + i * 4 + u;
+                                        y[u] = __uint_as_float(o[n]) * inv_l + sigmoid_fast(gv[u]) * __uint_as_float(x[n]);
+                                    }
+                                    w[i * 2] = pack_bf16(y[0], y[1]);
+                                    w[i * 2 + 1] = pack_bf16(y[2], y[3]);
+                                }
+                                asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(
+                                                 orow + hv * 64 + c * 32 + e * 16),
+                                             "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                                             : "memory");
+                            }
+                        }
+                    }
+                    tc_fence_before();
+                    if (hv == 0) mbar_arrive(bar_p);   // the first half of X has been read
+                }
+                continue;
+            }
             // ---- epilogue: O_t / l -> bf16 -> global                              (Eq. 6-7)
             ARL2_ITER(true, 256 + item * 16 + t * 8 + 2);
             if (!wait_bar(bars + 8 * (kBarOFinal0 + t), of_cnt & 1, ab, 40 + t)) return;
@@ -542,6 +596,7 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
     }
 }
 
+template <bool kElemGate>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_w,
@@ -593,7 +648,7 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
     if (warp < 8) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
-        softmax_role(p, smem, bars, tmem_base, ab, item_slots, warp >> 2, (warp & 3) * 32 + lane, warp & 3);
+        softmax_role<kElemGate>(p, smem, bars, tmem_base, ab, item_slots, warp >> 2, (warp & 3) * 32 + lane, warp & 3);
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
     }
@@ -799,10 +854,32 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     ++p_cnt;
                     if (!ok) break;
                     tc_fence_after();
-                    issue_pv(slot_addr(e_s), true);
-                    release_mine(e_s, !shared);
-                    mma_commit(bars + 8 * (kBarOFinal0 + t));
-                    ++of_cnt;
+                    if (kElemGate && p.gate_mode == 2 && p.gate != nullptr) {
+                        // per-channel gates: X = Q' S kept apart from O_t, 64 channels at a time into
+                        // columns 64-127 of S_t (Q' sits in columns 0-63)
+                        constexpr uint32_t idesc_x = idesc_bf16(kTile, 64, 0, 1);
+                        for (int hv = 0; hv < 2 && ok; ++hv) {
+                            if (hv == 1) {
+                                ok = wait_bar(bar_p, p_cnt & 1, ab, 72 + t);   // first half consumed
+                                ++p_cnt;
+                                if (!ok) break;
+                                tc_fence_after();
+                            }
+                            const uint32_t x_lo = ((slot_addr(e_s) + hv * kHalfBytes) >> 4) | kLboMN;
+#pragma unroll
+                            for (int ks = 0; ks < 8; ++ks)
+                                mma_ts(s_col + 64, s_col + ks * 8, desc64(x_lo + (uint32_t)(ks * (2048 >> 4))), idesc_x,
+                                       ks > 0 ? 1u : 0u);
+                            mma_commit(bar_s);
+                        }
+                        if (!ok) break;
+                        release_mine(e_s, !shared);
+                    } else {
+                        issue_pv(slot_addr(e_s), true);
+                        release_mine(e_s, !shared);
+                        mma_commit(bars + 8 * (kBarOFinal0 + t));
+                        ++of_cnt;
+                    }
                 }
                 cons += shared ? 1 : ntile;
             }
@@ -1865,7 +1942,9 @@ int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* 
             set_error("cannot read the SM count");
             return ARL2_ERR_CUDA;
         }
-        cudaError_t e = cudaFuncSetAttribute(tc_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(tc_step_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(tc_step_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) { set_error("cudaFuncSetAttribute(tc_step_kernel, %d): %s", kSmemBytes, cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
         attr_set = true;
     }
@@ -1880,6 +1959,7 @@ int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* 
     TcStepParams p;
     p.s = a.s;
     p.gate = a.gate;
+    p.gate_mode = a.gate_mode;
     p.rope_cos = a.rope_cos;
     p.rope_sin = a.rope_sin;
     p.rope_h = static_cast<const uint4*>(a.rope_h);
@@ -1895,7 +1975,10 @@ int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* 
     p.sched_counter = a.status + kStatusSched + (a.launch_parity & 1);
     p.sched_next = a.status + kStatusSched + ((a.launch_parity + 1) & 1);
     const int grid = p.n_items < num_sms ? p.n_items : num_sms;
-    tc_step_kernel<<<grid, kThreads, kSmemBytes, st>>>(tm_q, tm_k, tm_v, tm_w, tm_s, p);
+    if (p.gate_mode == 2 && p.gate != nullptr)
+        tc_step_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(tm_q, tm_k, tm_v, tm_w, tm_s, p);
+    else
+        tc_step_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(tm_q, tm_k, tm_v, tm_w, tm_s, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_error("launch of tc_step_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
     return 1;
