@@ -28,7 +28,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
     size_t status, k_rot, partials, state_bf16, wq_op, wk_op, wv_op, rope_h, dec_w, dec_total, tok_w, tok_u1, tok_kh, tok_gc, total;
-    int nsplit, nchunk;
+    int nsplit, nchunk, nslot;
 };
 
 bool valid_config(const arl2_config* c)
@@ -82,7 +82,17 @@ Layout make_layout(const arl2_config& c)
     size_t off = 0;
     l.status = off;     off += align_up(kStatusWords * sizeof(uint32_t));
     l.k_rot = off;      off += align_up(tensor);
-    l.partials = off;   off += align_up((size_t)c.B * c.H * (l.nsplit + 1) * dd * sizeof(float));
+    // partial-sum slots per (stream, head): the plain-FMA kernels use one per 512-token chunk; the
+    // tensor-core kernel one per run of tiles a head falls into, runs sized for a 148-SM device
+    // (with more SMs the launcher lengthens the runs to fit)
+    {
+        const long ntile = (c.L + 127) / 128, total = (long)c.B * c.H * ntile;
+        long share = (total + 147) / 148;
+        if (share < 2) share = 2;
+        const long tc_slots = (ntile + share - 1) / share + 1;
+        l.nslot = (int)(tc_slots > l.nsplit ? tc_slots : l.nsplit);
+    }
+    l.partials = off;   off += align_up((size_t)c.B * c.H * l.nslot * dd * sizeof(float));
     l.state_bf16 = off; off += align_up((size_t)c.B * c.H * dd * 2);
     l.wq_op = off;      off += align_up((size_t)c.H * dd * 2);
     l.wk_op = off;      off += align_up((size_t)c.H * dd * 2);
@@ -378,6 +388,7 @@ int commit_impl(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
     a.state_bf16 = ctx->use_tc ? reinterpret_cast<__nv_bfloat16*>(ctx->ws + ctx->lay.state_bf16)
                                : nullptr;
     a.nsplit = ctx->lay.nsplit;
+    a.nslot = ctx->lay.nslot;
     a.rope_h = (ctx->use_tc && ctx->rope_cos != nullptr) ? ctx->ws + ctx->lay.rope_h : nullptr;
     a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status);
     a.mode = mode;

@@ -2029,17 +2029,18 @@ int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat
             return ARL2_ERR_CUDA;
         }
     }
-    // equal runs of the flattened tile sequence, at least 4 tiles each (a head then has at most
-    // ceil(ntile / 4) + 1 partial sums, which is what the workspace holds)
+    // equal runs of the flattened tile sequence, at least 2 tiles each and long enough for a head's
+    // partial sums (one per run it falls into, at most ceil(ntile / share) + 1) to fit the slots
     p.ntile = (a.s.L + kTile - 1) / kTile;
     p.total_tiles = a.s.B * a.s.H * p.ntile;
     p.share = (p.total_tiles + num_sms - 1) / num_sms;
-    if (p.share < 4) p.share = 4;
-    p.nslot = a.nsplit + 1;
-    if ((p.ntile + p.share - 1) / p.share + 1 > p.nslot) {
-        set_error("tc_commit: partial-sum slots (%d) do not cover %d tiles in runs of %d", p.nslot, p.ntile, p.share);
+    if (p.share < 2) p.share = 2;
+    p.nslot = a.nslot;
+    if (p.nslot < 2) {
+        set_error("tc_commit: needs at least two partial-sum slots per head (got %d)", p.nslot);
         return ARL2_ERR_WORKSPACE;
     }
+    if ((p.ntile + p.share - 1) / p.share + 1 > p.nslot) p.share = (p.ntile + p.nslot - 2) / (p.nslot - 1);
     const unsigned grid = (unsigned)((p.total_tiles + p.share - 1) / p.share);
     if (a.mode == 1)
         tc_commit_kernel<1><<<grid, kCommitThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, tm_wv, tm_s, p);
