@@ -867,32 +867,57 @@ int launch_commit(const CommitArgs& a, cudaStream_t st)
 
 }  // namespace
 
-// Suffix products of the per-token forget gates of one (stream, head): each thread takes a
-// contiguous run of tokens, the runs are combined through shared memory, everything in log space.
+// Suffix products of the per-token forget gates of one (stream, head), in log space.  The block
+// walks the tokens from the end of the sequence in tiles of 256 x 8; inside a tile every thread owns
+// 8 consecutive tokens, the threads' sums are combined by a suffix scan (warp shuffles, then the 8
+// warp totals through shared memory), and `carry` holds the log-product of all later tiles.
 __global__ void __launch_bounds__(256) decay_weights_kernel(const float* __restrict__ alpha,
                                                             float* __restrict__ w, float* __restrict__ total,
                                                             int L, int H)
 {
-    __shared__ float seg_sum[256];
-    const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
-    const int seg = (L + 255) / 256;
-    const int l0 = min(L, tid * seg), l1 = min(L, l0 + seg);
-    auto log_alpha = [&](int l) {
-        const float x = alpha[((size_t)b * L + l) * H + h];
-        return x >= 0.0f ? -log1pf(expf(-x)) : x - log1pf(expf(x));
-    };
-    float s = 0.0f;
-    for (int l = l0; l < l1; ++l) s += log_alpha(l);
-    seg_sum[tid] = s;
-    __syncthreads();
-    float after = 0.0f;   // log of the product over every later run
-    for (int t = tid + 1; t < 256; ++t) after += seg_sum[t];
-    float run = after;
-    for (int l = l1 - 1; l >= l0; --l) {
-        w[((size_t)b * L + l) * H + h] = expf(run);
-        run += log_alpha(l);
+    constexpr int SEG = 8, TILE = 256 * SEG;
+    __shared__ float warp_tot[8];
+    const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const size_t base = (size_t)b * L * H + h;
+    float carry = 0.0f;
+    const int ntile = (L + TILE - 1) / TILE;
+    for (int tile = ntile - 1; tile >= 0; --tile) {
+        const int l0 = tile * TILE + tid * SEG;
+        float la[SEG];
+        float mine = 0.0f;
+#pragma unroll
+        for (int i = 0; i < SEG; ++i) {
+            float v = 0.0f;   // tokens past L: alpha = 1
+            if (l0 + i < L) {
+                const float x = alpha[base + (size_t)(l0 + i) * H];
+                v = x >= 0.0f ? -log1pf(expf(-x)) : x - log1pf(expf(x));
+            }
+            la[i] = v;
+            mine += v;
+        }
+        // exclusive suffix sum of `mine` over the threads of the block (later threads = later tokens)
+        float incl = mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const float dn = __shfl_down_sync(0xffffffffu, incl, off);
+            if (lane + off < 32) incl += dn;
+        }
+        if (lane == 0) warp_tot[wid] = incl;
+        __syncthreads();
+        float later_warps = 0.0f;
+        for (int q = wid + 1; q < 8; ++q) later_warps += warp_tot[q];
+        float tile_total = 0.0f;
+        for (int q = 0; q < 8; ++q) tile_total += warp_tot[q];
+        float run = carry + later_warps + (incl - mine);   // log-product of every token after mine
+#pragma unroll
+        for (int i = SEG - 1; i >= 0; --i) {
+            if (l0 + i < L) w[base + (size_t)(l0 + i) * H] = expf(run);
+            run += la[i];
+        }
+        carry += tile_total;
+        __syncthreads();   // warp_tot is rewritten by the next tile
     }
-    if (tid == 0) total[(size_t)b * H + h] = expf(run);   // run now covers every token
+    if (tid == 0) total[(size_t)b * H + h] = expf(carry);
 }
 
 int decay_weights(const Shape& s, const float* alpha_logits, float* w, float* total, cudaStream_t st)
