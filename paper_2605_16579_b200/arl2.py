@@ -140,7 +140,10 @@ class Layer:
     """
 
     def __init__(self, B, H, L, D, dtype="bf16", device="cuda:0", softmax_scale=0.0, l2_eps=0.0,
-                 flags=0):
+                 flags=0, state=None, workspace=None):
+        """``state`` ([B, H, D, D] fp32) and ``workspace`` (uint8, >= arl2_workspace_bytes, 256-byte
+        aligned) may be handed in by a caller that manages its own device memory; by default torch
+        allocates them here."""
         lib = load()
         self.cfg = make_config(B, H, L, D, dtype, softmax_scale, l2_eps, 0, flags)
         self.B, self.H, self.L, self.D = B, H, L, D
@@ -149,12 +152,18 @@ class Layer:
         self.dtype = torch.bfloat16 if self.cfg.io_dtype == ARL2_BF16 else torch.float32
         self.workspace_bytes = arl2_workspace_bytes(self.cfg)
         with torch.cuda.device(self.device):
-            self.state = torch.empty(B, H, D, D, dtype=torch.float32, device=self.device)
-            self.workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8,
-                                         device=self.device)
+            if state is None:
+                state = torch.empty(B, H, D, D, dtype=torch.float32, device=self.device)
+            if workspace is None:
+                workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=self.device)
+            self._want(state, (B, H, D, D), torch.float32, "state")
+            if not (workspace.is_cuda and workspace.dtype == torch.uint8 and workspace.is_contiguous()
+                    and workspace.numel() >= self.workspace_bytes):
+                raise Arl2Error(f"workspace: expected >= {self.workspace_bytes} contiguous CUDA bytes")
+            self.state, self.workspace = state, workspace
             ctx = ctypes.c_void_p()
             _check(lib.arl2_create(ctypes.byref(self.cfg), _ptr(self.state), _ptr(self.workspace),
-                                   self.workspace_bytes, _stream(), ctypes.byref(ctx)),
+                                   self.workspace.numel(), _stream(), ctypes.byref(ctx)),
                    "arl2_create")
         self._ctx = ctx
         self._params = None  # keeps the parameter tensors alive

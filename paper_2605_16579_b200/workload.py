@@ -149,27 +149,44 @@ def rope_tables(L: int, D: int, base: float = 10000.0):
     return ang.cos().float().contiguous(), ang.sin().float().contiguous()
 
 
-def sample_rows(cfg: Config, block: int, step: int, heads_per_stream: int = 2,
-                rows_per_head: int = 64, tile: int = 128):
-    """Seeded (b, h, i) triples for sampled parity at full size.
-
-    Per stream: head 0, the last head and random others up to ``heads_per_stream``; per
-    head: rows 0, tile-1, tile, the last row of the last full tile, every row of the ragged
-    tail tile (or the last 8 rows when L is a multiple of the tile) and random rows up to
-    ``rows_per_head``.
-    """
-    gen = _gen(cfg, block, step, salt=3)
+def sample_units(cfg: Config, heads_per_stream: int = 3):
+    """Seeded (b, h) pairs for parity at full size: per stream head 0, the last head and randomly
+    drawn heads from the middle of the grid, up to ``heads_per_stream`` (fixed for a whole run, so
+    that a checker can follow their states from the first block to the last)."""
+    gen = _gen(cfg, 0, 0, salt=4)
     out = []
     for b in range(cfg.B):
         heads = {0, cfg.H - 1}
         while len(heads) < min(heads_per_stream, cfg.H):
             heads.add(int(torch.randint(0, cfg.H, (1,), generator=gen)))
-        for h in sorted(heads):
-            full = (cfg.L // tile) * tile
-            rows = {0, min(tile - 1, cfg.L - 1), min(tile, cfg.L - 1), max(full - 1, 0)}
-            tail = range(full, cfg.L) if full < cfg.L else range(max(cfg.L - 8, 0), cfg.L)
-            rows.update(tail)
-            while len(rows) < min(rows_per_head + len(tail), cfg.L):
-                rows.add(int(torch.randint(0, cfg.L, (1,), generator=gen)))
-            out.extend((b, h, i) for i in sorted(rows))
+        out.extend((b, h) for h in sorted(heads))
+    return out
+
+
+def sample_rows(cfg: Config, block: int, step: int, heads_per_stream: int = 2,
+                rows_per_head: int = 64, tile: int = 128, units=None):
+    """Seeded (b, h, i) triples for sampled parity at full size.
+
+    Units: ``units`` if given, else per stream head 0, the last head and random others up to
+    ``heads_per_stream``; per unit: rows 0, tile-1, tile, the last row of the last full tile, every
+    row of the ragged tail tile (or the last 8 rows when L is a multiple of the tile) and random
+    rows up to ``rows_per_head``.
+    """
+    gen = _gen(cfg, block, step, salt=3)
+    if units is None:
+        units = []
+        for b in range(cfg.B):
+            heads = {0, cfg.H - 1}
+            while len(heads) < min(heads_per_stream, cfg.H):
+                heads.add(int(torch.randint(0, cfg.H, (1,), generator=gen)))
+            units.extend((b, h) for h in sorted(heads))
+    out = []
+    for b, h in units:
+        full = (cfg.L // tile) * tile
+        rows = {0, min(tile - 1, cfg.L - 1), min(tile, cfg.L - 1), max(full - 1, 0)}
+        tail = range(full, cfg.L) if full < cfg.L else range(max(cfg.L - 8, 0), cfg.L)
+        rows.update(tail)
+        while len(rows) < min(rows_per_head + len(tail), cfg.L):
+            rows.add(int(torch.randint(0, cfg.L, (1,), generator=gen)))
+        out.extend((b, h, i) for i in sorted(rows))
     return out

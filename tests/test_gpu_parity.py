@@ -12,36 +12,77 @@ from parity_util import Pair, head_errors
 pytestmark = pytest.mark.gpu
 
 
-def run_schedule(pair, blocks, steps, full=True, heads_per_stream=2, rows_per_head=64):
+CLOSED = -40.0   # combine-gate logit of a pass that compares the softmax branch alone
+
+
+def run_schedule(pair, blocks, steps, closed_gate_blocks=()):
+    """Every element of every pass and the whole state after every commit.  In the blocks listed in
+    closed_gate_blocks one more pass runs with the gate closed (the softmax branch on its own)."""
     cfg = pair.cfg
-    worst_o, worst_s = 0.0, 0.0
+    worst_o, worst_s, worst_c = 0.0, 0.0, 0.0
     for blk in range(blocks):
         for st in range(steps):
             q, k, v, g = workload.step_inputs(cfg, blk, st)
-            if full:
-                e = pair.step_full(q, k, v, g)
-            else:
-                rows = workload.sample_rows(cfg, blk, st, heads_per_stream, rows_per_head)
-                e = pair.step_sampled(q, k, v, g, rows)
+            e = pair.step_full(q, k, v, g)
             worst_o = max(worst_o, e)
             assert e <= pair.tol, f"block {blk} step {st}: output error {e:.3e} > {pair.tol}"
+            if blk in closed_gate_blocks and st == steps - 1:
+                e = pair.step_full(q, k, v, torch.full_like(g, CLOSED))
+                worst_c = max(worst_c, e)
+                assert e <= pair.tol, f"block {blk}: closed-gate output error {e:.3e} > {pair.tol}"
         kc, vc, a = workload.commit_inputs(cfg, blk)
-        heads = None
-        if not full:
-            heads = sorted({(b, h) for b, h, _ in workload.sample_rows(cfg, blk, 0, heads_per_stream, 1)})
-        e = pair.commit(kc, vc, a, heads)
+        e = pair.commit(kc, vc, a)
         worst_s = max(worst_s, e)
         assert e <= pair.tol, f"block {blk}: state error {e:.3e} > {pair.tol}"
     pair.layer.sync_status()
-    return worst_o, worst_s
+    return worst_o, worst_s, worst_c
+
+
+def run_horizon(pair, check_blocks, rows_per_head=32, reset_at=None):
+    """A configuration's whole schedule at full size.  The oracle follows the pair's units from the
+    first block to the last: their state is compared after EVERY commit; in check_blocks every pass
+    runs on fresh seeded inputs and is compared on sampled rows of those units (the ragged tail tile
+    in full), plus one pass with the gate closed; in the other blocks the passes run on a ring of
+    resident inputs (they cannot change the state, which a bitwise check confirms).
+    reset_at = (block, stream): that stream starts a new video there."""
+    cfg, d = pair.cfg, pair.dev
+    units = pair.units
+    ring = [tuple(t.to(d) for t in workload.step_inputs(cfg, 0, s)) for s in range(2)]
+    out = torch.empty(cfg.B, cfg.L, cfg.H, cfg.D, dtype=cfg.torch_dtype, device=d)
+    worst_o, worst_s, worst_c = 0.0, 0.0, 0.0
+    for blk in range(cfg.blocks):
+        if reset_at is not None and blk == reset_at[0]:
+            pair.reset(reset_at[1])
+        if blk in check_blocks:
+            for st in range(cfg.steps):
+                q, k, v, g = workload.step_inputs(cfg, blk, st)
+                rows = workload.sample_rows(cfg, blk, st, rows_per_head=rows_per_head, units=units)
+                e = pair.step_sampled(q, k, v, g, rows)
+                worst_o = max(worst_o, e)
+                assert e <= pair.tol, f"block {blk} step {st}: output error {e:.3e} > {pair.tol}"
+            e = pair.step_sampled(q, k, v, torch.full_like(g, CLOSED), rows)
+            worst_c = max(worst_c, e)
+            assert e <= pair.tol, f"block {blk}: closed-gate output error {e:.3e} > {pair.tol}"
+        else:
+            before = pair.layer.state.clone() if blk % 16 == 5 else None
+            for st in range(cfg.steps):
+                pair.layer.denoise_step(*ring[st % 2], out=out)
+            if before is not None:
+                assert torch.equal(before, pair.layer.state), "a denoise pass changed the state"
+        kc, vc, a = workload.commit_inputs(cfg, blk)
+        e = pair.commit(kc, vc, a)
+        worst_s = max(worst_s, e)
+        assert e <= pair.tol, f"block {blk}: state error {e:.3e} > {pair.tol}"
+    pair.layer.sync_status()
+    return worst_o, worst_s, worst_c
 
 
 def test_tiny_full_schedule_fp32(oracle):
     """Configuration 1 in full: 4 blocks x 2 steps + commit, fp32 mode, every element."""
     cfg = workload.CONFIGS["tiny"]
     pair = Pair(oracle, cfg)
-    o, s = run_schedule(pair, cfg.blocks, cfg.steps, full=True)
-    print(f"tiny: worst output error {o:.2e}, worst state error {s:.2e}")
+    o, s, c = run_schedule(pair, cfg.blocks, cfg.steps, closed_gate_blocks=(2,))
+    print(f"tiny: worst output error {o:.2e}, closed gate {c:.2e}, worst state error {s:.2e}")
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
@@ -50,7 +91,7 @@ def test_ragged_shapes(oracle, dtype, D, L):
     """Edge sizes: a single token, tails shorter and longer than a tile, several tiles."""
     cfg = workload.custom(B=2, H=3, D=D, L=L, dtype=dtype, cfg_id=11)
     pair = Pair(oracle, cfg)
-    run_schedule(pair, 2, 2, full=True)
+    run_schedule(pair, 2, 2, closed_gate_blocks=(1,))
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
@@ -59,21 +100,22 @@ def test_no_maps_no_rope(oracle, dtype):
     cfg = workload.custom(B=1, H=2, D=64, L=150, dtype=dtype, cfg_id=12)
     for rope, maps in ((False, False), (True, False), (False, True)):
         pair = Pair(oracle, cfg, rope=rope, maps=maps)
-        run_schedule(pair, 2, 1, full=True)
+        run_schedule(pair, 2, 1)
 
 
 def test_custom_scale_and_eps(oracle):
     cfg = workload.custom(B=1, H=2, D=64, L=100, dtype="fp32", cfg_id=13)
     pair = Pair(oracle, cfg, eps=1e-3, scale=0.05)
-    run_schedule(pair, 2, 2, full=True)
+    run_schedule(pair, 2, 2, closed_gate_blocks=(1,))
 
 
 def test_small_config_bf16(oracle):
-    """Configuration 2 (one 30x52 frame, H=12, D=128): two blocks in full, then sampled."""
+    """Configuration 2 (one 30x52 frame, H=12, D=128) in full: 8 blocks x 4 steps + commit, every
+    element of every pass and of the state after every commit."""
     cfg = workload.CONFIGS["small"]
     pair = Pair(oracle, cfg)
-    o, s = run_schedule(pair, 2, 2, full=True)
-    print(f"small: worst output error {o:.2e}, worst state error {s:.2e}")
+    o, s, c = run_schedule(pair, cfg.blocks, cfg.steps, closed_gate_blocks=(1, cfg.blocks - 1))
+    print(f"small: worst output error {o:.2e}, closed gate {c:.2e}, worst state error {s:.2e}")
 
 
 def test_step_never_writes_state(oracle):
@@ -176,18 +218,22 @@ def test_argument_errors_leave_state_untouched(oracle):
 
 
 @pytest.mark.parametrize("name", ["chunked", "batched", "long"])
-def test_full_size_configs_sampled(oracle, name):
-    """Configurations 3-5 at full size, in the launch configuration the bench times: sampled
-    rows of sampled heads per step (every row of the ragged tail tile included) and the whole
-    state of those heads after every commit."""
+def test_full_size_configs_whole_horizon(oracle, name):
+    """Configurations 3-5 at full size, in the launch configuration the bench times, over their whole
+    schedules (16 / 32 / 120 blocks x 4 steps + commit).  The oracle follows three (stream, head)
+    units per stream (head 0, the last head, one drawn from the middle of the grid): their state is
+    compared after every commit, their outputs on sampled rows (every row of the ragged tail tile
+    included) in the first, second, a middle and the last block.  On `batched`, stream 3 starts a new
+    video at block 16."""
     cfg = workload.CONFIGS[name]
-    pair = Pair(oracle, cfg)
-    o, s = run_schedule(pair, 2, 2, full=False, heads_per_stream=2, rows_per_head=32)
-    if name == "batched":  # per-stream reset in the middle of a run
-        pair.reset(3)
-        o2, s2 = run_schedule(pair, 1, 1, full=False, heads_per_stream=2, rows_per_head=16)
-        o, s = max(o, o2), max(s, s2)
-    print(f"{name}: worst sampled output error {o:.2e}, worst state error {s:.2e}")
+    units = workload.sample_units(cfg, heads_per_stream=3)
+    assert any(0 < h < cfg.H - 1 for _, h in units)
+    pair = Pair(oracle, cfg, units=units)
+    check = (0, 1, cfg.blocks // 2, cfg.blocks - 1)
+    o, s, c = run_horizon(pair, check, rows_per_head=24 if name == "batched" else 32,
+                          reset_at=(16, 3) if name == "batched" else None)
+    print(f"{name}: {cfg.blocks} blocks, {len(units)} units followed; worst sampled output error {o:.2e}, "
+          f"closed gate {c:.2e}, worst state error {s:.2e}")
 
 
 @pytest.mark.parametrize("B,H,L", [(1, 1, 100), (1, 3, 333), (3, 1, 200), (1, 5, 640)])
@@ -197,4 +243,4 @@ def test_odd_unit_counts_bf16(oracle, B, H, L):
     leaves none."""
     cfg = workload.custom(B=B, H=H, D=128, L=L, dtype="bf16", cfg_id=23)
     pair = Pair(oracle, cfg)
-    run_schedule(pair, 2, 2, full=True)
+    run_schedule(pair, 2, 2, closed_gate_blocks=(1,))

@@ -344,6 +344,29 @@ def sig(x):
     return 1.0 / (1.0 + np.exp(-x))
 
 
+def test_token_sequential_rule_decays_before_the_tokens(oracle):
+    """Rule 2 (decay once, then Eq. 4 token by token) with orthonormal keys and GENERAL alpha and
+    beta: the tokens do not interact, so S_new = alpha S_0 + sum_j beta_j K'_j^T (V'_j - alpha K'_j S_0),
+    i.e. K'_j S_new = alpha (1 - beta_j) K'_j S_0 + beta_j V'_j and directions no key spans are only
+    decayed.  A decay applied after the tokens, to the correction only, or not at all fails this."""
+    B, L, H, D = 2, 5, 2, 8
+    k, v = orthonormal_keys(B, L, H, D), rnd(B, L, H, D)
+    S0 = rnd(B, H, D, D)
+    a, bl = rnd(B, H), rnd(B, L, H)
+    got = oracle.commit(k, v, a, S0, eps=0.0, rule=2, beta_logit=bl)
+    alpha, beta = sig(a), sig(bl)
+    tk, tv, tS = torch.from_numpy(k), torch.from_numpy(v), torch.from_numpy(S0)
+    aS = torch.from_numpy(alpha)[..., None, None] * tS
+    resid = (tv - torch.einsum("blhd,bhde->blhe", tk, aS)) * torch.from_numpy(beta)[..., None]
+    ref = aS + torch.einsum("blhd,blhe->bhde", tk, resid)
+    np.testing.assert_allclose(got, ref.numpy(), rtol=1e-11, atol=1e-13)
+    read = torch.einsum("blhd,bhde->blhe", tk, torch.from_numpy(got)).numpy()
+    old = torch.einsum("blhd,bhde->blhe", tk, tS).numpy()
+    np.testing.assert_allclose(read, alpha[:, None, :, None] * (1 - beta[..., None]) * old + beta[..., None] * v,
+                               rtol=1e-10, atol=1e-12)
+    assert not np.allclose(got, oracle.commit(k, v, np.full((B, H), 800.0), S0, eps=0.0, rule=2, beta_logit=bl))
+
+
 def test_gate_granularities(oracle):
     """Scalar and elementwise combine gates: with the same logit repeated they are the headwise
     layer; an elementwise gate closed on some channels leaves exactly the intra branch there and
