@@ -58,6 +58,14 @@ typedef enum {
 #define ARL2_FLAG_GATE_ELEMENTWISE 8u /* d_gate_logits is [B, L, H, D]: one gate per output channel */
 #define ARL2_FLAG_TOKEN_GATES 2u /* reserve workspace for arl2_commit_tokens (3 fp32 copies of a
                                     [B, H, ceil(L/64)*64, D] tensor)                             */
+/* Test hook for the time-out path: every bounded wait inside the tensor-core kernels gives up
+   after `polls` polls of its barrier (0 .. 65534) instead of 2^24.  With 0 the first wait of a
+   launch expires at once: the kernel records ARL2_ERR_TIMEOUT and the wait's site in the status
+   block, every role leaves through the common exit (copies in flight are still awaited with the
+   full bound, tensor memory is freed), the output is undefined, S is untouched by a denoise
+   pass, and arl2_sync_status reports it.  Never set in production.                              */
+#define ARL2_FLAG_DEBUG_WAIT_LIMIT_SHIFT 16
+#define ARL2_FLAG_DEBUG_WAIT_LIMIT(polls) (((uint32_t)(polls) + 1u) << ARL2_FLAG_DEBUG_WAIT_LIMIT_SHIFT)
 
 typedef struct {
     uint32_t struct_size; /* sizeof(arl2_config), for versioning                            */
@@ -177,7 +185,9 @@ int arl2_commit_decay_tokens(arl2_ctx* ctx, const void* d_k_clean, const void* d
  *   alpha_l = sigmoid(d_alpha_logits[b,l,h]), beta_l = sigmoid(d_beta_logits[b,l,h]),
  * both uses of S on the right being the state before token l (Eq. 4 as printed).  Computed in
  * chunkwise form (64 tokens per chunk: a triangular solve per chunk in parallel, then one ordered
- * pass over the chunks), in fp32 arithmetic for either I/O dtype; bitwise reproducible.
+ * pass over the chunks); bitwise reproducible.  With fp32 I/O, or D = 64, the arithmetic is fp32
+ * throughout; with bf16 I/O and D = 128 the chunk factors are bf16 tensor-core operands with fp32
+ * accumulation, the state itself staying fp32.
  * d_alpha_logits, d_beta_logits: [B, L, H] fp32, each may be NULL (gate = 1).  The context must
  * have been created with ARL2_FLAG_TOKEN_GATES (else ARL2_ERR_WORKSPACE).  K', V' as in
  * arl2_commit; calls of the three commit entry points may be mixed on one context.
@@ -201,6 +211,16 @@ int arl2_set_state(arl2_ctx* ctx, const float* src, void* stream);
  * is undefined, the context stays usable).  The word is cleared by the call.
  */
 int arl2_sync_status(arl2_ctx* ctx, void* stream);
+
+/*
+ * Test hook for the time-out path (no counterpart in the paper): from the next launch on, every
+ * bounded wait inside this context's tensor-core kernels gives up after `polls` polls (0 .. 65534;
+ * see ARL2_FLAG_DEBUG_WAIT_LIMIT, which sets the same limit at creation); negative = back to the
+ * default bound.  A denoise pass that timed out leaves its output undefined and S untouched; a
+ * commit whose partial-sum kernel timed out leaves S untouched as well (the reduction that
+ * follows it sees the recorded error and does nothing).
+ */
+int arl2_debug_set_wait_limit(arl2_ctx* ctx, int32_t polls);
 
 /*
  * Measurement hook (no counterpart in the paper).  `ev_before` / `ev_after` are
@@ -236,6 +256,8 @@ int arl2_set_profile_events(arl2_ctx* ctx, void* ev_before, void* ev_after);
  *   - All calls on a device share the one array, and it keeps the previous call's contents.
  *     Nothing in it needs clearing (every slot read is written first by the same call), but
  *     two calls that overlap on the GPU (different streams, no ordering) race on it: order them.
+ *   - d_state, d_k_clean, d_v_clean and the rope tables must be 16-byte aligned (a slice that
+ *     starts in the middle of a row is refused with ARL2_ERR_INVALID_ARG before any launch).
  */
 #define ARL2_STATIC_SCRATCH_BYTES (8u << 20)
 int arl2_commit_static_scratch(const arl2_config* cfg, void* d_state, const void* d_k_clean,

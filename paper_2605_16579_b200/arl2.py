@@ -21,11 +21,15 @@ ARL2_FLAG_TOKEN_GATES = 2
 ARL2_FLAG_GATE_SCALAR = 4
 ARL2_FLAG_GATE_ELEMENTWISE = 8
 
+
+def ARL2_FLAG_DEBUG_WAIT_LIMIT(polls: int) -> int:
+    return (polls + 1) << 16
+
 EXPORTS = (
     "arl2_workspace_bytes", "arl2_create", "arl2_set_params", "arl2_denoise_step", "arl2_commit",
     "arl2_reset", "arl2_get_state", "arl2_set_state", "arl2_sync_status", "arl2_launch_count",
     "arl2_set_profile_events", "arl2_commit_static_scratch", "arl2_commit_delta", "arl2_commit_tokens", "arl2_teacher_step", "arl2_commit_decay_tokens",
-    "arl2_step_kernel_name", "arl2_destroy", "arl2_last_error", "arl2_version",
+    "arl2_step_kernel_name", "arl2_destroy", "arl2_last_error", "arl2_version", "arl2_debug_set_wait_limit",
 )
 
 
@@ -88,6 +92,8 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     lib.arl2_set_state.argtypes = [vp, vp, vp]
     lib.arl2_sync_status.restype = ctypes.c_int
     lib.arl2_sync_status.argtypes = [vp, vp]
+    lib.arl2_debug_set_wait_limit.restype = ctypes.c_int
+    lib.arl2_debug_set_wait_limit.argtypes = [vp, ctypes.c_int32]
     lib.arl2_set_profile_events.restype = ctypes.c_int
     lib.arl2_set_profile_events.argtypes = [vp, vp, vp]
     lib.arl2_commit_static_scratch.restype = ctypes.c_int
@@ -281,6 +287,10 @@ class Layer:
     def sync_status(self):
         with torch.cuda.device(self.device):
             _check(load().arl2_sync_status(self._ctx, _stream()), "arl2_sync_status")
+
+    def debug_set_wait_limit(self, polls: int):
+        """Test hook: bounded waits in the tensor-core kernels give up after ``polls`` polls (< 0: default)."""
+        _check(load().arl2_debug_set_wait_limit(self._ctx, polls), "arl2_debug_set_wait_limit")
 
     def set_profile_events(self, before: "torch.cuda.Event", after: "torch.cuda.Event"):
         """The next denoise_step records these events around its dominant kernel."""

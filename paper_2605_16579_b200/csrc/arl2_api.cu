@@ -132,6 +132,7 @@ struct arl2_ctx {
     uint64_t launches;
     uint32_t step_calls;   // parity selects the scheduler counter of the next step launch
     cudaEvent_t ev_before, ev_after;  // one-shot timing hook around the step kernel
+    uint32_t wait_limit;   // 0: the kernels' default bound; n: waits give up after n - 1 polls (test hook)
 };
 
 namespace {
@@ -207,6 +208,7 @@ int arl2_create(const arl2_config* cfg, void* d_state, void* d_workspace, size_t
     ctx->use_tc = tc_supported(*cfg);
     ctx->launches = 0;
     ctx->step_calls = 0;
+    ctx->wait_limit = cfg->flags >> ARL2_FLAG_DEBUG_WAIT_LIMIT_SHIFT;
     ctx->ev_before = ctx->ev_after = nullptr;
     int r = account(ctx, fill_zero(ctx->ws + lay.status, kStatusWords * sizeof(uint32_t),
                                    as_stream(stream)));
@@ -293,18 +295,23 @@ int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const voi
     a.state = ctx->state; a.wq = ctx->wq;
     a.rope_cos = ctx->rope_cos; a.rope_sin = ctx->rope_sin;
     a.out = d_out;
+    a.wait_limit = ctx->wait_limit;
     a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status);
-    a.launch_parity = (int)(ctx->step_calls++ & 1u);
+    a.launch_parity = (int)(ctx->step_calls & 1u);
     a.rope_h = (ctx->use_tc && ctx->rope_cos != nullptr) ? ctx->ws + ctx->lay.rope_h : nullptr;
     cudaEvent_t e0 = ctx->ev_before, e1 = ctx->ev_after;
     ctx->ev_before = ctx->ev_after = nullptr;
     if (e0 != nullptr) cudaEventRecord(e0, st);
     int r;
-    if (ctx->use_tc)
+    if (ctx->use_tc) {
         r = account(ctx, tc_step(a, reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wq_op),
                                  reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.state_bf16), st));
-    else
+        // the launch consumed one scheduler counter and cleared the other: only a launch that
+        // really went out moves on to the other one
+        if (r == ARL2_OK) ++ctx->step_calls;
+    } else {
         r = account(ctx, simt_step(a, ctx->cfg.io_dtype, st));
+    }
     if (e1 != nullptr) cudaEventRecord(e1, st);
     return r;
 }
@@ -345,8 +352,9 @@ int arl2_teacher_step(arl2_ctx* ctx, const void* d_q, const void* d_k_cache, con
     a.state = ctx->state; a.wq = ctx->wq;
     a.rope_cos = nullptr; a.rope_sin = nullptr;
     a.out = d_out;
+    a.wait_limit = ctx->wait_limit;
     a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status);
-    a.launch_parity = (int)(ctx->step_calls++ & 1u);
+    a.launch_parity = (int)(ctx->step_calls & 1u);
     a.rope_h = nullptr;                    // the caller's Q and cache are already rotated
     a.Lk = cache_tokens;
     cudaStream_t st = as_stream(stream);
@@ -355,8 +363,20 @@ int arl2_teacher_step(arl2_ctx* ctx, const void* d_q, const void* d_k_cache, con
     if (e0 != nullptr) cudaEventRecord(e0, st);
     int r = account(ctx, tc_step(a, reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wq_op),
                                  reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.state_bf16), st));
+    if (r == ARL2_OK) ++ctx->step_calls;
     if (e1 != nullptr) cudaEventRecord(e1, st);
     return r;
+}
+
+int arl2_debug_set_wait_limit(arl2_ctx* ctx, int32_t polls)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    if (polls > 65534) {
+        set_error("debug_set_wait_limit: polls must be <= 65534, or negative for the default (got %d)", polls);
+        return ARL2_ERR_INVALID_ARG;
+    }
+    ctx->wait_limit = polls < 0 ? 0u : (uint32_t)polls + 1u;
+    return ARL2_OK;
 }
 
 int arl2_set_profile_events(arl2_ctx* ctx, void* ev_before, void* ev_after)
@@ -392,6 +412,7 @@ int commit_impl(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
     a.rope_h = (ctx->use_tc && ctx->rope_cos != nullptr) ? ctx->ws + ctx->lay.rope_h : nullptr;
     a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status);
     a.mode = mode;
+    a.wait_limit = ctx->wait_limit;
     a.beta = d_beta;
     a.decay_direct = decay_direct;
     if ((reinterpret_cast<uintptr_t>(d_k_clean) | reinterpret_cast<uintptr_t>(d_v_clean)) % 16 != 0) {
@@ -440,6 +461,7 @@ int arl2_commit_tokens(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_cle
     a.kh = reinterpret_cast<float*>(ctx->ws + ctx->lay.tok_kh);
     a.gc = reinterpret_cast<float*>(ctx->ws + ctx->lay.tok_gc);
     a.nchunk = ctx->lay.nchunk;
+    a.wait_limit = ctx->wait_limit;
     if ((reinterpret_cast<uintptr_t>(d_k_clean) | reinterpret_cast<uintptr_t>(d_v_clean)) % 16 != 0) {
         set_error("commit_tokens: k_clean and v_clean must be 16-byte aligned");
         return ARL2_ERR_INVALID_ARG;

@@ -43,6 +43,7 @@ struct StepArgs {
     const void* rope_h;     // [L, D/2] half2 (cos, sin) copy of the tables (tensor-core path), or nullptr
     int Lk = 0;             // > 0: K and V hold Lk tokens (a cache), [B, Lk, H, D]; 0: L
     int gate_mode = 0;      // 0: gate [B, L, H]; 1: [B, L]; 2: [B, L, H, D]
+    uint32_t wait_limit = 0;  // 0: default; n > 0: bounded waits give up after n - 1 polls (test hook)
 };
 
 struct CommitArgs {
@@ -71,6 +72,7 @@ struct CommitArgs {
     int run_share = 0;
     int run_ntile = 0;
     int nslot = 0;                 // slots per head in `partials` (0: nsplit)
+    uint32_t wait_limit = 0;       // as in StepArgs
 };
 
 // Eq. 4 token by token with per-token gates (chunkwise form): the two launches share these.
@@ -91,6 +93,7 @@ struct TokenCommitArgs {
     float* kh;              // same shape
     float* gc;              // [B, H, nchunk] decay of a whole chunk
     int nchunk;             // ceil(L / 64)
+    uint32_t wait_limit = 0;   // as in StepArgs
 };
 constexpr int kTokenChunk = 64;
 

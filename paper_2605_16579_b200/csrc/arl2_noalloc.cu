@@ -77,6 +77,17 @@ extern "C" int arl2_commit_static_scratch(const arl2_config* cfg, void* d_state,
         set_error("commit_static_scratch: rope_cos and rope_sin must both be given or both be NULL");
         return ARL2_ERR_INVALID_ARG;
     }
+    // the kernels read and write these with 16-byte (state, K, V), 8-byte (tables) and element-wide
+    // (maps) accesses: a misaligned slice must be refused here, before anything is launched
+    const size_t esz = cfg->io_dtype == ARL2_FP32 ? 4 : 2;
+    auto misaligned = [](const void* p, size_t a) { return reinterpret_cast<uintptr_t>(p) % a != 0; };
+    if (misaligned(d_state, 16) || misaligned(d_k_clean, 16) || misaligned(d_v_clean, 16) ||
+        misaligned(d_rope_cos, 16) || misaligned(d_rope_sin, 16) || misaligned(d_decay_logits, 4) ||
+        misaligned(d_wphi_k, esz) || misaligned(d_wphi_v, esz)) {
+        set_error("commit_static_scratch: state, k_clean, v_clean and the rope tables must be 16-byte "
+                  "aligned, decay_logits 4-byte and the feature maps element aligned");
+        return ARL2_ERR_INVALID_ARG;
+    }
     const int nsplit = (cfg->L + kCommitChunk - 1) / kCommitChunk;
     const unsigned long long need =
         (unsigned long long)cfg->B * cfg->H * nsplit * cfg->D * cfg->D * sizeof(float);

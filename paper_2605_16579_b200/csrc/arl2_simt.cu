@@ -725,10 +725,13 @@ __global__ void __launch_bounds__(NT) token_scan_kernel(TokenCommitArgs a)
 __global__ void commit_reduce_kernel(float* __restrict__ state, const float* __restrict__ partials,
                                      const float* __restrict__ decay, int decay_direct,
                                      __nv_bfloat16* __restrict__ state_bf16, int nsplit, int DD,
-                                     size_t total4, int run_share, int run_ntile, int nslot)
+                                     size_t total4, int run_share, int run_ntile, int nslot,
+                                     const uint32_t* __restrict__ status)
 {
     size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= total4) return;
+    // a partial-sum kernel that gave up on a bounded wait left its slots unwritten: S stays as it was
+    if (status != nullptr && status[kStatusError] != 0u) return;
     size_t e = t * 4;
     size_t bh = e / DD;
     size_t within = e % DD;
@@ -933,7 +936,7 @@ int commit_reduce(const CommitArgs& a, cudaStream_t st)
     size_t total4 = (size_t)a.s.B * a.s.H * DD / 4;
     commit_reduce_kernel<<<(unsigned)((total4 + 255) / 256), 256, 0, st>>>(
         a.state, a.partials, a.decay, a.decay_direct ? 1 : 0, a.state_bf16, a.nsplit, DD, total4,
-        a.run_share, a.run_ntile, a.nslot);
+        a.run_share, a.run_ntile, a.nslot, a.status);
     if (int r = check_launch("commit_reduce_kernel")) return r;
     return 1;
 }

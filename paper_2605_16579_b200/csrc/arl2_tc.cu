@@ -22,6 +22,8 @@
 #include <cuda.h>
 #include <cuda_fp16.h>
 
+#include <mutex>
+
 #include "arl2_internal.h"
 #include "tc_ptx.cuh"
 
@@ -44,14 +46,6 @@ constexpr int kLaunchRegs = (65536 / kThreads) / 8 * 8;
 static_assert(256 * kRegsSoftmax + (kThreads - 256) * kRegsOther <= kThreads * kLaunchRegs, "register pool");
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units of slack before O is rescaled
-#ifndef ARL2_POLY_COUNT
-#define ARL2_POLY_COUNT 0
-#endif
-#ifndef ARL2_POLY_PERIOD
-#define ARL2_POLY_PERIOD 2
-#endif
-constexpr int kPolyCount = ARL2_POLY_COUNT;    // of every kPolyPeriod element pairs, this many take the
-constexpr int kPolyPeriod = ARL2_POLY_PERIOD;  // polynomial exponential, the rest the special-function unit
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int kOffQ = 0;                                 // 2 query tiles (rotated in place)
@@ -69,6 +63,7 @@ enum Bar : int {
     kBarPFull0, kBarPFull1,
     kBarOFinal0, kBarOFinal1,
     kBarTok0, kBarTok1,                         // softmax groups take turns in the exponential phase
+    kBarDrain0, kBarDrain1,                     // an MMA issuer that gives up waits here for its MMAs in flight
     kNumBars
 };
 // after the barriers: TMEM base (4 B), abort flag (4 B), two item-id slots (8 B)
@@ -82,6 +77,7 @@ struct TcStepParams {
     const uint4* rope_h;       // half2 (cos, sin) table, warp-interleaved (see pack_rope_kernel), or nullptr
     __nv_bfloat16* out;
     uint32_t* status;
+    uint32_t spin_limit;       // polls a bounded wait makes before it gives up
     uint32_t* sched_counter;   // this launch's item counter (zero on entry)
     uint32_t* sched_next;      // the next launch's counter: cleared by this launch
     int gate_mode;             // 0: gate logits [B, L, H]; 1: [B, L] (one per token); 2: [B, L, H, D] (per channel)
@@ -95,11 +91,12 @@ struct TcStepParams {
 struct Abort {
     volatile int* flag;   // in shared memory
     uint32_t* status;     // device status block
+    uint32_t limit;       // polls before a wait gives up
 };
 
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Abort& ab, int site)
 {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    for (uint32_t it = 0; it < ab.limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 255u && *ab.flag) return false;
     }
@@ -115,22 +112,6 @@ __device__ __forceinline__ void drain_bar(uint32_t bar, uint32_t parity)
     for (uint32_t it = 0; it < kSpinLimit; ++it)
         if (mbar_try_wait(bar, parity)) return;
 }
-
-#ifdef ARL2_TRACE_ITER
-// Per-iteration log of tuning builds run WITHOUT RoPE: the words after the status block belong
-// to the rotated-K buffer, which is unused then.
-#define ARL2_ITER(cond, slot) do { if (blockIdx.x == 0 && item < 2 && r == 0 && (cond)) p.status[64 + (slot)] = (uint32_t)clock64(); } while (0)
-#else
-#define ARL2_ITER(cond, slot) do { } while (0)
-#endif
-
-#ifdef ARL2_TRACE
-// Timeline probe for tuning builds: one thread of CTA 0 stamps the SM clock into the status
-// block for two loop iterations of its first item.  Not compiled into the product library.
-#define ARL2_STAMP(cond, slot) do { if (cond) p.status[(slot)] = (uint32_t)clock64(); } while (0)
-#else
-#define ARL2_STAMP(cond, slot) do { } while (0)
-#endif
 
 __device__ __forceinline__ float sigmoid_fast(float x) { return 1.0f / (1.0f + __expf(-x)); }
 
@@ -162,29 +143,6 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
     uint64_t d;
     asm("add.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
-}
-
-// 2^x for a pair of values without the special-function unit: x = j + f with j = round(x),
-// f in [-0.5, 0.5]; 2^f by a cubic (max relative error 7.5e-5, well under the bf16 rounding of
-// the probabilities), 2^j by adding j to the exponent field.  x is clamped at -126.
-__device__ __forceinline__ void exp2_poly2(float x0, float x1, float& r0, float& r1)
-{
-    const float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
-    x0 = fmaxf(x0, -126.0f);
-    x1 = fmaxf(x1, -126.0f);
-    const uint64_t x2 = pack2(x0, x1);
-    const uint64_t t2 = add2(x2, pack2(kMagic, kMagic));
-    const uint64_t j2 = add2(t2, pack2(-kMagic, -kMagic));
-    const uint64_t f2 = fma2(j2, pack2(-1.0f, -1.0f), x2);
-    uint64_t p2 = fma2(pack2(0.05517132207751274f, 0.05517132207751274f), f2,
-                       pack2(0.24261054396629333f, 0.24261054396629333f));
-    p2 = fma2(p2, f2, pack2(0.6932609677314758f, 0.6932609677314758f));
-    p2 = fma2(p2, f2, pack2(0.9999281167984009f, 0.9999281167984009f));
-    float t0, t1, q0, q1;
-    unpack2(t2, t0, t1);
-    unpack2(p2, q0, q1);
-    r0 = __int_as_float(__float_as_int(q0) + (__float_as_int(t0) << 23));
-    r1 = __int_as_float(__float_as_int(q1) + (__float_as_int(t1) << 23));
 }
 
 // A work item drives up to two 128-row query tiles.  A "pair" item holds two consecutive tiles of
@@ -302,7 +260,6 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
 
     for (uint32_t item = 0;; ++item) {
         if (!wait_bar(bars + 8 * kBarQFull, item & 1, ab, 10)) return;
-        ARL2_ITER(true, 256 + item * 16 + t * 8 + 5);
         const int id = item_slots[item & 1];
         if (id < 0) return;
         const Item it = decode_item(id, p);
@@ -336,31 +293,21 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                     }
                     *reinterpret_cast<uint4*>(tile + off) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
-                ARL2_ITER(true, 256 + item * 16 + t * 8 + 7);
                 fence_proxy_async_smem();
             }
             mbar_arrive(bars + 8 * (kBarQRot0 + t));
-            ARL2_ITER(true, 256 + item * 16 + t * 8 + 6);
 
             float m_ref = -INFINITY;   // reference maximum (scaled, base 2) of the probabilities
             uint64_t l2 = pack2(0.0f, 0.0f);   // running row sum relative to m_ref, two lanes
 
             for (int j = 0; j < n_kv; ++j) {
-#ifdef ARL2_TRACE
-                const bool tr = blockIdx.x == 0 && item == 0 && r == 0 && (j == 8 || j == 9);
-                const int ts = 8 + t * 16 + (j - 8) * 8;
-#endif
-                ARL2_STAMP(tr, ts + 0);
                 if (!wait_bar(bar_s, s_cnt & 1, ab, 20 + t)) return;
                 ++s_cnt;
                 tc_fence_after();
-                ARL2_STAMP(tr, ts + 1);
-                ARL2_ITER(j < 60, item * 128 + t * 64 + j);
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
                     tmem_ld32(s_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
                 tmem_wait_ld();
-                ARL2_STAMP(tr, ts + 2);
 
                 const int n_valid = p.Lk - j * kTile;  // keys of this tile that exist
                 if (n_valid < kTile) {   // ragged last tile: zero-filled key rows must not count
@@ -378,7 +325,6 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                 const float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
                 const float m_new = fmaxf(m_ref, mx * c2);
                 const bool need = (m_new - m_ref) > kRescaleThreshold;   // first tile: inf > threshold
-                ARL2_STAMP(tr, ts + 3);
                 if (__any_sync(0xffffffffu, need)) {
                     float alpha = 1.0f;
                     if (need) {
@@ -408,46 +354,21 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                     if (!wait_bar(bars + 8 * (kBarTok0 + t), par, ab, 24 + t)) return;
                     ++tok_cnt;
                 }
-                ARL2_STAMP(tr, ts + 4);
-#ifndef ARL2_SOFTMAX_SCALAR
 #pragma unroll
                 for (int c = 0; c < 64; ++c) {
-                    float x0, x1, p0, p1;
+                    float x0, x1;
                     unpack2(fma2(pack2(__uint_as_float(sreg[2 * c]), __uint_as_float(sreg[2 * c + 1])), c2x2, neg_m2),
                             x0, x1);
-                    if ((c % kPolyPeriod) < kPolyCount) {
-                        exp2_poly2(x0, x1, p0, p1);      // FMA / integer pipes
-                    } else {
-                        p0 = ex2_approx(x0);             // special-function unit
-                        p1 = ex2_approx(x1);
-                    }
+                    const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);   // special-function unit
                     l2 = add2(l2, pack2(p0, p1));
                     sreg[c] = pack_bf16(p0, p1);
                 }
-#else
-                {
-                    float la, lb;
-                    unpack2(l2, la, lb);
-                    const float nm = -m_ref;
-#pragma unroll
-                    for (int c = 0; c < 64; ++c) {
-                        const float p0 = ex2_approx(fmaf(__uint_as_float(sreg[2 * c]), c2, nm));
-                        const float p1 = ex2_approx(fmaf(__uint_as_float(sreg[2 * c + 1]), c2, nm));
-                        la += p0;
-                        lb += p1;
-                        sreg[c] = pack_bf16(p0, p1);
-                    }
-                    l2 = pack2(la, lb);
-                }
-#endif
                 if (it.ntile == 2) mbar_arrive(bars + 8 * (kBarTok0 + (t ^ 1)));
-                ARL2_STAMP(tr, ts + 5);
                 tmem_st32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sreg[0]));
                 tmem_st32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[32]));
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar_p);
-                ARL2_STAMP(tr, ts + 6);
             }
             float l_lo, l_hi;
             unpack2(l2, l_lo, l_hi);
@@ -467,10 +388,8 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
 #pragma unroll
                 for (int c = 0; c < 16; ++c) cs[c] = __ldg(tab + c * 32);
             }
-            ARL2_ITER(true, 256 + item * 16 + t * 8 + 0);
             if (!wait_bar(bar_s, s_cnt & 1, ab, 30 + t)) return;
             ++s_cnt;
-            ARL2_ITER(true, 256 + item * 16 + t * 8 + 1);
             tc_fence_after();
 #pragma unroll
             for (int c = 0; c < 4; ++c)
@@ -562,9 +481,7 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                 continue;
             }
             // ---- epilogue: O_t / l -> bf16 -> global                              (Eq. 6-7)
-            ARL2_ITER(true, 256 + item * 16 + t * 8 + 2);
             if (!wait_bar(bars + 8 * (kBarOFinal0 + t), of_cnt & 1, ab, 40 + t)) return;
-            ARL2_ITER(true, 256 + item * 16 + t * 8 + 3);
             ++of_cnt;
             tc_fence_after();
             const float inv_l = 1.0f / l_sum;
@@ -591,7 +508,6 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                 }
             }
             tc_fence_before();
-            ARL2_ITER(true, 256 + item * 16 + t * 8 + 4);
         }
     }
 }
@@ -610,7 +526,7 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffBars + kNumBars * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffBars + kNumBars * 8 + 4);
     volatile int* item_slots = reinterpret_cast<volatile int*>(smem + kOffBars + kNumBars * 8 + 8);
-    const Abort ab{abort_flag, p.status};
+    const Abort ab{abort_flag, p.status, p.spin_limit};
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_kv = p.n_kv;
@@ -632,6 +548,8 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         mbar_init(bars + 8 * kBarOFinal1, 1);
         mbar_init(bars + 8 * kBarTok0, 128);
         mbar_init(bars + 8 * kBarTok1, 128);
+        mbar_init(bars + 8 * kBarDrain0, 1);
+        mbar_init(bars + 8 * kBarDrain1, 1);
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async_smem();
@@ -663,7 +581,7 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             const uint32_t bar_q = bars + 8 * kBarQFull;
             uint32_t n = 0;       // ring entries produced so far (all items)
             bool ok = true;
-            bool q_in_flight = false;
+            int q_item = -1;      // item whose Q tiles were requested last
             int id = (int)blockIdx.x;
             for (uint32_t item = 0; ok; ++item) {
                 if (item > 0) ok = wait_bar(bars + 8 * kBarQFree, (item - 1) & 1, ab, 50);
@@ -677,7 +595,7 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const Item it = decode_item(id, p);
                 const int ntile = it.ntile;
                 mbar_expect_tx(bar_q, ntile * kTileBytes);
-                q_in_flight = true;
+                q_item = (int)item;
                 for (int t = 0; t < ntile; ++t) {
                     uint32_t dst = smem_base + kOffQ + t * kTileBytes;
                     tma_load_4d(dst, &tm_q, bar_q, 0, it.h[t], it.row0[t], it.b[t]);
@@ -714,10 +632,7 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
             if (!ok || *abort_flag) {
                 // do not leave the CTA while bulk copies into its shared memory are in flight
-                if (q_in_flight) {
-                    drain_bar(bar_q, 0);
-                    drain_bar(bar_q, 1);
-                }
+                if (q_item >= 0) drain_bar(bar_q, (uint32_t)q_item & 1);
                 for (uint32_t m = (n > (uint32_t)kStages ? n - kStages : 0); m < n; ++m)
                     drain_bar(bars + 8 * (kBarFull0 + m % kStages), (m / kStages) & 1);
             }
@@ -816,10 +731,6 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     const bool last = j + 1 == n_kv;     // then the next "S" is the inter branch's Q W
                     const int per_tile = last ? 3 : 2;   // ragged item: V, K or W, [Qraw] per tile
                     const int group = shared ? (last ? 2 + ntile : 2) : per_tile * ntile;
-#ifdef ARL2_TRACE
-                    const bool tr = blockIdx.x == 0 && item == 0 && (j == 8 || j == 9);
-                    const int ts = 40 + t * 8 + (j - 8) * 4;
-#endif
                     if (active) {
                         const uint32_t e_v = shared ? cons : cons + per_tile * t;   // V_j
                         const uint32_t e_b = e_v + 1;                               // K_{j+1} or W
@@ -828,16 +739,13 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                         if (ok) ok = wait_full(e_b, 66);
                         if (ok && last) ok = wait_full(e_q, 68);
                         if (!ok) break;
-                        ARL2_STAMP(tr, ts + 0);
                         ok = wait_bar(bar_p, p_cnt & 1, ab, 64 + t);
                         ++p_cnt;
                         if (!ok) break;
                         tc_fence_after();
-                        ARL2_STAMP(tr, ts + 1);
                         issue_pv(slot_addr(e_v), j > 0);
                         issue_qk(last ? slot_addr(e_q) : q_tile, slot_addr(e_b));
                         mma_commit(bar_s);
-                        ARL2_STAMP(tr, ts + 2);
                         release_mine(e_v, !shared);
                         release_mine(e_b, !shared);
                         if (last) release_mine(e_q, true);
@@ -884,6 +792,11 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 cons += shared ? 1 : ntile;
             }
             (void)of_cnt;
+            if (!ok || *abort_flag) {
+                // tensor memory is freed below: none of this thread's MMAs may still be running
+                mma_commit(bars + 8 * (kBarDrain0 + t));
+                drain_bar(bars + 8 * (kBarDrain0 + t), 0);
+            }
         }
     }
 
@@ -917,7 +830,7 @@ constexpr int kCOffBars = kCOffState + kTileBytes;
 constexpr int kCommitSmemBytes = kCOffBars + 128 + 1024 + 1024;   // barriers, row-norm exchange, alignment slack
 constexpr int kCommitThreads = 256;
 
-enum CBar : int { kCBarW = 0, kCBarFull0, kCBarFull1, kCBarU, kCBarS, kCBarP, kCNumBars };
+enum CBar : int { kCBarW = 0, kCBarFull0, kCBarFull1, kCBarU, kCBarS, kCBarP, kCBarDrain, kCNumBars };
 
 struct TcCommitParams {
     Shape s;
@@ -925,6 +838,7 @@ struct TcCommitParams {
     const float* beta;     // [B, L, H] learning-rate logits (delta rule), or nullptr = 1
     float* partials;     // [B * H, nslot, 128, 128] fp32
     uint32_t* status;
+    uint32_t spin_limit;
     int ntile;           // 128-token tiles per (stream, head)
     int total_tiles;     // B * H * ntile
     int share;           // tiles per CTA: CTA c takes tiles [c * share, (c + 1) * share) of the flattened order
@@ -987,7 +901,7 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     const uint32_t bars = smem_base + kCOffBars;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kCOffBars + kCNumBars * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kCOffBars + kCNumBars * 8 + 4);
-    const Abort ab{abort_flag, p.status};
+    const Abort ab{abort_flag, p.status, p.spin_limit};
 
     const int tid = threadIdx.x, warp = tid >> 5;
     const int L = p.s.L, H = p.s.H;
@@ -1239,6 +1153,9 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         if (w_loads > 0) drain_bar(bars + 8 * kCBarW, (w_loads - 1) & 1);
         for (int m = (loads_issued > 2 ? loads_issued - 2 : 0); m < loads_issued; ++m)
             drain_bar(bars + 8 * (kCBarFull0 + (m & 1)), (uint32_t)((m >> 1) & 1));
+        // nor an MMA still writing tensor memory when it is freed
+        mma_commit(bars + 8 * kCBarDrain);
+        drain_bar(bars + 8 * kCBarDrain, 0);
     }
     tc_fence_before();
     __syncthreads();
@@ -1271,7 +1188,7 @@ constexpr int kTokC = 64;                          // tokens per chunk
 constexpr int kLdA = kTokC + 4;   // 16-byte aligned rows, conflict-free 16-byte stores
 static_assert(2 * kTokC * kLdA * 4 <= 2 * kTileBytes, "A fits over the two maps");
 
-enum TPBar : int { kTPBarLoad = 0, kTPBarU, kTPBarG, kTPBarW, kTPNumBars };
+enum TPBar : int { kTPBarLoad = 0, kTPBarU, kTPBarG, kTPBarW, kTPBarDrain, kTPNumBars };
 
 struct TcTokenParams {
     Shape s;
@@ -1285,6 +1202,7 @@ struct TcTokenParams {
     float* state;              // scan kernel only
     __nv_bfloat16* state_bf16;
     uint32_t* status;
+    uint32_t spin_limit;
     int ntile;                 // 128-token tiles; rows_pad = 128 * ntile
     int nchunk;                // ceil(L / 64): chunks the scan walks
 };
@@ -1303,7 +1221,7 @@ tc_token_prepare_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kTPOffBars + kTPNumBars * 8 + 4);
     float* cl_s = reinterpret_cast<float*>(smem + kTPOffBars + 64);          // [128] log g_j (inclusive)
     float* wsum = reinterpret_cast<float*>(smem + kTPOffBars + 64 + 512);    // [4] warp totals
-    const Abort ab{abort_flag, p.status};
+    const Abort ab{abort_flag, p.status, p.spin_limit};
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int tile = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
@@ -1542,7 +1460,11 @@ tc_token_prepare_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
         if (jj == kTokC - 1)
             p.gc[(((size_t)b * H + h) * p.ntile + tile) * 2 + chunk] = expf(cl_total);
     }
-    if (tid == 0 && (!ok || *abort_flag)) drain_bar(bars + 8 * kTPBarLoad, 0);   // no bulk copy left in flight
+    if (tid == 0 && (!ok || *abort_flag)) {
+        drain_bar(bars + 8 * kTPBarLoad, 0);   // no bulk copy left in flight
+        mma_commit(bars + 8 * kTPBarDrain);    // and no MMA still writing tensor memory
+        drain_bar(bars + 8 * kTPBarDrain, 0);
+    }
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
@@ -1569,7 +1491,7 @@ constexpr int kTSSmemBytes = kTSOffBars + 128 + 1024;
 constexpr int kChunkHalf = kTokC * 128;              // bytes of a 64-row, 64-column box
 constexpr uint32_t kChunkTx = kTileBytes + 4 * kChunkHalf;   // W tile + Khat + U1 per chunk
 
-enum TSBar : int { kTSBarS0 = 0, kTSBarFull0, kTSBarFull1, kTSBarY, kTSBarS2, kTSNumBars };
+enum TSBar : int { kTSBarS0 = 0, kTSBarFull0, kTSBarFull1, kTSBarY, kTSBarS2, kTSBarDrain, kTSNumBars };
 
 constexpr int kTSThreads = 256;
 __global__ void __launch_bounds__(kTSThreads, 1)
@@ -1584,7 +1506,7 @@ tc_token_scan_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
     const uint32_t bars = smem_base + kTSOffBars;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kTSOffBars + kTSNumBars * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kTSOffBars + kTSNumBars * 8 + 4);
-    const Abort ab{abort_flag, p.status};
+    const Abort ab{abort_flag, p.status, p.spin_limit};
 
     const int tid = threadIdx.x, warp = tid >> 5;
     const int h = blockIdx.x, b = blockIdx.y;
@@ -1778,6 +1700,8 @@ tc_token_scan_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
         drain_bar(bars + 8 * kTSBarS0, 0);
         for (int m = (loads_issued > 2 ? loads_issued - 2 : 0); m < loads_issued; ++m)
             drain_bar(bars + 8 * (kTSBarFull0 + (m & 1)), (uint32_t)((m >> 1) & 1));
+        mma_commit(bars + 8 * kTSBarDrain);    // no MMA still writing tensor memory when it is freed
+        drain_bar(bars + 8 * kTSBarDrain, 0);
     }
     tc_fence_before();
     __syncthreads();
@@ -1894,6 +1818,56 @@ int make_map_rows(CUtensorMap* m, const void* base, size_t rows, int box_rows = 
     return 0;
 }
 
+// Per-device, once, under a lock: the SM count and the opt-in to large dynamic shared memory for
+// every kernel of this file (the attribute belongs to the device that is current when it is set).
+constexpr int kMaxDevices = 64;
+struct DeviceSetup {
+    bool ready = false;
+    int num_sms = 0;
+};
+std::mutex g_setup_mutex;
+DeviceSetup g_setup[kMaxDevices];
+
+template <typename K>
+cudaError_t opt_in_smem(K kernel, int bytes)
+{
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
+
+int device_setup(int* num_sms)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        set_error("cannot identify the current device (%s)", cudaGetErrorString(e));
+        return ARL2_ERR_CUDA;
+    }
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    DeviceSetup& d = g_setup[dev];
+    if (!d.ready) {
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
+            set_error("cannot read the SM count of device %d", dev);
+            return ARL2_ERR_CUDA;
+        }
+        e = opt_in_smem(tc_step_kernel<false>, kSmemBytes);
+        if (e == cudaSuccess) e = opt_in_smem(tc_step_kernel<true>, kSmemBytes);
+        if (e == cudaSuccess) e = opt_in_smem(tc_commit_kernel<0>, kCommitSmemBytes);
+        if (e == cudaSuccess) e = opt_in_smem(tc_commit_kernel<1>, kCommitSmemBytes);
+        if (e == cudaSuccess) e = opt_in_smem(tc_commit_kernel<2>, kCommitSmemBytes);
+        if (e == cudaSuccess) e = opt_in_smem(tc_token_prepare_kernel, kTPSmemBytes);
+        if (e == cudaSuccess) e = opt_in_smem(tc_token_scan_kernel, kTSSmemBytes);
+        if (e != cudaSuccess) {
+            set_error("cudaFuncSetAttribute(dynamic shared memory) on device %d: %s", dev, cudaGetErrorString(e));
+            return ARL2_ERR_CUDA;
+        }
+        d.num_sms = sms;
+        d.ready = true;
+    }
+    *num_sms = d.num_sms;
+    return 0;
+}
+
 }  // namespace
 
 bool tc_supported(const arl2_config& c)
@@ -1933,21 +1907,8 @@ int tc_prepare_rope(const float* cos_t, const float* sin_t, void* out, int L, cu
 
 int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* state_bf16, cudaStream_t st)
 {
-    static bool attr_set = false;
-    static int num_sms = 0;
-    if (!attr_set) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0) {
-            set_error("cannot read the SM count");
-            return ARL2_ERR_CUDA;
-        }
-        cudaError_t e = cudaFuncSetAttribute(tc_step_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(tc_step_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e != cudaSuccess) { set_error("cudaFuncSetAttribute(tc_step_kernel, %d): %s", kSmemBytes, cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
-        attr_set = true;
-    }
+    int num_sms = 0;
+    if (int r = device_setup(&num_sms)) return r;
     CUtensorMap tm_q, tm_k, tm_v, tm_w, tm_s;
     if (int r = make_map_blhd(&tm_q, a.q, a.s)) return r;
     Shape ks = a.s;
@@ -1965,6 +1926,7 @@ int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* 
     p.rope_h = static_cast<const uint4*>(a.rope_h);
     p.out = static_cast<__nv_bfloat16*>(a.out);
     p.status = a.status;
+    p.spin_limit = a.wait_limit ? a.wait_limit - 1 : kSpinLimit;
     p.Lk = ks.L;
     p.n_q = (a.s.L + kTile - 1) / kTile;
     p.n_kv = (ks.L + kTile - 1) / kTile;
@@ -1986,19 +1948,8 @@ int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* 
 
 int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat16* wv_op, cudaStream_t st)
 {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc_commit_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             kCommitSmemBytes);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(tc_commit_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     kCommitSmemBytes);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(tc_commit_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     kCommitSmemBytes);
-        if (e != cudaSuccess) { set_error("cudaFuncSetAttribute(tc_commit_kernel, %d): %s", kCommitSmemBytes, cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
-        attr_set = true;
-    }
+    int num_sms = 0;
+    if (int r = device_setup(&num_sms)) return r;
     if (a.mode == 1 && a.state_bf16 == nullptr) {
         set_error("tc_commit: the delta rule needs the bf16 copy of the state");
         return ARL2_ERR_INVALID_ARG;
@@ -2019,16 +1970,7 @@ int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat
     p.beta = a.beta;
     p.partials = a.partials;
     p.status = a.status;
-    static int num_sms = 0;
-    if (num_sms == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0) {
-            num_sms = 0;
-            set_error("cannot read the SM count");
-            return ARL2_ERR_CUDA;
-        }
-    }
+    p.spin_limit = a.wait_limit ? a.wait_limit - 1 : kSpinLimit;
     // equal runs of the flattened tile sequence, at least 2 tiles each and long enough for a head's
     // partial sums (one per run it falls into, at most ceil(ntile / share) + 1) to fit the slots
     p.ntile = (a.s.L + kTile - 1) / kTile;
@@ -2064,15 +2006,9 @@ int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat
 int tc_commit_tokens(const TokenCommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat16* wv_op,
                      const void* rope_h, uint32_t* status, cudaStream_t st)
 {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc_token_prepare_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             kTPSmemBytes);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(tc_token_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSSmemBytes);
-        if (e != cudaSuccess) { set_error("cudaFuncSetAttribute(token kernels): %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
-        attr_set = true;
-    }
+    int num_sms = 0;
+    if (int r = device_setup(&num_sms)) return r;
+    (void)num_sms;
     if (a.state_bf16 == nullptr) { set_error("tc_commit_tokens: needs the bf16 copy of the state"); return ARL2_ERR_INVALID_ARG; }
     TcTokenParams p;
     p.s = a.s;
@@ -2086,6 +2022,7 @@ int tc_commit_tokens(const TokenCommitArgs& a, const __nv_bfloat16* wk_op, const
     p.state = a.state;
     p.state_bf16 = a.state_bf16;
     p.status = status;
+    p.spin_limit = a.wait_limit ? a.wait_limit - 1 : kSpinLimit;
     p.ntile = (a.s.L + kTile - 1) / kTile;
     p.nchunk = (a.s.L + kTokC - 1) / kTokC;
     const size_t rows = (size_t)a.s.B * a.s.H * p.ntile * kTile;

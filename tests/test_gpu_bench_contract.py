@@ -25,6 +25,10 @@ def test_bench_line_has_the_contract_keys():
     for key in ("bound", "achieved", "peak", "unit", "frac", "traffic"):
         assert key in line["roofline"], key
     assert abs(line["roofline"]["frac"] - line["roofline"]["achieved"] / line["roofline"]["peak"]) < 1e-9
+    # one denominator whatever the run length (the burst figure), the sustained one beside it
+    assert line["roofline"]["frac"] == line["roofline"]["frac_of_burst"]
+    assert line["roofline"]["frac_of_sustained"] > line["roofline"]["frac_of_burst"]
+    assert line["denoise_pass_all_kernels"]["ms_mean"] >= line["denoise_pass"]["kernel_ms_mean"]
     for key in ("value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step"):
         assert key in line["e2e"], key
     assert line["e2e"]["h2d_bytes_per_step"] > 0 and line["e2e"]["d2h_bytes_per_step"] > 0

@@ -51,3 +51,20 @@ def test_whole_job_value_scales_with_replicas():
     assert abs(one - cfg.B * cfg.L * cfg.steps / 2e-3) < 1e-6
     assert abs(bench.whole_job_value(cfg, 8, 2.0) - 8 * one) < 1e-3
     assert bench.max_over_ranks([1.5, 2.5], 1, None) == [1.5, 2.5]
+
+
+def test_gpus_flag_starts_that_many_ranks():
+    """`--gpus N` outside a launcher starts N ranks itself; inside one it must agree with it."""
+    import subprocess
+
+    sys.path.insert(0, ROOT)
+    import bench
+
+    cmd = bench.launcher_command(4, ["--gpus", "4", "--steps", "2"], port=29777)
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"]
+    assert "--nproc-per-node=4" in cmd and cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[-4:] == ["--gpus", "4", "--steps", "2"] and cmd[-5].endswith("bench.py")
+    env = dict(os.environ, WORLD_SIZE="2", RANK="0", LOCAL_RANK="0")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "1"], env=env,
+                         capture_output=True, text=True, timeout=120)
+    assert out.returncode != 0 and "WORLD_SIZE=2" in out.stderr
