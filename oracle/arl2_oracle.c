@@ -357,6 +357,22 @@ void arl2_oracle_commit(int B, int H, int L, int D,
 }
 
 /*
+ * The clean pass of one block (Algorithm 1, clean-pass branch; Sec. 3.3): the layer's output for
+ * the clean latent's Q, K, V, read against the state as it stands (Eq. 8: every token queries the
+ * same PRE-update state), and only then the gated-linear commit of that block from the same K, V:
+ *   out = step(q, kc, vc, g; S),   S <- sigmoid(a) S + sum_j K'_j^T V'_j.
+ */
+void arl2_oracle_clean_pass(int B, int H, int L, int D,
+                            const double *q, const double *kc, const double *vc, const double *g,
+                            const double *a, const double *wq, const double *wk, const double *wv,
+                            const double *rope_cos, const double *rope_sin, double scale, double eps,
+                            double *S, double *out)
+{
+    arl2_oracle_step(B, H, L, D, q, kc, vc, g, S, wq, rope_cos, rope_sin, scale, eps, out);
+    arl2_oracle_commit(B, H, L, D, kc, vc, a, NULL, wk, wv, rope_cos, rope_sin, eps, 0, 0, NULL, NULL, S);
+}
+
+/*
  * Eq. 4 applied token by token with per-token gates (the sentence after Eq. 4: the update
  * runs sequentially over the L tokens of the frame, with gates alpha^(j), beta^(j)):
  *   for j = 0..L-1:   S <- alpha_j S + beta_j K'_j^T (V'_j - K'_j S)

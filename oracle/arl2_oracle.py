@@ -175,6 +175,24 @@ def commit(kc, vc, a, S, wk=None, wv=None, rope_cos=None, rope_sin=None, eps=1e-
     return S
 
 
+def clean_pass(q, kc, vc, g, a, S, wq=None, wk=None, wv=None, rope_cos=None, rope_sin=None, scale=None,
+               eps=1e-6):
+    """The clean pass of a block: returns (out, S_new); out is read against the state passed in."""
+    q, kc, vc, g, a = _f64(q), _f64(kc), _f64(vc), _f64(g), _f64(a)
+    wq, wk, wv, rope_cos, rope_sin = _f64(wq), _f64(wk), _f64(wv), _f64(rope_cos), _f64(rope_sin)
+    S = _f64(S).copy()
+    B, L, H, D = q.shape
+    assert S.shape == (B, H, D, D) and a.shape == (B, H) and g.shape == (B, L, H)
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    out = np.empty_like(q)
+    _load().arl2_oracle_clean_pass(
+        B, H, L, D, _p(q), _p(kc), _p(vc), _p(g), _p(a), _p(wq), _p(wk), _p(wv), _p(rope_cos), _p(rope_sin),
+        ctypes.c_double(scale), ctypes.c_double(eps), _p(S), _p(out),
+    )
+    return out, S
+
+
 def commit_tokens(kc, vc, S, alpha_logit=None, beta_logit=None, wk=None, wv=None, rope_cos=None,
                   rope_sin=None, eps=1e-6, heads=None):
     """Eq. 4 token by token with per-token gates [B, L, H] (None = gate 1).  Returns the new S."""

@@ -38,6 +38,11 @@ MUTANTS = [
     ("softmax normalised by the maximum term only", "double w = p[j] / den;", "double w = p[j];"),
     ("elementwise gate indexed per head", "gate_mode == 2 ? (((size_t)b * L + i) * H + h) * D + e",
      "gate_mode == 2 ? (((size_t)b * L + i) * H + h) * D"),
+    ("clean pass reads the state it has just written",
+     "    arl2_oracle_step(B, H, L, D, q, kc, vc, g, S, wq, rope_cos, rope_sin, scale, eps, out);\n"
+     "    arl2_oracle_commit(B, H, L, D, kc, vc, a, NULL, wk, wv, rope_cos, rope_sin, eps, 0, 0, NULL, NULL, S);",
+     "    arl2_oracle_commit(B, H, L, D, kc, vc, a, NULL, wk, wv, rope_cos, rope_sin, eps, 0, 0, NULL, NULL, S);\n"
+     "    arl2_oracle_step(B, H, L, D, q, kc, vc, g, S, wq, rope_cos, rope_sin, scale, eps, out);"),
     ("reset clears the wrong stream", "else memset(S + per * stream, 0, sizeof(double) * per);",
      "else memset(S, 0, sizeof(double) * per);"),
 ]

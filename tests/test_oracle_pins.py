@@ -528,6 +528,28 @@ def test_state_norm_stays_bounded(oracle):
     assert max(norms[T // 2:]) < 1.5 * max(norms[: T // 2])   # flat, not growing with T
 
 
+def test_clean_pass_reads_the_state_before_it_commits(oracle):
+    """The clean pass is the step on the pre-update state followed by the commit (Sec. 3.3, Eq. 8).
+    Pinned through a case with a closed form: with V_c = 0 nothing is written (S_new = alpha S) and
+    the output is sigmoid(g) Q' S_old, so alpha * out must equal what a step reads from S_new --
+    an output that saw the new state would be off by the factor alpha."""
+    B, L, H, D = 2, 7, 2, 8
+    q, k, v, g = rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H)
+    a, S0 = rnd(B, H), rnd(B, H, D, D)
+    wq, wk, wv = rnd(H, D, D), rnd(H, D, D), rnd(H, D, D)
+    cos, sin = tables(L, D)
+    out, S1 = oracle.clean_pass(q, k, v, g, a, S0, wq, wk, wv, cos, sin)
+    np.testing.assert_array_equal(out, oracle.step(q, k, v, g, S0, wq, cos, sin))
+    np.testing.assert_array_equal(S1, oracle.commit(k, v, a, S0, wk, wv, cos, sin))
+    assert not np.allclose(out, oracle.step(q, k, v, g, S1, wq, cos, sin))
+    zero = np.zeros_like(v)
+    out0, S1z = oracle.clean_pass(q, k, zero, g, a, S0, wq, wk, wv, cos, sin)
+    alpha = sig(a)
+    np.testing.assert_allclose(S1z, alpha[..., None, None] * S0, rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(alpha[:, None, :, None] * out0, oracle.step(q, k, zero, g, S1z, wq, cos, sin),
+                               rtol=1e-11, atol=1e-13)
+
+
 def test_reset(oracle):
     S = rnd(3, 2, 4, 4)
     r = oracle.reset(S, 1)
