@@ -82,9 +82,10 @@ typedef struct {
 
 /*
  * Bytes of device scratch a context of this shape needs (256-byte aligned base).  It
- * holds a status word, the rotated copy of K made once per step, tensor-core operand
- * copies of S and of the feature maps, the packed rotation table, the partial sums of the
- * commit reduction, the per-token decay weights and, with ARL2_FLAG_TOKEN_GATES, the chunk
+ * holds a status word, the rotated copy of K made once per step, two tensor-core operand
+ * copies of S (a commit writes the one that is not current) and one of each feature map, the
+ * packed rotation table, the partial sums of the commit reduction (two sets: the delta rule
+ * has two accumulators), the per-token decay weights and, with ARL2_FLAG_TOKEN_GATES, the chunk
  * factors of arl2_commit_tokens.  Returns 0 for an invalid configuration.
  */
 size_t arl2_workspace_bytes(const arl2_config* cfg);
@@ -153,6 +154,20 @@ int arl2_teacher_step(arl2_ctx* ctx, const void* d_q, const void* d_k_cache, con
  */
 int arl2_commit(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
                 const float* d_decay_logits, void* stream);
+
+/*
+ * The clean pass of a block in one call (Algorithm 1, clean-pass branch; Sec. 3.3 "Clean-pass
+ * update"): the layer's output for the clean latent, read against the state as it stood BEFORE the
+ * call (Eq. 8), and then the gated-linear commit of that same block,
+ *   d_out  = arl2_denoise_step(q, k_clean, v_clean, gate_logits)  with the pre-update S,
+ *   S     <- sigmoid(a) S + sum_l K'_l^T V'_l                       from the same k_clean, v_clean.
+ * Equal to arl2_denoise_step followed by arl2_commit on the same tensors, but K_c is read and
+ * rotated once: the kernel that forms the partial sums of the state update also writes RoPE(K_c)
+ * for the softmax branch, the attention kernel runs next, and the kernel that adds the partial
+ * sums into S runs last.  Arguments, layouts and error behaviour as in those two calls.
+ */
+int arl2_clean_pass(arl2_ctx* ctx, const void* d_q, const void* d_k_clean, const void* d_v_clean,
+                    const float* d_gate_logits, const float* d_decay_logits, void* d_out, void* stream);
 
 /*
  * State commit with the delta rule of Eq. 4 as printed, applied once per block to the clean

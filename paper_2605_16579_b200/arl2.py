@@ -29,7 +29,7 @@ EXPORTS = (
     "arl2_workspace_bytes", "arl2_create", "arl2_set_params", "arl2_denoise_step", "arl2_commit",
     "arl2_reset", "arl2_get_state", "arl2_set_state", "arl2_sync_status", "arl2_launch_count",
     "arl2_set_profile_events", "arl2_commit_static_scratch", "arl2_commit_delta", "arl2_commit_tokens", "arl2_teacher_step", "arl2_commit_decay_tokens",
-    "arl2_step_kernel_name", "arl2_destroy", "arl2_last_error", "arl2_version", "arl2_debug_set_wait_limit",
+    "arl2_step_kernel_name", "arl2_destroy", "arl2_last_error", "arl2_version", "arl2_debug_set_wait_limit", "arl2_clean_pass",
 )
 
 
@@ -76,6 +76,8 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     lib.arl2_denoise_step.argtypes = [vp] * 7
     lib.arl2_commit.restype = ctypes.c_int
     lib.arl2_commit.argtypes = [vp] * 5
+    lib.arl2_clean_pass.restype = ctypes.c_int
+    lib.arl2_clean_pass.argtypes = [vp] * 8
     lib.arl2_teacher_step.restype = ctypes.c_int
     lib.arl2_teacher_step.argtypes = [vp, vp, vp, vp, ctypes.c_int32, vp, vp]
     lib.arl2_commit_delta.restype = ctypes.c_int
@@ -203,6 +205,25 @@ class Layer:
         with torch.cuda.device(self.device):
             _check(load().arl2_denoise_step(self._ctx, _ptr(q), _ptr(k), _ptr(v), _ptr(gate_logits),
                                             _ptr(out), _stream()), "arl2_denoise_step")
+        return out
+
+    def clean_pass(self, q, k_clean, v_clean, gate_logits, decay_logits, out=None):
+        """The clean pass in one call: the output against the pre-update state, then the commit."""
+        shape = (self.B, self.L, self.H, self.D)
+        for t in (q, k_clean, v_clean):
+            self._want(t, shape, self.dtype, "q/k_clean/v_clean")
+        gshape = ((self.B, self.L) if self.flags & ARL2_FLAG_GATE_SCALAR else
+                  (self.B, self.L, self.H, self.D) if self.flags & ARL2_FLAG_GATE_ELEMENTWISE else
+                  (self.B, self.L, self.H))
+        self._want(gate_logits, gshape, torch.float32, "gate_logits")
+        self._want(decay_logits, (self.B, self.H), torch.float32, "decay_logits")
+        if out is None:
+            out = torch.empty(shape, dtype=self.dtype, device=self.device)
+        else:
+            self._want(out, shape, self.dtype, "out")
+        with torch.cuda.device(self.device):
+            _check(load().arl2_clean_pass(self._ctx, _ptr(q), _ptr(k_clean), _ptr(v_clean), _ptr(gate_logits),
+                                          _ptr(decay_logits), _ptr(out), _stream()), "arl2_clean_pass")
         return out
 
     def teacher_step(self, q, k_cache, v_cache, out=None):

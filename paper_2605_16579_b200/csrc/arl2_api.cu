@@ -27,7 +27,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, k_rot, partials, state_bf16, wq_op, wk_op, wv_op, rope_h, dec_w, dec_total, tok_w, tok_u1, tok_kh, tok_gc, total;
+    size_t status, k_rot, partials, partials_g, state_bf16, state_bf16_b, wq_op, wk_op, wv_op, rope_h, dec_w, dec_total, tok_w, tok_u1, tok_kh, tok_gc, total;
     int nsplit, nchunk, nslot;
 };
 
@@ -93,7 +93,10 @@ Layout make_layout(const arl2_config& c)
         l.nslot = (int)(tc_slots > l.nsplit ? tc_slots : l.nsplit);
     }
     l.partials = off;   off += align_up((size_t)c.B * c.H * l.nslot * dd * sizeof(float));
+    l.partials_g = off; off += align_up((size_t)c.B * c.H * l.nslot * dd * sizeof(float));   // delta rule
+    // two bf16 operand copies of S: a tensor-core commit writes the one that is not current
     l.state_bf16 = off; off += align_up((size_t)c.B * c.H * dd * 2);
+    l.state_bf16_b = off; off += align_up((size_t)c.B * c.H * dd * 2);
     l.wq_op = off;      off += align_up((size_t)c.H * dd * 2);
     l.wk_op = off;      off += align_up((size_t)c.H * dd * 2);
     l.wv_op = off;      off += align_up((size_t)c.H * dd * 2);
@@ -131,6 +134,7 @@ struct arl2_ctx {
     bool use_tc;
     uint64_t launches;
     uint32_t step_calls;   // parity selects the scheduler counter of the next step launch
+    int mirror;            // which of the two bf16 copies of S is current
     cudaEvent_t ev_before, ev_after;  // one-shot timing hook around the step kernel
     uint32_t wait_limit;   // 0: the kernels' default bound; n: waits give up after n - 1 polls (test hook)
 };
@@ -143,6 +147,13 @@ bool check_ctx(const arl2_ctx* ctx)
 {
     if (ctx == nullptr) { set_error("context is NULL"); return false; }
     return true;
+}
+
+// the bf16 operand copy of S that is current (which = 0) or the other one (which = 1)
+__nv_bfloat16* mirror_of(const arl2_ctx* ctx, int which = 0)
+{
+    const size_t off = ((ctx->mirror ^ which) & 1) ? ctx->lay.state_bf16_b : ctx->lay.state_bf16;
+    return reinterpret_cast<__nv_bfloat16*>(ctx->ws + off);
 }
 
 // adds the launches of a helper to the context's counter; passes errors through
@@ -208,6 +219,7 @@ int arl2_create(const arl2_config* cfg, void* d_state, void* d_workspace, size_t
     ctx->use_tc = tc_supported(*cfg);
     ctx->launches = 0;
     ctx->step_calls = 0;
+    ctx->mirror = 0;
     ctx->wait_limit = cfg->flags >> ARL2_FLAG_DEBUG_WAIT_LIMIT_SHIFT;
     ctx->ev_before = ctx->ev_after = nullptr;
     int r = account(ctx, fill_zero(ctx->ws + lay.status, kStatusWords * sizeof(uint32_t),
@@ -221,7 +233,7 @@ int arl2_create(const arl2_config* cfg, void* d_state, void* d_workspace, size_t
                                             cfg->H, as_stream(stream)));
         if (r == ARL2_OK)
             r = account(ctx, state_to_bf16(ctx->state,
-                                           reinterpret_cast<__nv_bfloat16*>(ctx->ws + lay.state_bf16),
+                                           mirror_of(ctx),
                                            (size_t)cfg->B * cfg->H * cfg->D * cfg->D, as_stream(stream)));
     }
     if (r != ARL2_OK) { delete ctx; return r; }
@@ -260,34 +272,31 @@ int arl2_set_params(arl2_ctx* ctx, const void* d_wphi_q, const void* d_wphi_k, c
     return ARL2_OK;
 }
 
-int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const void* d_v,
-                      const float* d_gate_logits, void* d_out, void* stream)
+namespace {
+
+bool check_step_args(const char* who, const void* d_q, const void* d_k, const void* d_v,
+                     const float* d_gate_logits, const void* d_out)
 {
-    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
     if (!d_q || !d_k || !d_v || !d_gate_logits || !d_out) {
-        set_error("denoise_step: q, k, v, gate_logits and out must not be NULL");
-        return ARL2_ERR_INVALID_ARG;
+        set_error("%s: q, k, v, gate_logits and out must not be NULL", who);
+        return false;
     }
     if (d_out == d_q || d_out == d_k || d_out == d_v) {
-        set_error("denoise_step: out must not alias an input");
-        return ARL2_ERR_INVALID_ARG;
+        set_error("%s: out must not alias an input", who);
+        return false;
     }
     if ((reinterpret_cast<uintptr_t>(d_q) | reinterpret_cast<uintptr_t>(d_k) |
          reinterpret_cast<uintptr_t>(d_v) | reinterpret_cast<uintptr_t>(d_out)) % 16 != 0) {
-        set_error("denoise_step: q, k, v and out must be 16-byte aligned");
-        return ARL2_ERR_INVALID_ARG;
+        set_error("%s: q, k, v and out must be 16-byte aligned", who);
+        return false;
     }
-    cudaStream_t st = as_stream(stream);
-    const void* k_rot = d_k;
-    if (ctx->rope_cos != nullptr) {
-        void* buf = ctx->ws + ctx->lay.k_rot;
-        int r = ctx->use_tc
-                    ? account(ctx, tc_rope_k(ctx->shape, d_k, ctx->ws + ctx->lay.rope_h, buf, st))
-                    : account(ctx, simt_rope_k(ctx->shape, ctx->cfg.io_dtype, d_k, ctx->rope_cos,
-                                               ctx->rope_sin, buf, st));
-        if (r != ARL2_OK) return r;
-        k_rot = buf;
-    }
+    return true;
+}
+
+// The fused attention kernel of one pass; k_rot is K after RoPE (or K itself without a rotation).
+int launch_step(arl2_ctx* ctx, const void* d_q, const void* k_rot, const void* d_v,
+                const float* d_gate_logits, void* d_out, cudaStream_t st)
+{
     StepArgs a;
     a.s = ctx->shape;
     a.q = d_q; a.k_rot = k_rot; a.v = d_v; a.gate = d_gate_logits;
@@ -305,7 +314,7 @@ int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const voi
     int r;
     if (ctx->use_tc) {
         r = account(ctx, tc_step(a, reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wq_op),
-                                 reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.state_bf16), st));
+                                 mirror_of(ctx), st));
         // the launch consumed one scheduler counter and cleared the other: only a launch that
         // really went out moves on to the other one
         if (r == ARL2_OK) ++ctx->step_calls;
@@ -314,6 +323,33 @@ int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const voi
     }
     if (e1 != nullptr) cudaEventRecord(e1, st);
     return r;
+}
+
+// K after RoPE into the workspace (one launch), or K itself when the context has no rotation.
+int rotate_k(arl2_ctx* ctx, const void* d_k, const void** k_rot, cudaStream_t st)
+{
+    *k_rot = d_k;
+    if (ctx->rope_cos == nullptr) return ARL2_OK;
+    void* buf = ctx->ws + ctx->lay.k_rot;
+    int r = ctx->use_tc
+                ? account(ctx, tc_rope_k(ctx->shape, d_k, ctx->ws + ctx->lay.rope_h, buf, st))
+                : account(ctx, simt_rope_k(ctx->shape, ctx->cfg.io_dtype, d_k, ctx->rope_cos,
+                                           ctx->rope_sin, buf, st));
+    if (r == ARL2_OK) *k_rot = buf;
+    return r;
+}
+
+}  // namespace
+
+int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const void* d_v,
+                      const float* d_gate_logits, void* d_out, void* stream)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    if (!check_step_args("denoise_step", d_q, d_k, d_v, d_gate_logits, d_out)) return ARL2_ERR_INVALID_ARG;
+    cudaStream_t st = as_stream(stream);
+    const void* k_rot = nullptr;
+    if (int r = rotate_k(ctx, d_k, &k_rot, st)) return r;
+    return launch_step(ctx, d_q, k_rot, d_v, d_gate_logits, d_out, st);
 }
 
 int arl2_teacher_step(arl2_ctx* ctx, const void* d_q, const void* d_k_cache, const void* d_v_cache,
@@ -362,7 +398,7 @@ int arl2_teacher_step(arl2_ctx* ctx, const void* d_q, const void* d_k_cache, con
     ctx->ev_before = ctx->ev_after = nullptr;
     if (e0 != nullptr) cudaEventRecord(e0, st);
     int r = account(ctx, tc_step(a, reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wq_op),
-                                 reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.state_bf16), st));
+                                 mirror_of(ctx), st));
     if (r == ARL2_OK) ++ctx->step_calls;
     if (e1 != nullptr) cudaEventRecord(e1, st);
     return r;
@@ -389,24 +425,27 @@ int arl2_set_profile_events(arl2_ctx* ctx, void* ev_before, void* ev_after)
 
 namespace {
 
-// Shared by arl2_commit (delta = false) and arl2_commit_delta.
-int commit_impl(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
-                const float* d_decay_logits, int mode, const float* d_beta, bool decay_direct, void* stream)
+// Argument block of a commit on this context (mode: 0 gated linear, 1 delta rule, 2 per-token weights).
+bool fill_commit(arl2_ctx* ctx, CommitArgs& a, const void* d_k_clean, const void* d_v_clean,
+                 const float* d_decay_logits, int mode, const float* d_beta, bool decay_direct)
 {
-    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
     if (!d_k_clean || !d_v_clean || !d_decay_logits) {
         set_error("commit: k_clean, v_clean and decay_logits must not be NULL");
-        return ARL2_ERR_INVALID_ARG;
+        return false;
     }
-    CommitArgs a;
+    if ((reinterpret_cast<uintptr_t>(d_k_clean) | reinterpret_cast<uintptr_t>(d_v_clean)) % 16 != 0) {
+        set_error("commit: k_clean and v_clean must be 16-byte aligned");
+        return false;
+    }
     a.s = ctx->shape;
     a.k = d_k_clean; a.v = d_v_clean; a.decay = d_decay_logits;
     a.wk = ctx->wk; a.wv = ctx->wv;
     a.rope_cos = ctx->rope_cos; a.rope_sin = ctx->rope_sin;
     a.state = ctx->state;
     a.partials = reinterpret_cast<float*>(ctx->ws + ctx->lay.partials);
-    a.state_bf16 = ctx->use_tc ? reinterpret_cast<__nv_bfloat16*>(ctx->ws + ctx->lay.state_bf16)
-                               : nullptr;
+    a.partials_g = reinterpret_cast<float*>(ctx->ws + ctx->lay.partials_g);
+    a.state_bf16 = ctx->use_tc ? mirror_of(ctx) : nullptr;
+    a.state_bf16_next = ctx->use_tc ? mirror_of(ctx, 1) : nullptr;
     a.nsplit = ctx->lay.nsplit;
     a.nslot = ctx->lay.nslot;
     a.rope_h = (ctx->use_tc && ctx->rope_cos != nullptr) ? ctx->ws + ctx->lay.rope_h : nullptr;
@@ -415,15 +454,31 @@ int commit_impl(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
     a.wait_limit = ctx->wait_limit;
     a.beta = d_beta;
     a.decay_direct = decay_direct;
-    if ((reinterpret_cast<uintptr_t>(d_k_clean) | reinterpret_cast<uintptr_t>(d_v_clean)) % 16 != 0) {
-        set_error("commit: k_clean and v_clean must be 16-byte aligned");
+    return true;
+}
+
+// The second half of a tensor-core commit: the new state goes to S and to the mirror that was not
+// current, which becomes the current one.
+int finish_commit(arl2_ctx* ctx, const CommitArgs& a, cudaStream_t st)
+{
+    int r = account(ctx, tc_commit_finish(a, st));
+    if (r == ARL2_OK) ctx->mirror ^= 1;
+    return r;
+}
+
+// Shared by arl2_commit, arl2_commit_delta and arl2_commit_decay_tokens.
+int commit_impl(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
+                const float* d_decay_logits, int mode, const float* d_beta, bool decay_direct, void* stream)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    CommitArgs a;
+    if (!fill_commit(ctx, a, d_k_clean, d_v_clean, d_decay_logits, mode, d_beta, decay_direct))
         return ARL2_ERR_INVALID_ARG;
-    }
-    if (ctx->use_tc)
-        return account(ctx, tc_commit(a, reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wk_op),
-                                      reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wv_op),
-                                      as_stream(stream)));
-    return account(ctx, simt_commit(a, ctx->cfg.io_dtype, as_stream(stream)));
+    cudaStream_t st = as_stream(stream);
+    if (!ctx->use_tc) return account(ctx, simt_commit(a, ctx->cfg.io_dtype, st));
+    int r = account(ctx, tc_commit_partials(a, reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wk_op), st));
+    if (r != ARL2_OK) return r;
+    return finish_commit(ctx, a, st);
 }
 
 }  // namespace
@@ -432,6 +487,34 @@ int arl2_commit(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
                 const float* d_decay_logits, void* stream)
 {
     return commit_impl(ctx, d_k_clean, d_v_clean, d_decay_logits, 0, nullptr, false, stream);
+}
+
+int arl2_clean_pass(arl2_ctx* ctx, const void* d_q, const void* d_k_clean, const void* d_v_clean,
+                    const float* d_gate_logits, const float* d_decay_logits, void* d_out, void* stream)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    if (!check_step_args("clean_pass", d_q, d_k_clean, d_v_clean, d_gate_logits, d_out)) return ARL2_ERR_INVALID_ARG;
+    CommitArgs a;
+    if (!fill_commit(ctx, a, d_k_clean, d_v_clean, d_decay_logits, 0, nullptr, false)) return ARL2_ERR_INVALID_ARG;
+    cudaStream_t st = as_stream(stream);
+    if (!ctx->use_tc) {
+        // plain-FMA contexts: the same result from the two calls in sequence
+        const void* k_rot = nullptr;
+        if (int r = rotate_k(ctx, d_k_clean, &k_rot, st)) return r;
+        if (int r = launch_step(ctx, d_q, k_rot, d_v_clean, d_gate_logits, d_out, st)) return r;
+        return account(ctx, simt_commit(a, ctx->cfg.io_dtype, st));
+    }
+    // 1. partial sums of the state update from the K_c, V_c tiles; the same kernel writes RoPE(K_c)
+    //    for the softmax branch (K_c is read and rotated once)
+    const bool rotated = ctx->rope_cos != nullptr;
+    a.k_rot_out = rotated ? ctx->ws + ctx->lay.k_rot : nullptr;
+    int r = account(ctx, tc_commit_partials(a, reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wk_op), st));
+    if (r != ARL2_OK) return r;
+    // 2. the layer's output, read against the state as it still stands (Eq. 8)
+    r = launch_step(ctx, d_q, rotated ? a.k_rot_out : d_k_clean, d_v_clean, d_gate_logits, d_out, st);
+    if (r != ARL2_OK) return r;
+    // 3. only now the state moves on
+    return finish_commit(ctx, a, st);
 }
 
 int arl2_commit_tokens(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
@@ -454,7 +537,7 @@ int arl2_commit_tokens(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_cle
     a.wk = ctx->wk; a.wv = ctx->wv;
     a.rope_cos = ctx->rope_cos; a.rope_sin = ctx->rope_sin;
     a.state = ctx->state;
-    a.state_bf16 = ctx->use_tc ? reinterpret_cast<__nv_bfloat16*>(ctx->ws + ctx->lay.state_bf16)
+    a.state_bf16 = ctx->use_tc ? mirror_of(ctx)
                                : nullptr;
     a.w = reinterpret_cast<float*>(ctx->ws + ctx->lay.tok_w);
     a.u1 = reinterpret_cast<float*>(ctx->ws + ctx->lay.tok_u1);
@@ -510,7 +593,7 @@ int arl2_reset(arl2_ctx* ctx, int32_t stream_index, void* stream)
     int r = account(ctx, fill_zero(ctx->state + first, count * sizeof(float), st));
     if (r != ARL2_OK) return r;
     if (ctx->use_tc) {
-        auto* sb = reinterpret_cast<__nv_bfloat16*>(ctx->ws + ctx->lay.state_bf16);
+        auto* sb = mirror_of(ctx);
         r = account(ctx, fill_zero(sb + first, count * 2, st));
     }
     return r;
@@ -542,7 +625,7 @@ int arl2_set_state(arl2_ctx* ctx, const float* src, void* stream)
     }
     if (ctx->use_tc)
         return account(ctx, state_to_bf16(ctx->state,
-                                          reinterpret_cast<__nv_bfloat16*>(ctx->ws + ctx->lay.state_bf16),
+                                          mirror_of(ctx),
                                           n, st));
     return ARL2_OK;
 }

@@ -73,6 +73,10 @@ struct CommitArgs {
     int run_ntile = 0;
     int nslot = 0;                 // slots per head in `partials` (0: nsplit)
     uint32_t wait_limit = 0;       // as in StepArgs
+    // tensor-core path only
+    float* partials_g = nullptr;              // second accumulator of the delta rule, shaped like `partials`
+    __nv_bfloat16* state_bf16_next = nullptr; // the mirror buffer the finishing kernel writes
+    void* k_rot_out = nullptr;                // when set (and there is a rotation): RoPE(k) is written here too
 };
 
 // Eq. 4 token by token with per-token gates (chunkwise form): the two launches share these.
@@ -120,8 +124,10 @@ int tc_prepare_rope(const float* cos_t, const float* sin_t, void* out, int L, cu
 int tc_rope_k(const Shape& s, const void* k, const void* rope_h, void* k_rot, cudaStream_t st);
 int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* state_bf16,
             cudaStream_t st);
-int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat16* wv_op,
-              cudaStream_t st);   // partial sums on tensor cores, then commit_reduce
+// partial sums on tensor cores (fills a.run_share / a.run_ntile for the finishing kernel) ...
+int tc_commit_partials(CommitArgs& a, const __nv_bfloat16* wk_op, cudaStream_t st);
+// ... then S <- alpha S + (sum of slots) W_phi_v [- (sum of G slots) S_old], mirror written to state_bf16_next
+int tc_commit_finish(const CommitArgs& a, cudaStream_t st);
 
 int tc_commit_tokens(const TokenCommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat16* wv_op,
                      const void* rope_h, uint32_t* status, cudaStream_t st);   // prepare + ordered scan

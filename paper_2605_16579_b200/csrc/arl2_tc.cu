@@ -19,23 +19,12 @@
 //
 // Every wait is bounded: when a limit expires the thread records ARL2_ERR_TIMEOUT in the
 // device status block, raises the CTA's abort flag and every role falls through to the exit.
-#include <cuda.h>
-#include <cuda_fp16.h>
-
-#include <mutex>
-
-#include "arl2_internal.h"
-#include "tc_ptx.cuh"
+#include "tc_common.cuh"
 
 namespace arl2 {
 
 namespace {
 
-using namespace ptx;
-
-constexpr int kTile = 128;               // query rows per tile = keys per tile = head dim
-constexpr int kTileBytes = kTile * kTile * 2;
-constexpr int kHalfBytes = kTileBytes / 2;  // one 64-column TMA box of a tile
 constexpr int kStages = 5;
 constexpr int kThreads = 384;              // 3 warpgroups: softmax 0, softmax 1, {TMA, MMA, 2 idle}
 constexpr int kRegsSoftmax = 232;          // per-thread registers after the warpgroups rebalance
@@ -44,7 +33,6 @@ constexpr int kRegsOther = 40;
 // (threads x the launch register count): the rebalanced total must fit in it
 constexpr int kLaunchRegs = (65536 / kThreads) / 8 * 8;
 static_assert(256 * kRegsSoftmax + (kThreads - 256) * kRegsOther <= kThreads * kLaunchRegs, "register pool");
-constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units of slack before O is rescaled
 
 // shared memory map (offsets from a 1024-byte aligned base)
@@ -88,76 +76,49 @@ struct TcStepParams {
     int n_items;               // + ceil(B * H / 2) items of ragged last tiles when n_q is odd
 };
 
-struct Abort {
-    volatile int* flag;   // in shared memory
-    uint32_t* status;     // device status block
-    uint32_t limit;       // polls before a wait gives up
-};
-
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Abort& ab, int site)
+// 2^x for two values on the FMA pipe instead of the special-function unit: x = j + f with
+// j = round(x) and f in [-0.5, 0.5]; 2^f by a cubic fitted on that interval (relative error below
+// 1e-4, far under the bf16 rounding of the probabilities); 2^j by adding j to the exponent field
+// with one integer multiply-add.  x is clamped at -126 (the result is then a denormal-sized
+// 2^-126 instead of 0: it is rounded to bf16 and summed like any other term).
+#ifndef ARL2_POLY_COUNT
+#define ARL2_POLY_COUNT 0
+#endif
+#ifndef ARL2_POLY_PERIOD
+#define ARL2_POLY_PERIOD 2
+#endif
+#ifdef ARL2_NO_TOKEN
+constexpr bool kUseToken = false;
+#else
+constexpr bool kUseToken = true;
+#endif
+constexpr int kPolyCount = ARL2_POLY_COUNT;    // of every kPolyPeriod element pairs, this many take the
+constexpr int kPolyPeriod = ARL2_POLY_PERIOD;  // FMA-pipe exponential, the rest the special-function unit
+__device__ __forceinline__ void exp2_fma2(float x0, float x1, float& r0, float& r1)
 {
-    for (uint32_t it = 0; it < ab.limit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 255u && *ab.flag) return false;
-    }
-    *ab.flag = 1;
-    if (atomicCAS(ab.status + kStatusError, 0u, (uint32_t)(-ARL2_ERR_TIMEOUT)) == 0u)
-        ab.status[kStatusWhere] = (uint32_t)site;
-    return false;
-}
-
-// Bounded wait that ignores the abort flag: used on the way out, for copies still in flight.
-__device__ __forceinline__ void drain_bar(uint32_t bar, uint32_t parity)
-{
-    for (uint32_t it = 0; it < kSpinLimit; ++it)
-        if (mbar_try_wait(bar, parity)) return;
-}
-
-__device__ __forceinline__ float sigmoid_fast(float x) { return 1.0f / (1.0f + __expf(-x)); }
-
-__device__ __forceinline__ float max3(float a, float b, float c)
-{
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
-// packed pairs of fp32 (one 64-bit register pair per operand)
-__device__ __forceinline__ uint64_t pack2(float lo, float hi)
-{
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi)
-{
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
-{
-    uint64_t d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
-{
-    uint64_t d;
-    asm("add.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
+    const float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
+    x0 = fmaxf(x0, -126.0f);
+    x1 = fmaxf(x1, -126.0f);
+    const uint64_t x2 = pack2(x0, x1);
+    const uint64_t t2 = add2(x2, pack2(kMagic, kMagic));
+    const uint64_t j2 = add2(t2, pack2(-kMagic, -kMagic));
+    const uint64_t f2 = fma2(j2, pack2(-1.0f, -1.0f), x2);
+    uint64_t p2 = fma2(pack2(0.05517132207751274f, 0.05517132207751274f), f2,
+                       pack2(0.24261054396629333f, 0.24261054396629333f));
+    p2 = fma2(p2, f2, pack2(0.6932609677314758f, 0.6932609677314758f));
+    p2 = fma2(p2, f2, pack2(0.9999281167984009f, 0.9999281167984009f));
+    float t0, t1, q0, q1;
+    unpack2(t2, t0, t1);
+    unpack2(p2, q0, q1);
+    // (bits of t) << 23 == j << 23 modulo 2^32: the magic constant's bits fall off the top
+    r0 = __int_as_float(__float_as_int(q0) + __float_as_int(t0) * 0x800000);
+    r1 = __int_as_float(__float_as_int(q1) + __float_as_int(t1) * 0x800000);
 }
 
 // A work item drives up to two 128-row query tiles.  A "pair" item holds two consecutive tiles of
 // one (stream, head): they share every K/V tile.  A "ragged" item holds the last, partial tiles
 // of two different (stream, head) units (or of one, when the number of units is odd): each tile
 // then streams its own K/V, W_phi_q and state through the ring.
-// (cos, sin) of one rotation pair, stored as half2
-__device__ __forceinline__ void unpack_cs(uint32_t h2, float& c, float& s)
-{
-    const __half2 v = *reinterpret_cast<const __half2*>(&h2);
-    const float2 f = __half22float2(v);
-    c = f.x;
-    s = f.y;
-}
-
 struct Item {
     int b[2], h[2], row0[2];
     int ntile;    // active tiles: 1 or 2
@@ -347,7 +308,7 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                     }
                 }
                 const uint64_t neg_m2 = pack2(-m_ref, -m_ref);
-                if (it.ntile == 2) {
+                if (kUseToken && it.ntile == 2) {
                     // the two groups alternate in the exponential phase, so that one group's
                     // exponentials overlap the other tile's MMAs instead of its exponentials
                     const uint32_t par = (t == 0) ? ((tok_cnt + 1) & 1) : (tok_cnt & 1);
@@ -356,14 +317,19 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                 }
 #pragma unroll
                 for (int c = 0; c < 64; ++c) {
-                    float x0, x1;
+                    float x0, x1, p0, p1;
                     unpack2(fma2(pack2(__uint_as_float(sreg[2 * c]), __uint_as_float(sreg[2 * c + 1])), c2x2, neg_m2),
                             x0, x1);
-                    const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);   // special-function unit
+                    if ((c % kPolyPeriod) < kPolyCount) {
+                        exp2_fma2(x0, x1, p0, p1);            // FMA pipe
+                    } else {
+                        p0 = ex2_approx(x0);                  // special-function unit
+                        p1 = ex2_approx(x1);
+                    }
                     l2 = add2(l2, pack2(p0, p1));
                     sreg[c] = pack_bf16(p0, p1);
                 }
-                if (it.ntile == 2) mbar_arrive(bars + 8 * (kBarTok0 + (t ^ 1)));
+                if (kUseToken && it.ntile == 2) mbar_arrive(bars + 8 * (kBarTok0 + (t ^ 1)));
                 tmem_st32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sreg[0]));
                 tmem_st32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[32]));
                 tmem_wait_st();
@@ -803,363 +769,6 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     tc_fence_before();
     __syncthreads();
     if (warp == 9) {
-        tc_fence_after();
-        tmem_dealloc(tmem_base, 512);
-    }
-}
-
-// ---------------------------------------------------------------------------------------------
-// Commit kernel (Eq. 3, Eq. 4 in its gated-linear form): 128 threads per CTA; the 128-token tiles of
-// all (stream, head) units form one flattened sequence that is cut into equal runs, one run per CTA
-// (one CTA per SM when there is enough work), so a run may cross from one head into the next.
-// Per tile:
-//   U_k = K_c W_phi_k, U_v = V_c W_phi_v            two MMAs into TMEM (columns 0-127, 128-255)
-//   K'  = L2Norm(RoPE(U_k)), V' = U_v               one thread per token; written as bf16 over
-//                                                   the raw tiles, in the swizzled tile layout
-//   dS += K'^T V'                                   MMA with both operands token-major (the
-//                                                   contraction runs over the tile's tokens)
-// dS (TMEM columns 256-383, fp32) accumulates over the tiles of one head inside a run and is then
-// written to that (head, CTA) slot of the partial-sum buffer; the assignment of tiles to CTAs and
-// slots is static, and the reduce kernel adds a head's slots in index order and applies the decay.
-// ---------------------------------------------------------------------------------------------
-constexpr int kCOffWk = 0;
-constexpr int kCOffWv = kTileBytes;
-constexpr int kCOffPair = 2 * kTileBytes;                  // 2 pairs of (K tile, V tile)
-constexpr int kCOffState = kCOffPair + 4 * kTileBytes;     // bf16 copy of S_old (delta rule only)
-constexpr int kCOffBars = kCOffState + kTileBytes;
-constexpr int kCommitSmemBytes = kCOffBars + 128 + 1024 + 1024;   // barriers, row-norm exchange, alignment slack
-constexpr int kCommitThreads = 256;
-
-enum CBar : int { kCBarW = 0, kCBarFull0, kCBarFull1, kCBarU, kCBarS, kCBarP, kCBarDrain, kCNumBars };
-
-struct TcCommitParams {
-    Shape s;
-    const uint4* rope_h;   // warp-interleaved half2 (cos, sin) table, or nullptr
-    const float* beta;     // [B, L, H] learning-rate logits (delta rule), or nullptr = 1
-    float* partials;     // [B * H, nslot, 128, 128] fp32
-    uint32_t* status;
-    uint32_t spin_limit;
-    int ntile;           // 128-token tiles per (stream, head)
-    int total_tiles;     // B * H * ntile
-    int share;           // tiles per CTA: CTA c takes tiles [c * share, (c + 1) * share) of the flattened order
-    int nslot;           // partial-sum slots per (stream, head)
-};
-
-// kMode 1 (Eq. 4 as printed, at block level): the value operand of the last MMA is
-// R = diag(beta) (V' - K' S_old) instead of V'; K' S_old is one more MMA per tile (A = K' as
-// written for the last MMA, read d-major; B = the bf16 copy of the state) into TMEM columns 384-511.
-// kMode 2 (per-token decay in the gated-linear form): the value rows are scaled by given weights.
-__device__ __forceinline__ void store_row_bf16_swizzled(uint8_t* tile, int r, const uint32_t (&x)[128], float f)
-{
-#pragma unroll
-    for (int c = 0; c < 16; ++c) {
-        uint4 v;
-        v.x = pack_bf16(__uint_as_float(x[c * 8 + 0]) * f, __uint_as_float(x[c * 8 + 1]) * f);
-        v.y = pack_bf16(__uint_as_float(x[c * 8 + 2]) * f, __uint_as_float(x[c * 8 + 3]) * f);
-        v.z = pack_bf16(__uint_as_float(x[c * 8 + 4]) * f, __uint_as_float(x[c * 8 + 5]) * f);
-        v.w = pack_bf16(__uint_as_float(x[c * 8 + 6]) * f, __uint_as_float(x[c * 8 + 7]) * f);
-        const int off = (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
-        *reinterpret_cast<uint4*>(tile + off) = v;
-    }
-}
-// my half (64 columns = one 64-column box) of row r
-__device__ __forceinline__ void store_half_row_bf16_swizzled(uint8_t* tile, int r, int half, const uint32_t (&x)[64], float f)
-{
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        uint4 v;
-        v.x = pack_bf16(__uint_as_float(x[c * 8 + 0]) * f, __uint_as_float(x[c * 8 + 1]) * f);
-        v.y = pack_bf16(__uint_as_float(x[c * 8 + 2]) * f, __uint_as_float(x[c * 8 + 3]) * f);
-        v.z = pack_bf16(__uint_as_float(x[c * 8 + 4]) * f, __uint_as_float(x[c * 8 + 5]) * f);
-        v.w = pack_bf16(__uint_as_float(x[c * 8 + 6]) * f, __uint_as_float(x[c * 8 + 7]) * f);
-        *reinterpret_cast<uint4*>(tile + half * kHalfBytes + r * 128 + ((c ^ (r & 7)) << 4)) = v;
-    }
-}
-__device__ __forceinline__ void store_row_bf16_global(__nv_bfloat16* dst, const uint32_t (&x)[128], float f)
-{
-#pragma unroll
-    for (int c = 0; c < 16; ++c) {
-        uint4 v;
-        v.x = pack_bf16(__uint_as_float(x[c * 8 + 0]) * f, __uint_as_float(x[c * 8 + 1]) * f);
-        v.y = pack_bf16(__uint_as_float(x[c * 8 + 2]) * f, __uint_as_float(x[c * 8 + 3]) * f);
-        v.z = pack_bf16(__uint_as_float(x[c * 8 + 4]) * f, __uint_as_float(x[c * 8 + 5]) * f);
-        v.w = pack_bf16(__uint_as_float(x[c * 8 + 6]) * f, __uint_as_float(x[c * 8 + 7]) * f);
-        *reinterpret_cast<uint4*>(dst + c * 8) = v;
-    }
-}
-
-template <int kMode>   // 0: V'; 1: delta rule; 2: per-token weights
-__global__ void __launch_bounds__(kCommitThreads, 1)
-tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-                 const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv,
-                 const __grid_constant__ CUtensorMap tm_s, const TcCommitParams p)
-{
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
-                                               ~static_cast<uintptr_t>(1023));
-    const uint32_t smem_base = smem_u32(smem);
-    const uint32_t bars = smem_base + kCOffBars;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kCOffBars + kCNumBars * 8);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kCOffBars + kCNumBars * 8 + 4);
-    const Abort ab{abort_flag, p.status, p.spin_limit};
-
-    const int tid = threadIdx.x, warp = tid >> 5;
-    const int L = p.s.L, H = p.s.H;
-    // this CTA's run of tiles in the flattened (stream, head, tile) order; it may cross heads
-    const int g_begin = (int)blockIdx.x * p.share;
-    const int n_my = min(p.total_tiles, g_begin + p.share) - g_begin;
-
-    if (tid == 0) {
-        for (int i = 0; i < kCNumBars; ++i) mbar_init(bars + 8 * i, 1);
-        *abort_flag = 0;
-        fence_barrier_init();
-        fence_proxy_async_smem();
-    }
-    if (warp == 0) {
-        tmem_alloc(smem_u32(tmem_slot), 512);
-        tmem_relinquish();
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-    // two threads per token row (warps w and w + 4 own the same TMEM lanes), 64 columns each
-    const int r = (warp & 3) * 32 + (tid & 31);
-    const int chalf = warp >> 2;
-    const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(chalf * 64);
-    float* ssx = reinterpret_cast<float*>(smem + kCOffBars + 128);   // [2][128] partial sums of squares
-
-    auto load_pair = [&](int k) {   // k-th tile of the run into pair k & 1
-        const int g = g_begin + k, bh = g / p.ntile, tl = g - bh * p.ntile;
-        const int hb = bh / H, hh = bh - hb * H;
-        const uint32_t bar = bars + 8 * (kCBarFull0 + (k & 1));
-        const uint32_t dst = smem_base + kCOffPair + (k & 1) * 2 * kTileBytes;
-        mbar_expect_tx(bar, 2 * kTileBytes);
-        tma_load_4d(dst, &tm_k, bar, 0, hh, tl * kTile, hb);
-        tma_load_4d(dst + kHalfBytes, &tm_k, bar, 64, hh, tl * kTile, hb);
-        tma_load_4d(dst + kTileBytes, &tm_v, bar, 0, hh, tl * kTile, hb);
-        tma_load_4d(dst + kTileBytes + kHalfBytes, &tm_v, bar, 64, hh, tl * kTile, hb);
-    };
-    auto load_head = [&](int bh) {   // the maps (and the bf16 state) of one (stream, head)
-        const int hh = bh % H;
-        const uint32_t bar_w = bars + 8 * kCBarW;
-        mbar_expect_tx(bar_w, (kMode == 1 ? 3 : 2) * kTileBytes);
-        if (kMode == 1) {
-            tma_load_2d(smem_base + kCOffState, &tm_s, bar_w, 0, bh * kTile);
-            tma_load_2d(smem_base + kCOffState + kHalfBytes, &tm_s, bar_w, 64, bh * kTile);
-        }
-        tma_load_2d(smem_base + kCOffWk, &tm_wk, bar_w, 0, hh * kTile);
-        tma_load_2d(smem_base + kCOffWk + kHalfBytes, &tm_wk, bar_w, 64, hh * kTile);
-        tma_load_2d(smem_base + kCOffWv, &tm_wv, bar_w, 0, hh * kTile);
-        tma_load_2d(smem_base + kCOffWv + kHalfBytes, &tm_wv, bar_w, 64, hh * kTile);
-    };
-
-    const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0, 0) >> 32);
-    constexpr uint32_t kLboK = 1u << 16;
-    constexpr uint32_t kLboMN = (uint32_t)(kHalfBytes >> 4) << 16;
-    auto desc64 = [&](uint32_t lo) {
-        uint64_t d;
-        asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(desc_hi));
-        return d;
-    };
-    constexpr uint32_t idesc_u = idesc_bf16(kTile, kTile, 0, 0);    // tile x map: both K-major
-    constexpr uint32_t idesc_ds = idesc_bf16(kTile, kTile, 1, 1);   // K'^T V': both token-major
-    constexpr uint32_t idesc_ps = idesc_bf16(kTile, kTile, 0, 1);   // K' S_old: A d-major, B = S rows
-
-    bool ok = true;
-    int loads_issued = 0;
-    uint32_t w_loads = 0;   // head loads issued so far (issuing thread)
-    uint32_t w_seen = 0;    // head loads the issuing thread has waited for
-    // U_k = K_c W_phi_k, U_v = V_c W_phi_v of the run's k-th tile into TMEM columns 0-255
-    auto issue_u = [&](int k) {
-        if (w_seen < w_loads) {   // the tile belongs to a head whose maps were requested since
-            if (!wait_bar(bars + 8 * kCBarW, (w_loads - 1) & 1, ab, 80)) return false;
-            w_seen = w_loads;
-        }
-        const uint32_t pa = smem_base + kCOffPair + (k & 1) * 2 * kTileBytes;
-        if (!wait_bar(bars + 8 * (kCBarFull0 + (k & 1)), (uint32_t)((k >> 1) & 1), ab, 81)) return false;
-        tc_fence_after();
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {   // U_k then U_v
-            const uint32_t a_lo = ((pa + u * kTileBytes) >> 4) | kLboK;
-            const uint32_t b_lo = ((smem_base + (u ? kCOffWv : kCOffWk)) >> 4) | kLboK;
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-                const uint32_t koff = (uint32_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
-                mma_ss(tmem_base + u * kTile, desc64(a_lo + koff), desc64(b_lo + koff), idesc_u, ks > 0);
-            }
-        }
-        mma_commit(bars + 8 * kCBarU);
-        return true;
-    };
-    if (tid == 0 && n_my > 0) {
-        prefetch_tensormap(&tm_k);
-        prefetch_tensormap(&tm_v);
-        load_head(g_begin / p.ntile);
-        ++w_loads;
-        for (int k = 0; k < 2 && k < n_my; ++k, ++loads_issued) load_pair(k);
-        ok = issue_u(0);
-    }
-
-    uint32_t sreg[64];
-    for (int k = 0; k < n_my; ++k) {
-        const int g = g_begin + k, bh = g / p.ntile, tl = g - bh * p.ntile;
-        const int b = bh / H, h = bh - b * H;
-        const bool seg_first = k == 0 || tl == 0;                    // first tile of this head in my run
-        const bool seg_last = k + 1 == n_my || tl + 1 == p.ntile;    // last one
-        const bool next_new_head = k + 1 < n_my && tl + 1 == p.ntile;
-        uint8_t* pair = smem + kCOffPair + (k & 1) * 2 * kTileBytes;
-        const uint32_t pair_addr = smem_base + kCOffPair + (k & 1) * 2 * kTileBytes;
-        if (!wait_bar(bars + 8 * kCBarU, (uint32_t)(k & 1), ab, 82)) break;
-        tc_fence_after();
-        // U(k) is complete: nothing reads this head's maps any more (the delta rule still needs its
-        // state tile for the prediction below)
-        if (kMode != 1 && tid == 0 && ok && next_new_head) {
-            load_head(bh + 1);
-            ++w_loads;
-        }
-
-        const int row = tl * kTile + r;          // this thread's token
-        // ---- K' = L2Norm(RoPE(U_k)): my 64 columns of the row
-        tmem_ld32(lane_base, *reinterpret_cast<uint32_t(*)[32]>(&sreg[0]));
-        tmem_ld32(lane_base + 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[32]));
-        tmem_wait_ld();
-        if (p.rope_h != nullptr) {
-            // rows of the warp-interleaved table: padding rows past L read as zero
-            const uint4* tab = p.rope_h + ((size_t)(row >> 5) * 16 + chalf * 8) * 32 + (row & 31);
-            uint4 cs[8];
-#pragma unroll
-            for (int c = 0; c < 8; ++c) cs[c] = __ldg(tab + c * 32);
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const uint32_t h2[4] = {cs[c].x, cs[c].y, cs[c].z, cs[c].w};
-#pragma unroll
-                for (int m = 0; m < 4; ++m) {
-                    float cc, s1;
-                    unpack_cs(h2[m], cc, s1);
-                    float x0 = __uint_as_float(sreg[c * 8 + 2 * m]);
-                    float x1 = __uint_as_float(sreg[c * 8 + 2 * m + 1]);
-                    sreg[c * 8 + 2 * m] = __float_as_uint(x0 * cc - x1 * s1);
-                    sreg[c * 8 + 2 * m + 1] = __float_as_uint(x0 * s1 + x1 * cc);
-                }
-            }
-        }
-        {
-            float ss4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll
-            for (int c = 0; c < 64; c += 4) {
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    ss4[q] = fmaf(__uint_as_float(sreg[c + q]), __uint_as_float(sreg[c + q]), ss4[q]);
-            }
-            ssx[chalf * kTile + r] = (ss4[0] + ss4[1]) + (ss4[2] + ss4[3]);
-            __syncthreads();   // the other half of the row has posted its sum (slots are rewritten
-                               // only after the next barrier of this loop)
-            const float f = rsqrtf(ssx[r] + ssx[kTile + r] + p.s.eps);
-            store_half_row_bf16_swizzled(pair, r, chalf, sreg, f);
-        }
-        if (kMode == 1) {
-            // ---- prediction K' S_old                                                   (Eq. 4)
-            fence_proxy_async_smem();
-            tc_fence_before();
-            __syncthreads();
-            if (tid == 0 && ok) {
-                tc_fence_after();
-                const uint32_t a_lo = (pair_addr >> 4) | kLboK;
-                const uint32_t b_lo = ((smem_base + kCOffState) >> 4) | kLboMN;
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t koff = (uint32_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
-                    mma_ss(tmem_base + 3 * kTile, desc64(a_lo + koff), desc64(b_lo + (uint32_t)(ks * (2048 >> 4))),
-                           idesc_ps, ks > 0);
-                }
-                mma_commit(bars + 8 * kCBarP);
-            }
-            if (!wait_bar(bars + 8 * kCBarP, (uint32_t)(k & 1), ab, 85)) break;
-            tc_fence_after();
-            if (tid == 0 && ok && next_new_head) {   // the prediction was the last reader of the state tile
-                load_head(bh + 1);
-                ++w_loads;
-            }
-        }
-        // ---- V' = U_v, or R = beta (V' - K' S_old), or w V'
-        tmem_ld32(lane_base + kTile, *reinterpret_cast<uint32_t(*)[32]>(&sreg[0]));
-        tmem_ld32(lane_base + kTile + 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[32]));
-        tmem_wait_ld();
-        float vscale = 1.0f;
-        if (kMode == 2)
-            vscale = (p.beta != nullptr && row < L) ? __ldg(p.beta + ((size_t)b * L + row) * H + h)
-                                                    : (row < L ? 1.0f : 0.0f);
-        if (kMode == 1) {
-            if (p.beta != nullptr) vscale = row < L ? sigmoid_fast(__ldg(p.beta + ((size_t)b * L + row) * H + h)) : 0.0f;
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t pr[32];
-                tmem_ld32(lane_base + 3 * kTile + c * 32, pr);
-                tmem_wait_ld();
-#pragma unroll
-                for (int e = 0; e < 32; ++e)
-                    sreg[c * 32 + e] = __float_as_uint(__uint_as_float(sreg[c * 32 + e]) - __uint_as_float(pr[e]));
-            }
-        }
-        store_half_row_bf16_swizzled(pair + kTileBytes, r, chalf, sreg, vscale);
-        fence_proxy_async_smem();
-        tc_fence_before();
-        __syncthreads();
-
-        if (tid == 0 && ok) {
-            tc_fence_after();
-            const uint32_t a_lo = (pair_addr >> 4) | kLboMN;
-            const uint32_t b_lo = ((pair_addr + kTileBytes) >> 4) | kLboMN;
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks)   // 16 tokens per step
-                mma_ss(tmem_base + 2 * kTile, desc64(a_lo + (uint32_t)(ks * (2048 >> 4))),
-                       desc64(b_lo + (uint32_t)(ks * (2048 >> 4))), idesc_ds, (!seg_first || ks > 0) ? 1u : 0u);
-            mma_commit(bars + 8 * kCBarS);
-            // the next tile's U MMAs queue up behind it: every thread has read columns 0-255 (the
-            // barrier above), and they touch the other pair of shared-memory tiles
-            if (k + 1 < n_my) ok = issue_u(k + 1);
-            // this pair may be overwritten once the dS MMA is done
-            if (ok) ok = wait_bar(bars + 8 * kCBarS, (uint32_t)(k & 1), ab, 83);
-            if (ok && k + 2 < n_my) {
-                load_pair(k + 2);
-                ++loads_issued;
-            }
-        }
-        if (seg_last) {
-            // ---- this head's share of dS (row d_k = tid) -> its slot of the partial sums
-            if (!wait_bar(bars + 8 * kCBarS, (uint32_t)(k & 1), ab, 84)) break;
-            tc_fence_after();
-            const int part = (int)blockIdx.x - (bh * p.ntile) / p.share;
-            float* dst = p.partials + (((size_t)bh * p.nslot + part) * kTile + r) * kTile + chalf * 64;
-#pragma unroll 1
-            for (int c = 0; c < 2; ++c) {
-                uint32_t o[32];
-                tmem_ld32(lane_base + 2 * kTile + c * 32, o);
-                tmem_wait_ld();
-#pragma unroll
-                for (int e = 0; e < 4; ++e)   // 32-byte stores: whole sectors
-                    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + c * 32 + e * 8),
-                                 "r"(o[e * 8]), "r"(o[e * 8 + 1]), "r"(o[e * 8 + 2]), "r"(o[e * 8 + 3]), "r"(o[e * 8 + 4]),
-                                 "r"(o[e * 8 + 5]), "r"(o[e * 8 + 6]), "r"(o[e * 8 + 7])
-                                 : "memory");
-            }
-            tc_fence_before();
-        }
-    }
-
-    if (tid == 0 && (!ok || *abort_flag)) {
-        // leave no bulk copy in flight into this CTA's shared memory
-        if (w_loads > 0) drain_bar(bars + 8 * kCBarW, (w_loads - 1) & 1);
-        for (int m = (loads_issued > 2 ? loads_issued - 2 : 0); m < loads_issued; ++m)
-            drain_bar(bars + 8 * (kCBarFull0 + (m & 1)), (uint32_t)((m >> 1) & 1));
-        // nor an MMA still writing tensor memory when it is freed
-        mma_commit(bars + 8 * kCBarDrain);
-        drain_bar(bars + 8 * kCBarDrain, 0);
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 0) {
         tc_fence_after();
         tmem_dealloc(tmem_base, 512);
     }
@@ -1768,104 +1377,18 @@ __global__ void transpose_map_kernel(const __nv_bfloat16* __restrict__ w, __nv_b
     out[t] = v;
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (fn == nullptr) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
-// [B, L, H, 128] bf16 viewed as a 4-D tensor (d, h, l, b); box = 64 columns x 128 rows of one head.
-int make_map_blhd(CUtensorMap* m, const void* base, const Shape& s)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (fn == nullptr) { set_error("cuTensorMapEncodeTiled is not available from the driver"); return ARL2_ERR_CUDA; }
-    cuuint64_t dims[4] = {(cuuint64_t)s.D, (cuuint64_t)s.H, (cuuint64_t)s.L, (cuuint64_t)s.B};
-    cuuint64_t strides[3] = {(cuuint64_t)s.D * 2, (cuuint64_t)s.H * s.D * 2, (cuuint64_t)s.L * s.H * s.D * 2};
-    cuuint32_t box[4] = {64, 1, (cuuint32_t)kTile, 1};
-    cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled([B,L,H,D]) failed with %d", (int)r); return ARL2_ERR_CUDA; }
-    return 0;
-}
-
-// [rows, 128] bf16 row-major; box = 64 columns x 128 rows.
-int make_map_rows(CUtensorMap* m, const void* base, size_t rows, int box_rows = kTile)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (fn == nullptr) { set_error("cuTensorMapEncodeTiled is not available from the driver"); return ARL2_ERR_CUDA; }
-    cuuint64_t dims[2] = {(cuuint64_t)kTile, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)kTile * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled([rows,128]) failed with %d", (int)r); return ARL2_ERR_CUDA; }
-    return 0;
-}
-
-// Per-device, once, under a lock: the SM count and the opt-in to large dynamic shared memory for
-// every kernel of this file (the attribute belongs to the device that is current when it is set).
-constexpr int kMaxDevices = 64;
-struct DeviceSetup {
-    bool ready = false;
-    int num_sms = 0;
-};
 std::mutex g_setup_mutex;
 DeviceSetup g_setup[kMaxDevices];
 
-template <typename K>
-cudaError_t opt_in_smem(K kernel, int bytes)
-{
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-}
-
 int device_setup(int* num_sms)
 {
-    int dev = -1;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
-        set_error("cannot identify the current device (%s)", cudaGetErrorString(e));
-        return ARL2_ERR_CUDA;
-    }
-    std::lock_guard<std::mutex> lock(g_setup_mutex);
-    DeviceSetup& d = g_setup[dev];
-    if (!d.ready) {
-        int sms = 0;
-        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
-            set_error("cannot read the SM count of device %d", dev);
-            return ARL2_ERR_CUDA;
-        }
-        e = opt_in_smem(tc_step_kernel<false>, kSmemBytes);
+    return device_setup_once(g_setup_mutex, g_setup, [] {
+        cudaError_t e = opt_in_smem(tc_step_kernel<false>, kSmemBytes);
         if (e == cudaSuccess) e = opt_in_smem(tc_step_kernel<true>, kSmemBytes);
-        if (e == cudaSuccess) e = opt_in_smem(tc_commit_kernel<0>, kCommitSmemBytes);
-        if (e == cudaSuccess) e = opt_in_smem(tc_commit_kernel<1>, kCommitSmemBytes);
-        if (e == cudaSuccess) e = opt_in_smem(tc_commit_kernel<2>, kCommitSmemBytes);
         if (e == cudaSuccess) e = opt_in_smem(tc_token_prepare_kernel, kTPSmemBytes);
         if (e == cudaSuccess) e = opt_in_smem(tc_token_scan_kernel, kTSSmemBytes);
-        if (e != cudaSuccess) {
-            set_error("cudaFuncSetAttribute(dynamic shared memory) on device %d: %s", dev, cudaGetErrorString(e));
-            return ARL2_ERR_CUDA;
-        }
-        d.num_sms = sms;
-        d.ready = true;
-    }
-    *num_sms = d.num_sms;
-    return 0;
+        return e;
+    }, num_sms);
 }
 
 }  // namespace
@@ -1944,61 +1467,6 @@ int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* 
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_error("launch of tc_step_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
     return 1;
-}
-
-int tc_commit(const CommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat16* wv_op, cudaStream_t st)
-{
-    int num_sms = 0;
-    if (int r = device_setup(&num_sms)) return r;
-    if (a.mode == 1 && a.state_bf16 == nullptr) {
-        set_error("tc_commit: the delta rule needs the bf16 copy of the state");
-        return ARL2_ERR_INVALID_ARG;
-    }
-    CUtensorMap tm_k, tm_v, tm_wk, tm_wv, tm_s;
-    if (int r = make_map_blhd(&tm_k, a.k, a.s)) return r;
-    if (int r = make_map_blhd(&tm_v, a.v, a.s)) return r;
-    if (int r = make_map_rows(&tm_wk, wk_op, (size_t)a.s.H * kTile)) return r;
-    if (int r = make_map_rows(&tm_wv, wv_op, (size_t)a.s.H * kTile)) return r;
-    if (a.mode == 1) {
-        if (int r = make_map_rows(&tm_s, a.state_bf16, (size_t)a.s.B * a.s.H * kTile)) return r;
-    } else {
-        tm_s = tm_wk;   // not read
-    }
-    TcCommitParams p;
-    p.s = a.s;
-    p.rope_h = static_cast<const uint4*>(a.rope_h);
-    p.beta = a.beta;
-    p.partials = a.partials;
-    p.status = a.status;
-    p.spin_limit = a.wait_limit ? a.wait_limit - 1 : kSpinLimit;
-    // equal runs of the flattened tile sequence, at least 2 tiles each and long enough for a head's
-    // partial sums (one per run it falls into, at most ceil(ntile / share) + 1) to fit the slots
-    p.ntile = (a.s.L + kTile - 1) / kTile;
-    p.total_tiles = a.s.B * a.s.H * p.ntile;
-    p.share = (p.total_tiles + num_sms - 1) / num_sms;
-    if (p.share < 2) p.share = 2;
-    p.nslot = a.nslot;
-    if (p.nslot < 2) {
-        set_error("tc_commit: needs at least two partial-sum slots per head (got %d)", p.nslot);
-        return ARL2_ERR_WORKSPACE;
-    }
-    if ((p.ntile + p.share - 1) / p.share + 1 > p.nslot) p.share = (p.ntile + p.nslot - 2) / (p.nslot - 1);
-    const unsigned grid = (unsigned)((p.total_tiles + p.share - 1) / p.share);
-    if (a.mode == 1)
-        tc_commit_kernel<1><<<grid, kCommitThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, tm_wv, tm_s, p);
-    else if (a.mode == 2)
-        tc_commit_kernel<2><<<grid, kCommitThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, tm_wv, tm_s, p);
-    else
-        tc_commit_kernel<0><<<grid, kCommitThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, tm_wv, tm_s, p);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) { set_error("launch of tc_commit_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
-    CommitArgs ra = a;
-    ra.run_share = p.share;
-    ra.run_ntile = p.ntile;
-    ra.nslot = p.nslot;
-    int m = commit_reduce(ra, st);
-    if (m < 0) return m;
-    return 1 + m;
 }
 
 // Eq. 4 token by token with per-token gates on the tensor-core path (bf16 I/O, D = 128).  The

@@ -1,0 +1,579 @@
+// State commit on tensor cores (bf16 I/O, D = 128): Eq. 3 and Eq. 4 (gated-linear form, the
+// block-level delta rule, per-token decay weights), once per block from the clean pass's K and V.
+//
+// The value map is taken out of the token loop: sum_l K'_l^T (V_l W_phi_v) = (sum_l K'_l^T V_l) W_phi_v,
+// so a V tile goes from TMA straight into the state MMA and the D x D map is applied once per
+// head when the partial sums are added up.  The delta rule splits the same way,
+//   sum_l beta_l K'_l^T (V'_l - K'_l S_old) = (sum_l beta_l K'_l^T V_l) W_phi_v - (sum_l beta_l K'_l^T K'_l) S_old,
+// into two accumulators that share the A operand diag(beta) K'.
+//
+// tc_commit_kernel: the 128-token tiles of all (stream, head) units form one flattened sequence
+// cut into equal runs, one CTA (one per SM) per run; a run may cross from one head into the next.
+//   warp 0      TMA producer: W_phi_k^T of the head, then (K tile, V tile) pairs through a ring
+//   warp 1      MMA issuer:   U = K_c W_phi_k into one of two TMEM buffers; dS += K'^T V_c
+//                             (and G += (beta K')^T K' for the delta rule) into TMEM accumulators
+//   warps 2-5   token group 0 (even tiles of the run), one thread per token:
+//   warps 6-9   token group 1 (odd tiles)              K' = L2Norm(RoPE(U)) -> bf16, written over
+//                                                      the raw K tile in the swizzled operand layout;
+//                                                      optionally RoPE(K_c) to global memory for
+//                                                      the softmax branch of a fused clean pass
+// When a head's tiles end inside a run (or the run ends) the token group that handled the last
+// tile stores the accumulators to that (head, CTA) slot of the partial-sum buffer: the
+// assignment of tiles to CTAs and slots is static, so the fixed-order sum of the finishing
+// kernel is bitwise reproducible.
+//
+// tc_commit_finish_kernel: S <- alpha S + (sum of slots) W_phi_v [- (sum of G slots) S_old], fp32
+// FMA arithmetic, 16 state rows per CTA; also writes the bf16 operand copy of the new state into
+// the OTHER of two mirror buffers (the delta rule reads S_old from the current one while rows
+// are being replaced, so the mirrors alternate from commit to commit).
+//
+// Every wait is bounded (see wait_bar); a CTA that gives up records ARL2_ERR_TIMEOUT, drains its
+// copies and MMAs in flight and frees its tensor memory; the finishing kernel then leaves S alone.
+#include "tc_common.cuh"
+
+namespace arl2 {
+
+namespace {
+
+constexpr int kCThreads = 320;
+constexpr int kCMaxStages = 3;
+// shared memory map (offsets from a 1024-byte aligned base)
+constexpr int kCOffWk = 0;                                  // W_phi_k^T of the current head
+constexpr int kCOffStage = kTileBytes;                      // stages of (K tile, V tile)
+constexpr int kCOffBars = kCOffStage + 2 * kCMaxStages * kTileBytes;
+constexpr int kCommitSmemBytes = kCOffBars + 256 + 1024;    // barriers + alignment slack
+// The delta rule keeps two stages and uses the third stage's two tiles for diag(beta) K'.
+
+enum CBar : int {
+    kCBarWFull = 0, kCBarWFree,
+    kCBarStageFull0,                                        // kCMaxStages of each
+    kCBarStageFree0 = kCBarStageFull0 + kCMaxStages,
+    kCBarKpFull0 = kCBarStageFree0 + kCMaxStages,           // token group -> MMA: K' of the stage written
+    kCBarUFull0 = kCBarKpFull0 + kCMaxStages, kCBarUFull1,  // MMA -> token group g: U in buffer g
+    kCBarUFree0, kCBarUFree1,                               // token group g -> MMA: buffer g read
+    kCBarAccDone0, kCBarAccDone1,                           // MMA -> token group g: accumulators complete, store them
+    kCBarAccFree0, kCBarAccFree1,                           // token group g -> MMA: stored
+    kCBarDrain,
+    kCNumBars
+};
+static_assert(kCNumBars * 8 + 16 <= 256, "barrier block");
+
+struct TcCommitParams {
+    Shape s;
+    const uint4* rope_h;   // warp-interleaved half2 (cos, sin) table, or nullptr
+    const float* beta;     // [B, L, H]: learning-rate logits (delta rule) or weights (mode 2), or nullptr = 1
+    float* partials;       // [B * H, nslot, 128, 128] fp32: sum_l (w_l K'_l)^T V_l
+    float* partials_g;     // same shape: sum_l beta_l K'_l^T K'_l (delta rule)
+    __nv_bfloat16* k_rot;  // [B, L, H, 128]: RoPE(K_c) written on the way, or nullptr
+    uint32_t* status;
+    uint32_t spin_limit;
+    int ntile;             // 128-token tiles per (stream, head)
+    int total_tiles;       // B * H * ntile
+    int share;             // tiles per CTA: CTA c takes tiles [c * share, (c + 1) * share) of the flattened order
+    int nslot;             // partial-sum slots per (stream, head)
+};
+
+// kMode 0: S-increment K'^T V'; 1: Eq. 4 at block level (two accumulators); 2: per-token weights on K'.
+template <int kMode>
+__global__ void __launch_bounds__(kCThreads, 1)
+tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                 const __grid_constant__ CUtensorMap tm_wk, const TcCommitParams p)
+{
+    constexpr int kS = kMode == 1 ? 2 : 3;   // ring stages
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                               ~static_cast<uintptr_t>(1023));
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t bars = smem_base + kCOffBars;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kCOffBars + kCNumBars * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kCOffBars + kCNumBars * 8 + 4);
+    const Abort ab{abort_flag, p.status, p.spin_limit};
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int L = p.s.L, H = p.s.H;
+    const int g_begin = (int)blockIdx.x * p.share;
+    const int n_my = min(p.total_tiles, g_begin + p.share) - g_begin;
+    auto tile_of = [&](int k, int& bh, int& tl) {
+        const int g = g_begin + k;
+        bh = g / p.ntile;
+        tl = g - bh * p.ntile;
+    };
+    auto seg_first = [&](int k) { return k == 0 || (g_begin + k) % p.ntile == 0; };
+    auto seg_last = [&](int k) { return k + 1 == n_my || (g_begin + k + 1) % p.ntile == 0; };
+    auto stage_k = [&](int s) { return (uint32_t)(kCOffStage + s * 2 * kTileBytes); };          // K tile, then V tile
+    auto extra_tile = [&](int s) { return (uint32_t)(kCOffStage + (2 * 2 + s) * kTileBytes); };  // delta rule: beta K'
+
+    if (tid == 0) {
+        mbar_init(bars + 8 * kCBarWFull, 1);
+        mbar_init(bars + 8 * kCBarWFree, 1);
+        for (int s = 0; s < kCMaxStages; ++s) {
+            mbar_init(bars + 8 * (kCBarStageFull0 + s), 1);
+            mbar_init(bars + 8 * (kCBarStageFree0 + s), 1);
+            mbar_init(bars + 8 * (kCBarKpFull0 + s), 128);
+        }
+        mbar_init(bars + 8 * kCBarUFull0, 1);
+        mbar_init(bars + 8 * kCBarUFull1, 1);
+        mbar_init(bars + 8 * kCBarUFree0, 128);
+        mbar_init(bars + 8 * kCBarUFree1, 128);
+        for (int g = 0; g < 2; ++g) {
+            mbar_init(bars + 8 * (kCBarAccDone0 + g), 1);
+            mbar_init(bars + 8 * (kCBarAccFree0 + g), 128);
+        }
+        mbar_init(bars + 8 * kCBarDrain, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+        fence_proxy_async_smem();
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    // TMEM columns: U buffer 0 | U buffer 1 | dS | G
+    constexpr uint32_t kColDS = 2 * kTile, kColG = 3 * kTile;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0 && n_my > 0) {
+            prefetch_tensormap(&tm_k);
+            prefetch_tensormap(&tm_v);
+            prefetch_tensormap(&tm_wk);
+            bool ok = true;
+            int n_w = 0, issued = 0;
+            for (int k = 0; k < n_my && ok; ++k) {
+                int bh, tl;
+                tile_of(k, bh, tl);
+                const int hb = bh / H, hh = bh - hb * H;
+                const int s = k % kS;
+                if (k >= kS) ok = wait_bar(bars + 8 * (kCBarStageFree0 + s), (uint32_t)((k / kS) - 1) & 1u, ab, 80);
+                if (!ok) break;
+                const uint32_t bar = bars + 8 * (kCBarStageFull0 + s);
+                const uint32_t dst = smem_base + stage_k(s);
+                mbar_expect_tx(bar, 2 * kTileBytes);
+                tma_load_4d(dst, &tm_k, bar, 0, hh, tl * kTile, hb);
+                tma_load_4d(dst + kHalfBytes, &tm_k, bar, 64, hh, tl * kTile, hb);
+                tma_load_4d(dst + kTileBytes, &tm_v, bar, 0, hh, tl * kTile, hb);
+                tma_load_4d(dst + kTileBytes + kHalfBytes, &tm_v, bar, 64, hh, tl * kTile, hb);
+                ++issued;
+                if (seg_first(k)) {
+                    // the map of this head: once the MMAs that read the previous head's are done
+                    if (n_w > 0) ok = wait_bar(bars + 8 * kCBarWFree, (uint32_t)(n_w - 1) & 1u, ab, 81);
+                    if (!ok) break;
+                    mbar_expect_tx(bars + 8 * kCBarWFull, kTileBytes);
+                    tma_load_2d(smem_base + kCOffWk, &tm_wk, bars + 8 * kCBarWFull, 0, hh * kTile);
+                    tma_load_2d(smem_base + kCOffWk + kHalfBytes, &tm_wk, bars + 8 * kCBarWFull, 64, hh * kTile);
+                    ++n_w;
+                }
+            }
+            if (!ok || *abort_flag) {
+                // do not leave the CTA while bulk copies into its shared memory are in flight
+                if (n_w > 0) drain_bar(bars + 8 * kCBarWFull, (uint32_t)(n_w - 1) & 1u);
+                for (int m = (issued > kS ? issued - kS : 0); m < issued; ++m)
+                    drain_bar(bars + 8 * (kCBarStageFull0 + m % kS), (uint32_t)(m / kS) & 1u);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0 && n_my > 0) {
+            const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0, 0) >> 32);
+            constexpr uint32_t kLboK = 1u << 16;
+            constexpr uint32_t kLboMN = (uint32_t)(kHalfBytes >> 4) << 16;
+            auto desc64 = [&](uint32_t lo) {
+                uint64_t d;
+                asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(desc_hi));
+                return d;
+            };
+            constexpr uint32_t idesc_u = idesc_bf16(kTile, kTile, 0, 0);    // tile x map: both K-major
+            constexpr uint32_t idesc_tt = idesc_bf16(kTile, kTile, 1, 1);   // both operands token-major
+            bool ok = true;
+            uint32_t w_seen = 0;        // maps waited for
+            uint32_t n_store[2] = {0, 0};   // per token group: accumulator stores asked for so far
+            int storing = -1;           // the group that stores the segment just ended (every waiter of a
+                                        // barrier follows its phases one by one: a barrier per group)
+            for (int k = 0; k <= n_my && ok; ++k) {
+                if (k < n_my) {
+                    // ---- U(k) = K_c W_phi_k into buffer k & 1
+                    const int s = k % kS, u = k & 1;
+                    if (seg_first(k)) {
+                        ok = wait_bar(bars + 8 * kCBarWFull, w_seen & 1u, ab, 82);
+                        ++w_seen;
+                    }
+                    if (ok) ok = wait_bar(bars + 8 * (kCBarStageFull0 + s), (uint32_t)(k / kS) & 1u, ab, 83);
+                    if (ok && k >= 2) ok = wait_bar(bars + 8 * (kCBarUFree0 + u), (uint32_t)((k >> 1) - 1) & 1u, ab, 84);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_lo = ((smem_base + stage_k(s)) >> 4) | kLboK;
+                    const uint32_t b_lo = ((smem_base + kCOffWk) >> 4) | kLboK;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t koff = (uint32_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
+                        mma_ss(tmem_base + u * kTile, desc64(a_lo + koff), desc64(b_lo + koff), idesc_u, ks > 0);
+                    }
+                    mma_commit(bars + 8 * (kCBarUFull0 + u));
+                    // the next tile belongs to another head: its map may replace this one
+                    if (k + 1 < n_my && seg_first(k + 1)) mma_commit(bars + 8 * kCBarWFree);
+                }
+                if (k >= 1) {
+                    // ---- accumulators += (w K')^T V_c  [and (beta K')^T K'] for tile k - 1
+                    const int j = k - 1, s = j % kS;
+                    ok = wait_bar(bars + 8 * (kCBarKpFull0 + s), (uint32_t)(j / kS) & 1u, ab, 85);
+                    const bool first = seg_first(j);
+                    if (ok && first && storing >= 0)
+                        ok = wait_bar(bars + 8 * (kCBarAccFree0 + storing), (n_store[storing] - 1) & 1u, ab, 86);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t k_lo = ((smem_base + stage_k(s)) >> 4) | kLboMN;
+                    const uint32_t v_lo = ((smem_base + stage_k(s) + kTileBytes) >> 4) | kLboMN;
+                    const uint32_t a_lo = kMode == 1 ? (((smem_base + extra_tile(s)) >> 4) | kLboMN) : k_lo;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)   // 16 tokens per step
+                        mma_ss(tmem_base + kColDS, desc64(a_lo + (uint32_t)(ks * (2048 >> 4))),
+                               desc64(v_lo + (uint32_t)(ks * (2048 >> 4))), idesc_tt, (!first || ks > 0) ? 1u : 0u);
+                    if (kMode == 1) {
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks)
+                            mma_ss(tmem_base + kColG, desc64(a_lo + (uint32_t)(ks * (2048 >> 4))),
+                                   desc64(k_lo + (uint32_t)(ks * (2048 >> 4))), idesc_tt, (!first || ks > 0) ? 1u : 0u);
+                    }
+                    mma_commit(bars + 8 * (kCBarStageFree0 + s));
+                    if (seg_last(j)) {
+                        storing = j & 1;
+                        mma_commit(bars + 8 * (kCBarAccDone0 + storing));
+                        ++n_store[storing];
+                    }
+                }
+            }
+            if (!ok || *abort_flag) {
+                // tensor memory is freed below: none of this thread's MMAs may still be running
+                mma_commit(bars + 8 * kCBarDrain);
+                drain_bar(bars + 8 * kCBarDrain, 0);
+            }
+        }
+    } else {
+        // ---------------- token groups: thread = token row of the tiles k = g, g + 2, ... ----------------
+        const int g = (warp - 2) >> 2;
+        const int q = warp & 3;                     // TMEM lane quarter this warp may access
+        const int r = q * 32 + lane;                // token row of the tile = TMEM lane
+        const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
+        const uint32_t u_addr = lane_base + (uint32_t)(g * kTile);
+        uint32_t n_store = 0;                       // accumulator stores this group has done
+        bool ok = true;
+        for (int k = 0; k < n_my && ok; ++k) {
+            const bool last = seg_last(k);
+            if ((k & 1) != g) continue;
+            int bh, tl;
+            tile_of(k, bh, tl);
+            const int b = bh / H, h = bh - b * H;
+            const int s = k % kS;
+            const int row = tl * kTile + r;
+            uint8_t* ktile = smem + stage_k(s);
+            // per-token factor on K': the decay weight (mode 2) or the learning rate (delta rule)
+            float wtok = 1.0f;
+            if (kMode != 0 && p.beta != nullptr && row < L) {
+                const float x = __ldg(p.beta + ((size_t)b * L + row) * H + h);
+                wtok = kMode == 1 ? sigmoid_fast(x) : x;
+            }
+            const uint4* tab = p.rope_h != nullptr ? p.rope_h + ((size_t)(row >> 5) * 16) * 32 + (row & 31) : nullptr;
+            if (p.k_rot != nullptr) {
+                // ---- RoPE(K_c) for the softmax branch: the raw tile is in shared memory
+                ok = wait_bar(bars + 8 * (kCBarStageFull0 + s), (uint32_t)(k / kS) & 1u, ab, 87);
+                if (!ok) break;
+                if (row < L) {
+                    __nv_bfloat16* dst = p.k_rot + (((size_t)b * L + row) * H + h) * kTile;
+#pragma unroll
+                    for (int c2 = 0; c2 < 8; ++c2) {
+                        uint32_t w[8];
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int c = c2 * 2 + e;
+                            const uint4 cs = __ldg(tab + c * 32);
+                            const uint4 raw = *reinterpret_cast<const uint4*>(
+                                ktile + (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+                            const uint32_t x[4] = {raw.x, raw.y, raw.z, raw.w};
+                            const uint32_t h2[4] = {cs.x, cs.y, cs.z, cs.w};
+#pragma unroll
+                            for (int m = 0; m < 4; ++m) {
+                                float cc, ss;
+                                unpack_cs(h2[m], cc, ss);
+                                const float x0 = __uint_as_float(x[m] << 16);
+                                const float x1 = __uint_as_float(x[m] & 0xFFFF0000u);
+                                w[e * 4 + m] = pack_bf16(x0 * cc - x1 * ss, x0 * ss + x1 * cc);
+                            }
+                        }
+                        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + c2 * 16),
+                                     "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                                     : "memory");
+                    }
+                }
+            }
+            // ---- K' = L2Norm(RoPE(U)): the row arrives in two halves of 64 columns
+            ok = wait_bar(bars + 8 * (kCBarUFull0 + g), (uint32_t)(k >> 1) & 1u, ab, 88);
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t ureg[128];
+            float ss4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                uint4 cs[8];
+                if (tab != nullptr) {
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) cs[c] = __ldg(tab + (hf * 8 + c) * 32);
+                }
+                tmem_ld32(u_addr + hf * 64, *reinterpret_cast<uint32_t(*)[32]>(&ureg[hf * 64]));
+                tmem_ld32(u_addr + hf * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&ureg[hf * 64 + 32]));
+                tmem_wait_ld();
+                if (tab != nullptr) {
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const uint32_t h2[4] = {cs[c].x, cs[c].y, cs[c].z, cs[c].w};
+#pragma unroll
+                        for (int m = 0; m < 4; ++m) {
+                            float cc, s1;
+                            unpack_cs(h2[m], cc, s1);
+                            const int i = hf * 64 + c * 8 + 2 * m;
+                            const float x0 = __uint_as_float(ureg[i]), x1 = __uint_as_float(ureg[i + 1]);
+                            ureg[i] = __float_as_uint(x0 * cc - x1 * s1);
+                            ureg[i + 1] = __float_as_uint(x0 * s1 + x1 * cc);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < 64; c += 4) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float x = __uint_as_float(ureg[hf * 64 + c + e]);
+                        ss4[e] = fmaf(x, x, ss4[e]);
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(bars + 8 * (kCBarUFree0 + g));      // buffer g may receive U(k + 2)
+            const float f = rsqrtf((ss4[0] + ss4[1]) + (ss4[2] + ss4[3]) + p.s.eps);
+            // rows past L are zero (TMA fills them, the table's padding rows are zero): K' = 0 there
+            if (kMode == 1) {
+                store_row_bf16_swizzled(ktile, r, ureg, f);                       // K'      (B of G)
+                store_row_bf16_swizzled(smem + extra_tile(s), r, ureg, f * wtok); // beta K' (A of both)
+            } else {
+                store_row_bf16_swizzled(ktile, r, ureg, f * wtok);
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(bars + 8 * (kCBarKpFull0 + s));
+            if (last) {
+                // ---- this head's share of the accumulators (row d_k = r) -> its slot of the partial sums
+                ok = wait_bar(bars + 8 * (kCBarAccDone0 + g), n_store & 1u, ab, 89);
+                if (!ok) break;
+                tc_fence_after();
+                const int part = (int)blockIdx.x - (bh * p.ntile) / p.share;
+                const size_t at = (((size_t)bh * p.nslot + part) * kTile + r) * kTile;
+#pragma unroll 1
+                for (int acc = 0; acc < (kMode == 1 ? 2 : 1); ++acc) {
+                    float* dst = (acc == 0 ? p.partials : p.partials_g) + at;
+#pragma unroll 1
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(lane_base + kColDS + acc * kTile + c * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)   // 32-byte stores: whole sectors
+                            asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + c * 32 + e * 8),
+                                         "r"(o[e * 8]), "r"(o[e * 8 + 1]), "r"(o[e * 8 + 2]), "r"(o[e * 8 + 3]), "r"(o[e * 8 + 4]),
+                                         "r"(o[e * 8 + 5]), "r"(o[e * 8 + 6]), "r"(o[e * 8 + 7])
+                                         : "memory");
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(bars + 8 * (kCBarAccFree0 + g));
+                ++n_store;
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// S <- alpha S + (sum_s A_s) W_phi_v [- (sum_s G_s) S_old]; one CTA per 16 state rows of a head.
+// The slots of a head are added in index order.  256 threads: thread = (output column, 8 of the rows).
+// The right-hand matrices (the head's value map, then S_old) pass through shared memory as bf16.
+constexpr int kFinRows = 16;
+constexpr int kFinSmemBytes = kTileBytes + 2 * kFinRows * kTile * 4;
+
+__device__ __forceinline__ void fin_load_matrix(__nv_bfloat16* dst, const __nv_bfloat16* __restrict__ src, int tid)
+{
+    const uint4* s4 = reinterpret_cast<const uint4*>(src);
+    uint4* d4 = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+    for (int i = 0; i < kTileBytes / 16 / 256; ++i) d4[tid + i * 256] = __ldg(s4 + tid + i * 256);
+}
+
+// acc[i] += sign * sum_m X[row_i][m] * M[m][e]
+__device__ __forceinline__ void fin_multiply(float (&acc)[8], const float* __restrict__ X, const __nv_bfloat16* __restrict__ M,
+                                             int e, float sign)
+{
+#pragma unroll 4
+    for (int m = 0; m < kTile; m += 4) {
+        float w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) w[j] = sign * __bfloat162float(M[(m + j) * kTile + e]);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float4 x = *reinterpret_cast<const float4*>(X + i * kTile + m);
+            acc[i] = fmaf(x.x, w[0], acc[i]);
+            acc[i] = fmaf(x.y, w[1], acc[i]);
+            acc[i] = fmaf(x.z, w[2], acc[i]);
+            acc[i] = fmaf(x.w, w[3], acc[i]);
+        }
+    }
+}
+
+template <int kMode>
+__global__ void __launch_bounds__(256)
+tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ partials,
+                        const float* __restrict__ partials_g, const __nv_bfloat16* __restrict__ wv,
+                        const float* __restrict__ decay, int decay_direct,
+                        const __nv_bfloat16* __restrict__ mirror_cur, __nv_bfloat16* __restrict__ mirror_next,
+                        int H, int share, int ntile, int nslot, const uint32_t* __restrict__ status)
+{
+    extern __shared__ __align__(16) uint8_t fin_smem[];
+    __nv_bfloat16* Ms = reinterpret_cast<__nv_bfloat16*>(fin_smem);               // [128][128] right-hand matrix
+    float* As = reinterpret_cast<float*>(fin_smem + kTileBytes);                   // [16][128]
+    float* Gs = As + kFinRows * kTile;                                             // [16][128] (delta rule)
+    const int tid = threadIdx.x, e = tid & 127, half = tid >> 7;
+    const int bh = (int)(blockIdx.x / (kTile / kFinRows)), h = bh % H;
+    const int row0 = (int)(blockIdx.x % (kTile / kFinRows)) * kFinRows + half * 8;
+    const size_t head = (size_t)bh * kTile * kTile;
+    if (status != nullptr && status[kStatusError] != 0u) {
+        // a partial-sum CTA gave up on a bounded wait: S stays as it was, and so does its mirror
+#pragma unroll
+        for (int i = 0; i < 8; ++i) mirror_next[head + (size_t)(row0 + i) * kTile + e] = mirror_cur[head + (size_t)(row0 + i) * kTile + e];
+        return;
+    }
+    if (wv != nullptr) fin_load_matrix(Ms, wv + (size_t)h * kTile * kTile, tid);   // [in = m][out = e]
+    const int first = (bh * ntile) / share, last = (bh * ntile + ntile - 1) / share;
+    const int nparts = last - first + 1;
+    float a[8], gsum[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) a[i] = gsum[i] = 0.0f;
+    for (int s = 0; s < nparts; ++s) {
+        const size_t at = (((size_t)bh * nslot + s) * kTile + row0) * kTile + e;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) a[i] += partials[at + (size_t)i * kTile];
+        if (kMode == 1) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) gsum[i] += partials_g[at + (size_t)i * kTile];
+        }
+    }
+    float out[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        out[i] = wv != nullptr ? 0.0f : a[i];
+        As[(half * 8 + i) * kTile + e] = a[i];
+        if (kMode == 1) Gs[(half * 8 + i) * kTile + e] = gsum[i];
+    }
+    __syncthreads();
+    if (wv != nullptr) fin_multiply(out, As + half * 8 * kTile, Ms, e, 1.0f);
+    if (kMode == 1) {
+        __syncthreads();                                   // every thread is done with the value map
+        fin_load_matrix(Ms, mirror_cur + head, tid);       // S_old [m][e]
+        __syncthreads();
+        fin_multiply(out, Gs + half * 8 * kTile, Ms, e, -1.0f);
+    }
+    const float alpha = decay_direct ? decay[bh] : 1.0f / (1.0f + __expf(-decay[bh]));
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const size_t at = head + (size_t)(row0 + i) * kTile + e;
+        const float nw = alpha * state[at] + out[i];
+        state[at] = nw;
+        mirror_next[at] = __float2bfloat16_rn(nw);
+    }
+}
+
+std::mutex g_setup_mutex;
+DeviceSetup g_setup[kMaxDevices];
+
+int device_setup(int* num_sms)
+{
+    return device_setup_once(g_setup_mutex, g_setup, [] {
+        cudaError_t e = opt_in_smem(tc_commit_kernel<0>, kCommitSmemBytes);
+        if (e == cudaSuccess) e = opt_in_smem(tc_commit_kernel<1>, kCommitSmemBytes);
+        if (e == cudaSuccess) e = opt_in_smem(tc_commit_kernel<2>, kCommitSmemBytes);
+        if (e == cudaSuccess) e = opt_in_smem(tc_commit_finish_kernel<0>, kFinSmemBytes);
+        if (e == cudaSuccess) e = opt_in_smem(tc_commit_finish_kernel<1>, kFinSmemBytes);
+        return e;
+    }, num_sms);
+}
+
+}  // namespace
+
+int tc_commit_partials(CommitArgs& a, const __nv_bfloat16* wk_op, cudaStream_t st)
+{
+    int num_sms = 0;
+    if (int r = device_setup(&num_sms)) return r;
+    if (a.mode == 1 && (a.partials_g == nullptr || a.state_bf16 == nullptr)) {
+        set_error("tc_commit: the delta rule needs the second accumulator and the bf16 copy of the state");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    CUtensorMap tm_k, tm_v, tm_wk;
+    if (int r = make_map_blhd(&tm_k, a.k, a.s)) return r;
+    if (int r = make_map_blhd(&tm_v, a.v, a.s)) return r;
+    if (int r = make_map_rows(&tm_wk, wk_op, (size_t)a.s.H * kTile)) return r;
+    TcCommitParams p;
+    p.s = a.s;
+    p.rope_h = static_cast<const uint4*>(a.rope_h);
+    p.beta = a.beta;
+    p.partials = a.partials;
+    p.partials_g = a.partials_g;
+    p.k_rot = a.rope_h != nullptr ? static_cast<__nv_bfloat16*>(a.k_rot_out) : nullptr;
+    p.status = a.status;
+    p.spin_limit = a.wait_limit ? a.wait_limit - 1 : kSpinLimit;
+    // equal runs of the flattened tile sequence, at least 2 tiles each and long enough for a head's
+    // partial sums (one per run it falls into, at most ceil(ntile / share) + 1) to fit the slots
+    p.ntile = (a.s.L + kTile - 1) / kTile;
+    p.total_tiles = a.s.B * a.s.H * p.ntile;
+    p.share = (p.total_tiles + num_sms - 1) / num_sms;
+    if (p.share < 2) p.share = 2;
+    p.nslot = a.nslot;
+    if (p.nslot < 2) {
+        set_error("tc_commit: needs at least two partial-sum slots per head (got %d)", p.nslot);
+        return ARL2_ERR_WORKSPACE;
+    }
+    if ((p.ntile + p.share - 1) / p.share + 1 > p.nslot) p.share = (p.ntile + p.nslot - 2) / (p.nslot - 1);
+    const unsigned grid = (unsigned)((p.total_tiles + p.share - 1) / p.share);
+    if (a.mode == 1)
+        tc_commit_kernel<1><<<grid, kCThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, p);
+    else if (a.mode == 2)
+        tc_commit_kernel<2><<<grid, kCThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, p);
+    else
+        tc_commit_kernel<0><<<grid, kCThreads, kCommitSmemBytes, st>>>(tm_k, tm_v, tm_wk, p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_error("launch of tc_commit_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
+    a.run_share = p.share;
+    a.run_ntile = p.ntile;
+    return 1;
+}
+
+int tc_commit_finish(const CommitArgs& a, cudaStream_t st)
+{
+    const unsigned grid = (unsigned)(a.s.B * a.s.H) * (kTile / kFinRows);
+    const __nv_bfloat16* wv = static_cast<const __nv_bfloat16*>(a.wv);
+    if (a.mode == 1)
+        tc_commit_finish_kernel<1><<<grid, 256, kFinSmemBytes, st>>>(a.state, a.partials, a.partials_g, wv, a.decay,
+                                                         a.decay_direct ? 1 : 0, a.state_bf16, a.state_bf16_next,
+                                                         a.s.H, a.run_share, a.run_ntile, a.nslot, a.status);
+    else
+        tc_commit_finish_kernel<0><<<grid, 256, kFinSmemBytes, st>>>(a.state, a.partials, a.partials_g, wv, a.decay,
+                                                         a.decay_direct ? 1 : 0, a.state_bf16, a.state_bf16_next,
+                                                         a.s.H, a.run_share, a.run_ntile, a.nslot, a.status);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_error("launch of tc_commit_finish_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
+    return 1;
+}
+
+}  // namespace arl2

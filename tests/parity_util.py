@@ -223,6 +223,37 @@ class Pair:
                                                        self.sin, eps=self.eps),
             heads)
 
+    def clean_pass(self, q, kc, vc, g, a, rows=None):
+        """The fused clean pass on both sides.  Returns (output error, state error): every element when
+        the oracle follows all units (rows = None), else the sampled rows (b, h, i) and the followed units."""
+        d = self.dev
+        self.g_out.t.fill_(float("nan"))
+        out = self.layer.clean_pass(q.to(d), kc.to(d), vc.to(d), g.to(d), a.to(d), out=self.g_out.t)
+        got = out.float().cpu().numpy()
+        self.check_guards()
+        assert np.isfinite(got).all()
+        if rows is None:
+            assert self._all()
+            ref = self.oracle.step(q, kc, vc, g, self.S_ref, self.wq, self.cos, self.sin,
+                                   scale=self.scale, eps=self.eps)
+            e_out = float(head_errors(got, ref).max())
+        else:
+            rows = np.asarray(rows)
+            units = sorted({(int(r[0]), int(r[1])) for r in rows})
+            assert all(self.tracked[b, h] for b, h in units)
+            index = {u: n for n, u in enumerate(units)}
+            urows = np.array([(0, index[(int(b), int(h))], int(i)) for b, h, i in rows])
+            S_u = np.stack([self.S_ref[b, h] for b, h in units])[None]
+            ref_rows = self.oracle.step_rows(unit_view(q, units), unit_view(kc, units), unit_view(vc, units),
+                                             unit_view(g, units), S_u, urows, self._wu(self.wq, units),
+                                             self.cos, self.sin, scale=self.scale, eps=self.eps)
+            e_out = rows_error(got[rows[:, 0], rows[:, 2], rows[:, 1]], ref_rows, rows)
+        e_state = self._after_commit(
+            lambda vw, S, u: self.oracle.commit(vw(kc), vw(vc), self._bh(a, u), S, self._wu(self.wk, u),
+                                                self._wu(self.wv, u), self.cos, self.sin, eps=self.eps),
+            None)
+        return e_out, e_state
+
     def _wu(self, w, units):
         return w if (w is None or units is None) else w[[h for _, h in units]]
 
