@@ -10,17 +10,16 @@
 // tc_commit_kernel: the 128-token tiles of all (stream, head) units form one flattened sequence
 // cut into equal runs, one CTA (one per SM) per run; a run may cross from one head into the next.
 //   warp 0      TMA producer: W_phi_k^T of the head, then (K tile, V tile) pairs through a ring
-//   warp 1      MMA issuer:   U = K_c W_phi_k into one of two TMEM buffers; dS += K'^T V_c
-//                             (and G += (beta K')^T K' for the delta rule) into TMEM accumulators
-//   warps 2-5   token group 0 (even tiles of the run), one thread per token:
-//   warps 6-9   token group 1 (odd tiles)              K' = L2Norm(RoPE(U)) -> bf16, written over
-//                                                      the raw K tile in the swizzled operand layout;
-//                                                      optionally RoPE(K_c) to global memory for
-//                                                      the softmax branch of a fused clean pass
-// When a head's tiles end inside a run (or the run ends) the token group that handled the last
-// tile stores the accumulators to that (head, CTA) slot of the partial-sum buffer: the
-// assignment of tiles to CTAs and slots is static, so the fixed-order sum of the finishing
-// kernel is bitwise reproducible.
+//   warp 1      MMA issuer:   U = K_c W_phi_k into one of two TMEM buffers
+//   warp 10     MMA issuer:   dS += K'^T V_c (and G += (beta K')^T K' for the delta rule) into TMEM
+//                             accumulators
+//   warps 2-9   token threads, two per token (64 of the 128 columns each):
+//                             K' = L2Norm(RoPE(U)) -> bf16, written over the raw K tile in the
+//                             swizzled operand layout; optionally RoPE(K_c) to global memory for
+//                             the softmax branch of a fused clean pass
+// When a head's tiles end inside a run (or the run ends) the token threads store the accumulators
+// to that (head, CTA) slot of the partial-sum buffer: the assignment of tiles to CTAs and slots is
+// static, so the fixed-order sum of the finishing kernel is bitwise reproducible.
 //
 // tc_commit_finish_kernel: S <- alpha S + (sum of slots) W_phi_v [- (sum of G slots) S_old], fp32
 // FMA arithmetic, 16 state rows per CTA; also writes the bf16 operand copy of the new state into
@@ -35,7 +34,8 @@ namespace arl2 {
 
 namespace {
 
-constexpr int kCThreads = 320;
+constexpr int kCThreads = 352;        // producer, U issuer, 8 token warps, accumulator issuer
+constexpr int kCTokenThreads = 256;
 constexpr int kCMaxStages = 3;
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int kCOffWk = 0;                                  // W_phi_k^T of the current head
@@ -48,12 +48,11 @@ enum CBar : int {
     kCBarWFull = 0, kCBarWFree,
     kCBarStageFull0,                                        // kCMaxStages of each
     kCBarStageFree0 = kCBarStageFull0 + kCMaxStages,
-    kCBarKpFull0 = kCBarStageFree0 + kCMaxStages,           // token group -> MMA: K' of the stage written
-    kCBarUFull0 = kCBarKpFull0 + kCMaxStages, kCBarUFull1,  // MMA -> token group g: U in buffer g
-    kCBarUFree0, kCBarUFree1,                               // token group g -> MMA: buffer g read
-    kCBarAccDone0, kCBarAccDone1,                           // MMA -> token group g: accumulators complete, store them
-    kCBarAccFree0, kCBarAccFree1,                           // token group g -> MMA: stored
-    kCBarDrain,
+    kCBarKpFull0 = kCBarStageFree0 + kCMaxStages,           // token threads -> MMA: K' of the stage written
+    kCBarUFull0 = kCBarKpFull0 + kCMaxStages, kCBarUFull1,  // MMA -> token threads: U in buffer 0 / 1
+    kCBarUFree0, kCBarUFree1,                               // token threads -> MMA: buffer read
+    kCBarAccDone, kCBarAccFree,                             // accumulators complete: store them / stored
+    kCBarDrain0, kCBarDrain1,
     kCNumBars
 };
 static_assert(kCNumBars * 8 + 16 <= 256, "barrier block");
@@ -109,17 +108,16 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         for (int s = 0; s < kCMaxStages; ++s) {
             mbar_init(bars + 8 * (kCBarStageFull0 + s), 1);
             mbar_init(bars + 8 * (kCBarStageFree0 + s), 1);
-            mbar_init(bars + 8 * (kCBarKpFull0 + s), 128);
+            mbar_init(bars + 8 * (kCBarKpFull0 + s), kCTokenThreads);
         }
         mbar_init(bars + 8 * kCBarUFull0, 1);
         mbar_init(bars + 8 * kCBarUFull1, 1);
-        mbar_init(bars + 8 * kCBarUFree0, 128);
-        mbar_init(bars + 8 * kCBarUFree1, 128);
-        for (int g = 0; g < 2; ++g) {
-            mbar_init(bars + 8 * (kCBarAccDone0 + g), 1);
-            mbar_init(bars + 8 * (kCBarAccFree0 + g), 128);
-        }
-        mbar_init(bars + 8 * kCBarDrain, 1);
+        mbar_init(bars + 8 * kCBarUFree0, kCTokenThreads);
+        mbar_init(bars + 8 * kCBarUFree1, kCTokenThreads);
+        mbar_init(bars + 8 * kCBarAccDone, 1);
+        mbar_init(bars + 8 * kCBarAccFree, kCTokenThreads);
+        mbar_init(bars + 8 * kCBarDrain0, 1);
+        mbar_init(bars + 8 * kCBarDrain1, 1);
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async_smem();
@@ -175,8 +173,12 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     drain_bar(bars + 8 * (kCBarStageFull0 + m % kS), (uint32_t)(m / kS) & 1u);
             }
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
+    } else if (warp == 1 || warp == kCThreads / 32 - 1) {
+        // ---------------- two MMA issuers ----------------
+        // warp 1: U(k) = K_c W_phi_k for each tile whose K has landed, into the TMEM buffer k & 1 once the
+        // token threads have read U(k - 2) out of it.  Last warp: the accumulator MMAs of each tile whose
+        // K' has been written.  One thread each: a thread that has MMAs in flight is held at its next
+        // tcgen05 fence until they are done, so with a single issuer the two queues ran one after the other.
         if (lane == 0 && n_my > 0) {
             const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0, 0) >> 32);
             constexpr uint32_t kLboK = 1u << 16;
@@ -186,16 +188,11 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(desc_hi));
                 return d;
             };
-            constexpr uint32_t idesc_u = idesc_bf16(kTile, kTile, 0, 0);    // tile x map: both K-major
-            constexpr uint32_t idesc_tt = idesc_bf16(kTile, kTile, 1, 1);   // both operands token-major
             bool ok = true;
-            uint32_t w_seen = 0;        // maps waited for
-            uint32_t n_store[2] = {0, 0};   // per token group: accumulator stores asked for so far
-            int storing = -1;           // the group that stores the segment just ended (every waiter of a
-                                        // barrier follows its phases one by one: a barrier per group)
-            for (int k = 0; k <= n_my && ok; ++k) {
-                if (k < n_my) {
-                    // ---- U(k) = K_c W_phi_k into buffer k & 1
+            if (warp == 1) {
+                constexpr uint32_t idesc_u = idesc_bf16(kTile, kTile, 0, 0);    // tile x map: both K-major
+                uint32_t w_seen = 0;                                             // maps consumed
+                for (int k = 0; k < n_my && ok; ++k) {
                     const int s = k % kS, u = k & 1;
                     if (seg_first(k)) {
                         ok = wait_bar(bars + 8 * kCBarWFull, w_seen & 1u, ab, 82);
@@ -216,14 +213,16 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     // the next tile belongs to another head: its map may replace this one
                     if (k + 1 < n_my && seg_first(k + 1)) mma_commit(bars + 8 * kCBarWFree);
                 }
-                if (k >= 1) {
-                    // ---- accumulators += (w K')^T V_c  [and (beta K')^T K'] for tile k - 1
-                    const int j = k - 1, s = j % kS;
-                    ok = wait_bar(bars + 8 * (kCBarKpFull0 + s), (uint32_t)(j / kS) & 1u, ab, 85);
-                    const bool first = seg_first(j);
-                    if (ok && first && storing >= 0)
-                        ok = wait_bar(bars + 8 * (kCBarAccFree0 + storing), (n_store[storing] - 1) & 1u, ab, 86);
+            } else {
+                constexpr uint32_t idesc_tt = idesc_bf16(kTile, kTile, 1, 1);   // both operands token-major
+                uint32_t n_seg = 0;             // segments whose accumulators were handed over
+                for (int k = 0; k < n_my && ok; ++k) {
+                    const int s = k % kS;
+                    const bool first = seg_first(k);
+                    ok = wait_bar(bars + 8 * (kCBarKpFull0 + s), (uint32_t)(k / kS) & 1u, ab, 85);
+                    if (ok && first && n_seg > 0) ok = wait_bar(bars + 8 * kCBarAccFree, (n_seg - 1) & 1u, ab, 86);
                     if (!ok) break;
+                    // accumulators += (w K')^T V_c  [and (beta K')^T K']
                     tc_fence_after();
                     const uint32_t k_lo = ((smem_base + stage_k(s)) >> 4) | kLboMN;
                     const uint32_t v_lo = ((smem_base + stage_k(s) + kTileBytes) >> 4) | kLboMN;
@@ -239,61 +238,65 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                                    desc64(k_lo + (uint32_t)(ks * (2048 >> 4))), idesc_tt, (!first || ks > 0) ? 1u : 0u);
                     }
                     mma_commit(bars + 8 * (kCBarStageFree0 + s));
-                    if (seg_last(j)) {
-                        storing = j & 1;
-                        mma_commit(bars + 8 * (kCBarAccDone0 + storing));
-                        ++n_store[storing];
+                    if (seg_last(k)) {
+                        mma_commit(bars + 8 * kCBarAccDone);
+                        ++n_seg;
                     }
                 }
             }
             if (!ok || *abort_flag) {
                 // tensor memory is freed below: none of this thread's MMAs may still be running
-                mma_commit(bars + 8 * kCBarDrain);
-                drain_bar(bars + 8 * kCBarDrain, 0);
+                const uint32_t bar_drain = bars + 8 * (warp == 1 ? kCBarDrain0 : kCBarDrain1);
+                mma_commit(bar_drain);
+                drain_bar(bar_drain, 0);
             }
         }
     } else {
-        // ---------------- token groups: thread = token row of the tiles k = g, g + 2, ... ----------------
-        const int g = (warp - 2) >> 2;
+        // ---------------- token threads: (row r, half hf) of every tile of the run ----------------
+        const int hf = (warp - 2) >> 2;             // which 64 of the 128 columns
         const int q = warp & 3;                     // TMEM lane quarter this warp may access
         const int r = q * 32 + lane;                // token row of the tile = TMEM lane
         const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
-        const uint32_t u_addr = lane_base + (uint32_t)(g * kTile);
-        uint32_t n_store = 0;                       // accumulator stores this group has done
+        const bool rotate = p.rope_h != nullptr;
+        uint32_t n_seg = 0;                         // accumulator hand-overs so far
         bool ok = true;
         for (int k = 0; k < n_my && ok; ++k) {
-            const bool last = seg_last(k);
-            if ((k & 1) != g) continue;
             int bh, tl;
             tile_of(k, bh, tl);
             const int b = bh / H, h = bh - b * H;
             const int s = k % kS;
             const int row = tl * kTile + r;
             uint8_t* ktile = smem + stage_k(s);
+            const uint32_t u_addr = lane_base + (uint32_t)((k & 1) * kTile);
+            // my half of the row of the rotation table (32 pairs as half2, 8 vectors): requested before
+            // any wait, so its latency hides behind the wait for the tile
+            uint4 cs[8];
+            if (rotate) {
+                const uint4* tab = p.rope_h + ((size_t)(row >> 5) * 16 + hf * 8) * 32 + (row & 31);
+#pragma unroll
+                for (int c = 0; c < 8; ++c) cs[c] = __ldg(tab + c * 32);
+            }
             // per-token factor on K': the decay weight (mode 2) or the learning rate (delta rule)
             float wtok = 1.0f;
             if (kMode != 0 && p.beta != nullptr && row < L) {
                 const float x = __ldg(p.beta + ((size_t)b * L + row) * H + h);
                 wtok = kMode == 1 ? sigmoid_fast(x) : x;
             }
-            const uint4* tab = p.rope_h != nullptr ? p.rope_h + ((size_t)(row >> 5) * 16) * 32 + (row & 31) : nullptr;
             if (p.k_rot != nullptr) {
                 // ---- RoPE(K_c) for the softmax branch: the raw tile is in shared memory
                 ok = wait_bar(bars + 8 * (kCBarStageFull0 + s), (uint32_t)(k / kS) & 1u, ab, 87);
                 if (!ok) break;
                 if (row < L) {
-                    __nv_bfloat16* dst = p.k_rot + (((size_t)b * L + row) * H + h) * kTile;
+                    __nv_bfloat16* dst = p.k_rot + (((size_t)b * L + row) * H + h) * kTile + hf * 64;
 #pragma unroll
-                    for (int c2 = 0; c2 < 8; ++c2) {
+                    for (int c2 = 0; c2 < 4; ++c2) {
                         uint32_t w[8];
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
                             const int c = c2 * 2 + e;
-                            const uint4 cs = __ldg(tab + c * 32);
-                            const uint4 raw = *reinterpret_cast<const uint4*>(
-                                ktile + (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+                            const uint4 raw = *reinterpret_cast<const uint4*>(ktile + hf * kHalfBytes + r * 128 + ((c ^ (r & 7)) << 4));
                             const uint32_t x[4] = {raw.x, raw.y, raw.z, raw.w};
-                            const uint32_t h2[4] = {cs.x, cs.y, cs.z, cs.w};
+                            const uint32_t h2[4] = {cs[c].x, cs[c].y, cs[c].z, cs[c].w};
 #pragma unroll
                             for (int m = 0; m < 4; ++m) {
                                 float cc, ss;
@@ -309,72 +312,67 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     }
                 }
             }
-            // ---- K' = L2Norm(RoPE(U)): the row arrives in two halves of 64 columns
-            ok = wait_bar(bars + 8 * (kCBarUFull0 + g), (uint32_t)(k >> 1) & 1u, ab, 88);
+            // ---- K' = L2Norm(RoPE(U)).  Both threads of a row read the whole row for its norm (a
+            // rotation leaves the norm as it is, so the unrotated values serve), the other half first;
+            // each keeps, rotates, rounds and stores its own half.
+            ok = wait_bar(bars + 8 * (kCBarUFull0 + (k & 1)), (uint32_t)(k >> 1) & 1u, ab, 88);
             if (!ok) break;
             tc_fence_after();
-            uint32_t ureg[128];
+            uint32_t x[64];
             float ss4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                uint4 cs[8];
-                if (tab != nullptr) {
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) cs[c] = __ldg(tab + (hf * 8 + c) * 32);
-                }
-                tmem_ld32(u_addr + hf * 64, *reinterpret_cast<uint32_t(*)[32]>(&ureg[hf * 64]));
-                tmem_ld32(u_addr + hf * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&ureg[hf * 64 + 32]));
+            for (int part = 0; part < 2; ++part) {
+                const int col = (part == 0 ? (hf ^ 1) : hf) * 64;
+                tmem_ld32(u_addr + col, *reinterpret_cast<uint32_t(*)[32]>(&x[0]));
+                tmem_ld32(u_addr + col + 32, *reinterpret_cast<uint32_t(*)[32]>(&x[32]));
                 tmem_wait_ld();
-                if (tab != nullptr) {
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const uint32_t h2[4] = {cs[c].x, cs[c].y, cs[c].z, cs[c].w};
-#pragma unroll
-                        for (int m = 0; m < 4; ++m) {
-                            float cc, s1;
-                            unpack_cs(h2[m], cc, s1);
-                            const int i = hf * 64 + c * 8 + 2 * m;
-                            const float x0 = __uint_as_float(ureg[i]), x1 = __uint_as_float(ureg[i + 1]);
-                            ureg[i] = __float_as_uint(x0 * cc - x1 * s1);
-                            ureg[i + 1] = __float_as_uint(x0 * s1 + x1 * cc);
-                        }
-                    }
-                }
 #pragma unroll
                 for (int c = 0; c < 64; c += 4) {
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float x = __uint_as_float(ureg[hf * 64 + c + e]);
-                        ss4[e] = fmaf(x, x, ss4[e]);
-                    }
+                    for (int e = 0; e < 4; ++e) ss4[e] = fmaf(__uint_as_float(x[c + e]), __uint_as_float(x[c + e]), ss4[e]);
                 }
             }
             tc_fence_before();
-            mbar_arrive(bars + 8 * (kCBarUFree0 + g));      // buffer g may receive U(k + 2)
+            mbar_arrive(bars + 8 * (kCBarUFree0 + (k & 1)));      // the buffer may receive U(k + 2)
             const float f = rsqrtf((ss4[0] + ss4[1]) + (ss4[2] + ss4[3]) + p.s.eps);
+            if (rotate) {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t h2[4] = {cs[c].x, cs[c].y, cs[c].z, cs[c].w};
+#pragma unroll
+                    for (int m = 0; m < 4; ++m) {
+                        float cc, s1;
+                        unpack_cs(h2[m], cc, s1);
+                        const int i = c * 8 + 2 * m;
+                        const float x0 = __uint_as_float(x[i]), x1 = __uint_as_float(x[i + 1]);
+                        x[i] = __float_as_uint(x0 * cc - x1 * s1);
+                        x[i + 1] = __float_as_uint(x0 * s1 + x1 * cc);
+                    }
+                }
+            }
             // rows past L are zero (TMA fills them, the table's padding rows are zero): K' = 0 there
             if (kMode == 1) {
-                store_row_bf16_swizzled(ktile, r, ureg, f);                       // K'      (B of G)
-                store_row_bf16_swizzled(smem + extra_tile(s), r, ureg, f * wtok); // beta K' (A of both)
+                store_half_row_bf16_swizzled(ktile, r, hf, x, f);                       // K'      (B of G)
+                store_half_row_bf16_swizzled(smem + extra_tile(s), r, hf, x, f * wtok); // beta K' (A of both)
             } else {
-                store_row_bf16_swizzled(ktile, r, ureg, f * wtok);
+                store_half_row_bf16_swizzled(ktile, r, hf, x, f * wtok);
             }
             fence_proxy_async_smem();
             mbar_arrive(bars + 8 * (kCBarKpFull0 + s));
-            if (last) {
-                // ---- this head's share of the accumulators (row d_k = r) -> its slot of the partial sums
-                ok = wait_bar(bars + 8 * (kCBarAccDone0 + g), n_store & 1u, ab, 89);
+            if (seg_last(k)) {
+                // ---- this head's share of the accumulators (row d_k = r, my 64 columns) -> its slot
+                ok = wait_bar(bars + 8 * kCBarAccDone, n_seg & 1u, ab, 89);
                 if (!ok) break;
                 tc_fence_after();
                 const int part = (int)blockIdx.x - (bh * p.ntile) / p.share;
-                const size_t at = (((size_t)bh * p.nslot + part) * kTile + r) * kTile;
+                const size_t at = (((size_t)bh * p.nslot + part) * kTile + r) * kTile + hf * 64;
 #pragma unroll 1
                 for (int acc = 0; acc < (kMode == 1 ? 2 : 1); ++acc) {
                     float* dst = (acc == 0 ? p.partials : p.partials_g) + at;
 #pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
+                    for (int c = 0; c < 2; ++c) {
                         uint32_t o[32];
-                        tmem_ld32(lane_base + kColDS + acc * kTile + c * 32, o);
+                        tmem_ld32(lane_base + kColDS + acc * kTile + hf * 64 + c * 32, o);
                         tmem_wait_ld();
 #pragma unroll
                         for (int e = 0; e < 4; ++e)   // 32-byte stores: whole sectors
@@ -385,8 +383,8 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     }
                 }
                 tc_fence_before();
-                mbar_arrive(bars + 8 * (kCBarAccFree0 + g));
-                ++n_store;
+                mbar_arrive(bars + 8 * kCBarAccFree);
+                ++n_seg;
             }
         }
     }
@@ -399,42 +397,52 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     }
 }
 
-// S <- alpha S + (sum_s A_s) W_phi_v [- (sum_s G_s) S_old]; one CTA per 16 state rows of a head.
-// The slots of a head are added in index order.  256 threads: thread = (output column, 8 of the rows).
+// S <- alpha S + (sum_s A_s) W_phi_v [- (sum_s G_s) S_old]; one CTA per 16 state rows of a head, 128
+// threads, each a 4 x 4 block of the 16 x 128 output.  The slots of a head are added in index order.
 // The right-hand matrices (the head's value map, then S_old) pass through shared memory as bf16.
+// Every global load the CTA needs is requested before the first result is used.
 constexpr int kFinRows = 16;
+constexpr int kFinThreads = 128;
+constexpr int kFinMaxParts = 6;     // slots of one head the unrolled loads cover; more fall back to a loop
 constexpr int kFinSmemBytes = kTileBytes + 2 * kFinRows * kTile * 4;
 
 __device__ __forceinline__ void fin_load_matrix(__nv_bfloat16* dst, const __nv_bfloat16* __restrict__ src, int tid)
 {
     const uint4* s4 = reinterpret_cast<const uint4*>(src);
     uint4* d4 = reinterpret_cast<uint4*>(dst);
+    uint4 v[kTileBytes / 16 / kFinThreads];
 #pragma unroll
-    for (int i = 0; i < kTileBytes / 16 / 256; ++i) d4[tid + i * 256] = __ldg(s4 + tid + i * 256);
+    for (int i = 0; i < kTileBytes / 16 / kFinThreads; ++i) v[i] = __ldg(s4 + tid + i * kFinThreads);
+#pragma unroll
+    for (int i = 0; i < kTileBytes / 16 / kFinThreads; ++i) d4[tid + i * kFinThreads] = v[i];
 }
 
-// acc[i] += sign * sum_m X[row_i][m] * M[m][e]
-__device__ __forceinline__ void fin_multiply(float (&acc)[8], const float* __restrict__ X, const __nv_bfloat16* __restrict__ M,
-                                             int e, float sign)
+// acc[i][j] += sign * sum_m X[i][m] * M[m][4 cg + j]   (X: this thread's 4 rows, row stride 128)
+__device__ __forceinline__ void fin_multiply(float (&acc)[4][4], const float* __restrict__ X,
+                                             const __nv_bfloat16* __restrict__ M, int cg, float sign)
 {
-#pragma unroll 4
+#pragma unroll 2
     for (int m = 0; m < kTile; m += 4) {
-        float w[4];
+        float4 xr[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) w[j] = sign * __bfloat162float(M[(m + j) * kTile + e]);
+        for (int i = 0; i < 4; ++i) xr[i] = *reinterpret_cast<const float4*>(X + i * kTile + m);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float4 x = *reinterpret_cast<const float4*>(X + i * kTile + m);
-            acc[i] = fmaf(x.x, w[0], acc[i]);
-            acc[i] = fmaf(x.y, w[1], acc[i]);
-            acc[i] = fmaf(x.z, w[2], acc[i]);
-            acc[i] = fmaf(x.w, w[3], acc[i]);
+        for (int mm = 0; mm < 4; ++mm) {
+            const uint2 wb = *reinterpret_cast<const uint2*>(M + (m + mm) * kTile + 4 * cg);
+            const float w[4] = {sign * __uint_as_float(wb.x << 16), sign * __uint_as_float(wb.x & 0xFFFF0000u),
+                                sign * __uint_as_float(wb.y << 16), sign * __uint_as_float(wb.y & 0xFFFF0000u)};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float xv = mm == 0 ? xr[i].x : mm == 1 ? xr[i].y : mm == 2 ? xr[i].z : xr[i].w;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(xv, w[j], acc[i][j]);
+            }
         }
     }
 }
 
 template <int kMode>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kFinThreads)
 tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ partials,
                         const float* __restrict__ partials_g, const __nv_bfloat16* __restrict__ wv,
                         const float* __restrict__ decay, int decay_direct,
@@ -445,53 +453,95 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
     __nv_bfloat16* Ms = reinterpret_cast<__nv_bfloat16*>(fin_smem);               // [128][128] right-hand matrix
     float* As = reinterpret_cast<float*>(fin_smem + kTileBytes);                   // [16][128]
     float* Gs = As + kFinRows * kTile;                                             // [16][128] (delta rule)
-    const int tid = threadIdx.x, e = tid & 127, half = tid >> 7;
+    const int tid = threadIdx.x, cg = tid & 31, rg = tid >> 5;
     const int bh = (int)(blockIdx.x / (kTile / kFinRows)), h = bh % H;
-    const int row0 = (int)(blockIdx.x % (kTile / kFinRows)) * kFinRows + half * 8;
+    const int row0 = (int)(blockIdx.x % (kTile / kFinRows)) * kFinRows + rg * 4;   // this thread's 4 rows
     const size_t head = (size_t)bh * kTile * kTile;
-    if (status != nullptr && status[kStatusError] != 0u) {
-        // a partial-sum CTA gave up on a bounded wait: S stays as it was, and so does its mirror
-#pragma unroll
-        for (int i = 0; i < 8; ++i) mirror_next[head + (size_t)(row0 + i) * kTile + e] = mirror_cur[head + (size_t)(row0 + i) * kTile + e];
-        return;
-    }
-    if (wv != nullptr) fin_load_matrix(Ms, wv + (size_t)h * kTile * kTile, tid);   // [in = m][out = e]
+    const size_t mine = head + (size_t)row0 * kTile + 4 * cg;                      // rows 128 apart
+    const uint32_t err = status != nullptr ? status[kStatusError] : 0u;
     const int first = (bh * ntile) / share, last = (bh * ntile + ntile - 1) / share;
     const int nparts = last - first + 1;
-    float a[8], gsum[8];
+    const size_t slot0 = ((size_t)bh * nslot * kTile + row0) * kTile + 4 * cg;
+    // ---- all loads first: the slots, the old state rows, the value map
+    float4 pa[kFinMaxParts][4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) a[i] = gsum[i] = 0.0f;
-    for (int s = 0; s < nparts; ++s) {
-        const size_t at = (((size_t)bh * nslot + s) * kTile + row0) * kTile + e;
+    for (int s = 0; s < kFinMaxParts; ++s) {
+        if (s < nparts) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) a[i] += partials[at + (size_t)i * kTile];
-        if (kMode == 1) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) gsum[i] += partials_g[at + (size_t)i * kTile];
+            for (int i = 0; i < 4; ++i)
+                pa[s][i] = *reinterpret_cast<const float4*>(partials + slot0 + ((size_t)s * kTile + i) * kTile);
         }
     }
-    float out[8];
+    float4 old[4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        out[i] = wv != nullptr ? 0.0f : a[i];
-        As[(half * 8 + i) * kTile + e] = a[i];
-        if (kMode == 1) Gs[(half * 8 + i) * kTile + e] = gsum[i];
+    for (int i = 0; i < 4; ++i) old[i] = *reinterpret_cast<const float4*>(state + mine + (size_t)i * kTile);
+    if (wv != nullptr) fin_load_matrix(Ms, wv + (size_t)h * kTile * kTile, tid);   // [in = m][out = e]
+    if (err != 0u) {
+        // a partial-sum CTA gave up on a bounded wait: S stays as it was, and so does its mirror
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            *reinterpret_cast<uint2*>(mirror_next + mine + (size_t)i * kTile) =
+                *reinterpret_cast<const uint2*>(mirror_cur + mine + (size_t)i * kTile);
+        return;
+    }
+    float4 a[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) a[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int s = 0; s < kFinMaxParts; ++s) {
+        if (s < nparts) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                a[i].x += pa[s][i].x; a[i].y += pa[s][i].y; a[i].z += pa[s][i].z; a[i].w += pa[s][i].w;
+            }
+        }
+    }
+    for (int s = kFinMaxParts; s < nparts; ++s) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float4 v = *reinterpret_cast<const float4*>(partials + slot0 + ((size_t)s * kTile + i) * kTile);
+            a[i].x += v.x; a[i].y += v.y; a[i].z += v.z; a[i].w += v.w;
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(As + (rg * 4 + i) * kTile + 4 * cg) = a[i];
+    if (kMode == 1) {
+        float4 gs[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) gs[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s = 0; s < nparts; ++s) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float4 v = *reinterpret_cast<const float4*>(partials_g + slot0 + ((size_t)s * kTile + i) * kTile);
+                gs[i].x += v.x; gs[i].y += v.y; gs[i].z += v.z; gs[i].w += v.w;
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(Gs + (rg * 4 + i) * kTile + 4 * cg) = gs[i];
     }
     __syncthreads();
-    if (wv != nullptr) fin_multiply(out, As + half * 8 * kTile, Ms, e, 1.0f);
+    float out[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const bool id = wv == nullptr;
+        out[i][0] = id ? a[i].x : 0.0f; out[i][1] = id ? a[i].y : 0.0f;
+        out[i][2] = id ? a[i].z : 0.0f; out[i][3] = id ? a[i].w : 0.0f;
+    }
+    if (wv != nullptr) fin_multiply(out, As + rg * 4 * kTile, Ms, cg, 1.0f);
     if (kMode == 1) {
         __syncthreads();                                   // every thread is done with the value map
         fin_load_matrix(Ms, mirror_cur + head, tid);       // S_old [m][e]
         __syncthreads();
-        fin_multiply(out, Gs + half * 8 * kTile, Ms, e, -1.0f);
+        fin_multiply(out, Gs + rg * 4 * kTile, Ms, cg, -1.0f);
     }
     const float alpha = decay_direct ? decay[bh] : 1.0f / (1.0f + __expf(-decay[bh]));
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const size_t at = head + (size_t)(row0 + i) * kTile + e;
-        const float nw = alpha * state[at] + out[i];
-        state[at] = nw;
-        mirror_next[at] = __float2bfloat16_rn(nw);
+    for (int i = 0; i < 4; ++i) {
+        const float4 nw = make_float4(alpha * old[i].x + out[i][0], alpha * old[i].y + out[i][1],
+                                      alpha * old[i].z + out[i][2], alpha * old[i].w + out[i][3]);
+        *reinterpret_cast<float4*>(state + mine + (size_t)i * kTile) = nw;
+        *reinterpret_cast<uint2*>(mirror_next + mine + (size_t)i * kTile) =
+            make_uint2(pack_bf16(nw.x, nw.y), pack_bf16(nw.z, nw.w));
     }
 }
 
@@ -564,11 +614,11 @@ int tc_commit_finish(const CommitArgs& a, cudaStream_t st)
     const unsigned grid = (unsigned)(a.s.B * a.s.H) * (kTile / kFinRows);
     const __nv_bfloat16* wv = static_cast<const __nv_bfloat16*>(a.wv);
     if (a.mode == 1)
-        tc_commit_finish_kernel<1><<<grid, 256, kFinSmemBytes, st>>>(a.state, a.partials, a.partials_g, wv, a.decay,
+        tc_commit_finish_kernel<1><<<grid, kFinThreads, kFinSmemBytes, st>>>(a.state, a.partials, a.partials_g, wv, a.decay,
                                                          a.decay_direct ? 1 : 0, a.state_bf16, a.state_bf16_next,
                                                          a.s.H, a.run_share, a.run_ntile, a.nslot, a.status);
     else
-        tc_commit_finish_kernel<0><<<grid, 256, kFinSmemBytes, st>>>(a.state, a.partials, a.partials_g, wv, a.decay,
+        tc_commit_finish_kernel<0><<<grid, kFinThreads, kFinSmemBytes, st>>>(a.state, a.partials, a.partials_g, wv, a.decay,
                                                          a.decay_direct ? 1 : 0, a.state_bf16, a.state_bf16_next,
                                                          a.s.H, a.run_share, a.run_ntile, a.nslot, a.status);
     cudaError_t e = cudaGetLastError();

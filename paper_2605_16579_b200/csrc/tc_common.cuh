@@ -103,6 +103,19 @@ __device__ __forceinline__ void store_row_bf16_swizzled(uint8_t* tile, int r, co
         *reinterpret_cast<uint4*>(tile + off) = v;
     }
 }
+// half of row r (64 columns = one 64-column box of the tile)
+__device__ __forceinline__ void store_half_row_bf16_swizzled(uint8_t* tile, int r, int half, const uint32_t (&x)[64], float f)
+{
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        uint4 v;
+        v.x = pack_bf16(__uint_as_float(x[c * 8 + 0]) * f, __uint_as_float(x[c * 8 + 1]) * f);
+        v.y = pack_bf16(__uint_as_float(x[c * 8 + 2]) * f, __uint_as_float(x[c * 8 + 3]) * f);
+        v.z = pack_bf16(__uint_as_float(x[c * 8 + 4]) * f, __uint_as_float(x[c * 8 + 5]) * f);
+        v.w = pack_bf16(__uint_as_float(x[c * 8 + 6]) * f, __uint_as_float(x[c * 8 + 7]) * f);
+        *reinterpret_cast<uint4*>(tile + half * kHalfBytes + r * 128 + ((c ^ (r & 7)) << 4)) = v;
+    }
+}
 __device__ __forceinline__ void store_row_bf16_global(__nv_bfloat16* dst, const uint32_t (&x)[128], float f)
 {
 #pragma unroll
