@@ -165,6 +165,9 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     tma_load_2d(smem_base + kCOffWk + kHalfBytes, &tm_wk, bars + 8 * kCBarWFull, 64, hh * kTile);
                     ++n_w;
                 }
+                // the first tile alone first: with every CTA of the grid asking for its whole ring at
+                // once the first stage would land only after a third of that burst
+                if (k == 0 && n_my > 1) ok = wait_bar(bars + 8 * (kCBarStageFull0 + 0), 0u, ab, 79);
             }
             if (!ok || *abort_flag) {
                 // do not leave the CTA while bulk copies into its shared memory are in flight
@@ -404,38 +407,45 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 constexpr int kFinRows = 16;
 constexpr int kFinThreads = 128;
 constexpr int kFinMaxParts = 6;     // slots of one head the unrolled loads cover; more fall back to a loop
-constexpr int kFinSmemBytes = kTileBytes + 2 * kFinRows * kTile * 4;
+// shared memory: the right-hand matrix as bf16 [128][128], then A and G rows with every value stored
+// twice in a row (x, x): a 16-byte load then yields two packed-FMA operands
+constexpr int kFinSmemBytes = kTileBytes + 2 * kFinRows * kTile * 8;
 
 __device__ __forceinline__ void fin_load_matrix(__nv_bfloat16* dst, const __nv_bfloat16* __restrict__ src, int tid)
 {
     const uint4* s4 = reinterpret_cast<const uint4*>(src);
     uint4* d4 = reinterpret_cast<uint4*>(dst);
-    uint4 v[kTileBytes / 16 / kFinThreads];
+    constexpr int kPer = kTileBytes / 16 / kFinThreads;
+    uint4 v[kPer];
 #pragma unroll
-    for (int i = 0; i < kTileBytes / 16 / kFinThreads; ++i) v[i] = __ldg(s4 + tid + i * kFinThreads);
+    for (int i = 0; i < kPer; ++i) v[i] = __ldg(s4 + tid + i * kFinThreads);
 #pragma unroll
-    for (int i = 0; i < kTileBytes / 16 / kFinThreads; ++i) d4[tid + i * kFinThreads] = v[i];
+    for (int i = 0; i < kPer; ++i) d4[tid + i * kFinThreads] = v[i];
 }
 
-// acc[i][j] += sign * sum_m X[i][m] * M[m][4 cg + j]   (X: this thread's 4 rows, row stride 128)
-__device__ __forceinline__ void fin_multiply(float (&acc)[4][4], const float* __restrict__ X,
-                                             const __nv_bfloat16* __restrict__ M, int cg, float sign)
+// acc[i][j] (+/-)= sum_m X[i][m] * M[m][4 cg + j]   (X: this thread's 4 rows, each value doubled, row
+// stride 256 floats; two columns per packed FMA; bf16 -> fp32 by shifts, off the FMA pipe)
+template <bool kSubtract>
+__device__ __forceinline__ void fin_multiply(uint64_t (&acc)[4][2], const float* __restrict__ X,
+                                             const __nv_bfloat16* __restrict__ M, int cg)
 {
-#pragma unroll 2
-    for (int m = 0; m < kTile; m += 4) {
-        float4 xr[4];
+    constexpr uint32_t kSign = kSubtract ? 0x80000000u : 0u;
+#pragma unroll 4
+    for (int m = 0; m < kTile; m += 2) {
+        ulonglong2 xr[4];      // (x_m, x_m), (x_m+1, x_m+1) of each row
 #pragma unroll
-        for (int i = 0; i < 4; ++i) xr[i] = *reinterpret_cast<const float4*>(X + i * kTile + m);
+        for (int i = 0; i < 4; ++i) xr[i] = *reinterpret_cast<const ulonglong2*>(X + i * 2 * kTile + 2 * m);
 #pragma unroll
-        for (int mm = 0; mm < 4; ++mm) {
-            const uint2 wb = *reinterpret_cast<const uint2*>(M + (m + mm) * kTile + 4 * cg);
-            const float w[4] = {sign * __uint_as_float(wb.x << 16), sign * __uint_as_float(wb.x & 0xFFFF0000u),
-                                sign * __uint_as_float(wb.y << 16), sign * __uint_as_float(wb.y & 0xFFFF0000u)};
+        for (int mm = 0; mm < 2; ++mm) {
+            const uint2 wb = *reinterpret_cast<const uint2*>(M + (m + mm) * kTile + 4 * cg);   // 4 columns
+            uint64_t w01, w23;
+            asm("mov.b64 %0, {%1, %2};" : "=l"(w01) : "r"((wb.x << 16) ^ kSign), "r"((wb.x & 0xFFFF0000u) ^ kSign));
+            asm("mov.b64 %0, {%1, %2};" : "=l"(w23) : "r"((wb.y << 16) ^ kSign), "r"((wb.y & 0xFFFF0000u) ^ kSign));
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const float xv = mm == 0 ? xr[i].x : mm == 1 ? xr[i].y : mm == 2 ? xr[i].z : xr[i].w;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(xv, w[j], acc[i][j]);
+                const uint64_t xx = mm == 0 ? xr[i].x : xr[i].y;
+                acc[i][0] = fma2(xx, w01, acc[i][0]);
+                acc[i][1] = fma2(xx, w23, acc[i][1]);
             }
         }
     }
@@ -450,14 +460,20 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
                         int H, int share, int ntile, int nslot, const uint32_t* __restrict__ status)
 {
     extern __shared__ __align__(16) uint8_t fin_smem[];
-    __nv_bfloat16* Ms = reinterpret_cast<__nv_bfloat16*>(fin_smem);               // [128][128] right-hand matrix
-    float* As = reinterpret_cast<float*>(fin_smem + kTileBytes);                   // [16][128]
-    float* Gs = As + kFinRows * kTile;                                             // [16][128] (delta rule)
+    __nv_bfloat16* Ms = reinterpret_cast<__nv_bfloat16*>(fin_smem);                 // [128][128] right-hand matrix
+    float* As = reinterpret_cast<float*>(fin_smem + kTileBytes);                    // [16][128] x 2 (doubled)
+    float* Gs = As + kFinRows * kTile * 2;                                          // same (delta rule)
     const int tid = threadIdx.x, cg = tid & 31, rg = tid >> 5;
     const int bh = (int)(blockIdx.x / (kTile / kFinRows)), h = bh % H;
     const int row0 = (int)(blockIdx.x % (kTile / kFinRows)) * kFinRows + rg * 4;   // this thread's 4 rows
     const size_t head = (size_t)bh * kTile * kTile;
     const size_t mine = head + (size_t)row0 * kTile + 4 * cg;                      // rows 128 apart
+    // Launched with programmatic stream serialisation: the CTA may start while the partial-sum kernel
+    // is still draining.  What does not depend on that kernel (the value map) is fetched first; the
+    // wait below returns once the whole preceding kernel has finished and its writes are visible.
+    if (wv != nullptr) fin_load_matrix(Ms, wv + (size_t)h * kTile * kTile, tid);   // [in = m][out = e]
+    const float decay_v = decay[bh];
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t err = status != nullptr ? status[kStatusError] : 0u;
     const int first = (bh * ntile) / share, last = (bh * ntile + ntile - 1) / share;
     const int nparts = last - first + 1;
@@ -475,7 +491,6 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
     float4 old[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) old[i] = *reinterpret_cast<const float4*>(state + mine + (size_t)i * kTile);
-    if (wv != nullptr) fin_load_matrix(Ms, wv + (size_t)h * kTile * kTile, tid);   // [in = m][out = e]
     if (err != 0u) {
         // a partial-sum CTA gave up on a bounded wait: S stays as it was, and so does its mirror
 #pragma unroll
@@ -484,6 +499,12 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
                 *reinterpret_cast<const uint2*>(mirror_cur + mine + (size_t)i * kTile);
         return;
     }
+    auto add4 = [](float4& d, const float4& v) { d.x += v.x; d.y += v.y; d.z += v.z; d.w += v.w; };
+    auto store_doubled = [&](float* dst, int i, const float4& v) {     // row rg * 4 + i, columns 4 cg .. + 3
+        float4* d = reinterpret_cast<float4*>(dst + (size_t)(rg * 4 + i) * 2 * kTile + 8 * cg);
+        d[0] = make_float4(v.x, v.x, v.y, v.y);
+        d[1] = make_float4(v.z, v.z, v.w, v.w);
+    };
     float4 a[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) a[i] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -491,54 +512,51 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
     for (int s = 0; s < kFinMaxParts; ++s) {
         if (s < nparts) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                a[i].x += pa[s][i].x; a[i].y += pa[s][i].y; a[i].z += pa[s][i].z; a[i].w += pa[s][i].w;
-            }
+            for (int i = 0; i < 4; ++i) add4(a[i], pa[s][i]);
         }
     }
     for (int s = kFinMaxParts; s < nparts; ++s) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float4 v = *reinterpret_cast<const float4*>(partials + slot0 + ((size_t)s * kTile + i) * kTile);
-            a[i].x += v.x; a[i].y += v.y; a[i].z += v.z; a[i].w += v.w;
-        }
+        for (int i = 0; i < 4; ++i)
+            add4(a[i], *reinterpret_cast<const float4*>(partials + slot0 + ((size_t)s * kTile + i) * kTile));
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(As + (rg * 4 + i) * kTile + 4 * cg) = a[i];
+    for (int i = 0; i < 4; ++i) store_doubled(As, i, a[i]);
     if (kMode == 1) {
         float4 gs[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) gs[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int s = 0; s < nparts; ++s) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float4 v = *reinterpret_cast<const float4*>(partials_g + slot0 + ((size_t)s * kTile + i) * kTile);
-                gs[i].x += v.x; gs[i].y += v.y; gs[i].z += v.z; gs[i].w += v.w;
-            }
+            for (int i = 0; i < 4; ++i)
+                add4(gs[i], *reinterpret_cast<const float4*>(partials_g + slot0 + ((size_t)s * kTile + i) * kTile));
         }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(Gs + (rg * 4 + i) * kTile + 4 * cg) = gs[i];
+        for (int i = 0; i < 4; ++i) store_doubled(Gs, i, gs[i]);
     }
     __syncthreads();
-    float out[4][4];
+    uint64_t out[4][2];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const bool id = wv == nullptr;
-        out[i][0] = id ? a[i].x : 0.0f; out[i][1] = id ? a[i].y : 0.0f;
-        out[i][2] = id ? a[i].z : 0.0f; out[i][3] = id ? a[i].w : 0.0f;
+        out[i][0] = pack2(id ? a[i].x : 0.0f, id ? a[i].y : 0.0f);
+        out[i][1] = pack2(id ? a[i].z : 0.0f, id ? a[i].w : 0.0f);
     }
-    if (wv != nullptr) fin_multiply(out, As + rg * 4 * kTile, Ms, cg, 1.0f);
+    if (wv != nullptr) fin_multiply<false>(out, As + (size_t)rg * 4 * 2 * kTile, Ms, cg);
     if (kMode == 1) {
         __syncthreads();                                   // every thread is done with the value map
         fin_load_matrix(Ms, mirror_cur + head, tid);       // S_old [m][e]
         __syncthreads();
-        fin_multiply(out, Gs + rg * 4 * kTile, Ms, cg, -1.0f);
+        fin_multiply<true>(out, Gs + (size_t)rg * 4 * 2 * kTile, Ms, cg);
     }
-    const float alpha = decay_direct ? decay[bh] : 1.0f / (1.0f + __expf(-decay[bh]));
+    const float alpha = decay_direct ? decay_v : 1.0f / (1.0f + __expf(-decay_v));
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        const float4 nw = make_float4(alpha * old[i].x + out[i][0], alpha * old[i].y + out[i][1],
-                                      alpha * old[i].z + out[i][2], alpha * old[i].w + out[i][3]);
+        float o0, o1, o2, o3;
+        unpack2(out[i][0], o0, o1);
+        unpack2(out[i][1], o2, o3);
+        const float4 nw = make_float4(alpha * old[i].x + o0, alpha * old[i].y + o1,
+                                      alpha * old[i].z + o2, alpha * old[i].w + o3);
         *reinterpret_cast<float4*>(state + mine + (size_t)i * kTile) = nw;
         *reinterpret_cast<uint2*>(mirror_next + mine + (size_t)i * kTile) =
             make_uint2(pack_bf16(nw.x, nw.y), pack_bf16(nw.z, nw.w));
@@ -611,17 +629,32 @@ int tc_commit_partials(CommitArgs& a, const __nv_bfloat16* wk_op, cudaStream_t s
 
 int tc_commit_finish(const CommitArgs& a, cudaStream_t st)
 {
-    const unsigned grid = (unsigned)(a.s.B * a.s.H) * (kTile / kFinRows);
+    // programmatic stream serialisation: the grid is staged while the kernel before it in the stream
+    // (the partial sums) is still running; the kernel itself waits for that kernel where it must
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(a.s.B * a.s.H) * (kTile / kFinRows));
+    cfg.blockDim = dim3(kFinThreads);
+    cfg.dynamicSmemBytes = kFinSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     const __nv_bfloat16* wv = static_cast<const __nv_bfloat16*>(a.wv);
+    const float* partials = a.partials;
+    const float* partials_g = a.partials_g;
+    const __nv_bfloat16* cur = a.state_bf16;
+    const uint32_t* status = a.status;
+    const int direct = a.decay_direct ? 1 : 0;
+    cudaError_t e;
     if (a.mode == 1)
-        tc_commit_finish_kernel<1><<<grid, kFinThreads, kFinSmemBytes, st>>>(a.state, a.partials, a.partials_g, wv, a.decay,
-                                                         a.decay_direct ? 1 : 0, a.state_bf16, a.state_bf16_next,
-                                                         a.s.H, a.run_share, a.run_ntile, a.nslot, a.status);
+        e = cudaLaunchKernelEx(&cfg, tc_commit_finish_kernel<1>, a.state, partials, partials_g, wv, a.decay, direct, cur,
+                               a.state_bf16_next, a.s.H, a.run_share, a.run_ntile, a.nslot, status);
     else
-        tc_commit_finish_kernel<0><<<grid, kFinThreads, kFinSmemBytes, st>>>(a.state, a.partials, a.partials_g, wv, a.decay,
-                                                         a.decay_direct ? 1 : 0, a.state_bf16, a.state_bf16_next,
-                                                         a.s.H, a.run_share, a.run_ntile, a.nslot, a.status);
-    cudaError_t e = cudaGetLastError();
+        e = cudaLaunchKernelEx(&cfg, tc_commit_finish_kernel<0>, a.state, partials, partials_g, wv, a.decay, direct, cur,
+                               a.state_bf16_next, a.s.H, a.run_share, a.run_ntile, a.nslot, status);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { set_error("launch of tc_commit_finish_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
     return 1;
 }
