@@ -113,11 +113,11 @@ void arl2_oracle_feature(int B, int H, int L, int D, const double *x, const doub
  * gate_mode selects the granularity of the combine gate (the paper's layer is headwise; the other
  * two are the variants of its gate ablation): 0 headwise g [B, L, H]; 1 scalar g [B, L], one gate
  * per token shared by all heads; 2 elementwise g [B, L, H, D], one gate per output channel.
- * scratch: at least L + 3*D doubles.
+ * Sh: the D x D state of this (stream, head).  scratch: at least L + 3*D doubles.
  */
 static void step_row(int b, int h, int i, int H, int L, int D, int gate_mode,
                      const double *q, const double *k, const double *v, const double *g,
-                     const double *S, const double *wq,
+                     const double *Sh, const double *wq,
                      const double *rope_cos, const double *rope_sin,
                      double scale, double eps, double *o, double *scratch)
 {
@@ -155,7 +155,6 @@ static void step_row(int b, int h, int i, int H, int L, int D, int gate_mode,
     phi(q + qoff, wq, h, D, qf);
     rope(qf, D, rope_cos, rope_sin, i);
     l2norm(qf, D, eps);
-    const double *Sh = S + ((size_t)b * H + h) * D * D;
     for (int e = 0; e < D; ++e) {
         size_t gi = gate_mode == 1 ? (size_t)b * L + i
                   : gate_mode == 2 ? (((size_t)b * L + i) * H + h) * D + e
@@ -183,8 +182,8 @@ void arl2_oracle_step(int B, int H, int L, int D,
             int i = (int)(t % L);
             int h = (int)((t / L) % H);
             int b = (int)(t / ((long)L * H));
-            step_row(b, h, i, H, L, D, 0, q, k, v, g, S, wq, rope_cos, rope_sin, scale, eps,
-                     out + (((size_t)b * L + i) * H + h) * D, scratch);
+            step_row(b, h, i, H, L, D, 0, q, k, v, g, S + ((size_t)b * H + h) * D * D, wq, rope_cos, rope_sin,
+                     scale, eps, out + (((size_t)b * L + i) * H + h) * D, scratch);
         }
         free(scratch);
     }
@@ -206,8 +205,8 @@ void arl2_oracle_step_gate_mode(int B, int H, int L, int D, int gate_mode,
             int i = (int)(t % L);
             int h = (int)((t / L) % H);
             int b = (int)(t / ((long)L * H));
-            step_row(b, h, i, H, L, D, gate_mode, q, k, v, g, S, wq, rope_cos, rope_sin, scale, eps,
-                     out + (((size_t)b * L + i) * H + h) * D, scratch);
+            step_row(b, h, i, H, L, D, gate_mode, q, k, v, g, S + ((size_t)b * H + h) * D * D, wq, rope_cos,
+                     rope_sin, scale, eps, out + (((size_t)b * L + i) * H + h) * D, scratch);
         }
         free(scratch);
     }
@@ -230,9 +229,53 @@ void arl2_oracle_step_rows(int B, int H, int L, int D,
         double *scratch = (double *)malloc(sizeof(double) * ((size_t)L + 3 * (size_t)D));
 #pragma omp for schedule(dynamic, 4)
         for (int t = 0; t < n; ++t)
-            step_row(bs[t], hs[t], is[t], H, L, D, 0, q, k, v, g, S, wq, rope_cos, rope_sin,
-                     scale, eps, out_rows + (size_t)t * D, scratch);
+            step_row(bs[t], hs[t], is[t], H, L, D, 0, q, k, v, g, S + ((size_t)bs[t] * H + hs[t]) * D * D, wq,
+                     rope_cos, rope_sin, scale, eps, out_rows + (size_t)t * D, scratch);
         free(scratch);
+    }
+}
+
+/*
+ * Token-level state access, the comparison mode of Sec. 4.3 ("State access granularity"): instead of
+ * one pre-update state for the whole block, token i reads the state advanced by the block's tokens
+ * before it (each token sees its own sequentially accumulated state), the gated-linear update with
+ * one forget gate per token being applied token by token on a private copy:
+ *   S^(0) = S,   O_i = O_intra_i + sigmoid(g_i) Q'_i S^(i),   S^(i+1) = alpha_i S^(i) + K'_i^T V'_i,
+ * K' = L2Norm(RoPE(phi_k(K))), V' = phi_v(V) from the pass's own K, V; alpha_i = sigmoid(alpha_logit)
+ * or 1 when alpha_logit is NULL.  Token 0 reads S itself.  The intra-block softmax is unchanged
+ * (bidirectional over the block) and the caller's S is not written.
+ */
+void arl2_oracle_step_token_level(int B, int H, int L, int D,
+                                  const double *q, const double *k, const double *v, const double *g,
+                                  const double *alpha_logit, const double *S,
+                                  const double *wq, const double *wk, const double *wv,
+                                  const double *rope_cos, const double *rope_sin,
+                                  double scale, double eps, double *out)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int bh = 0; bh < B * H; ++bh) {
+        int b = bh / H, h = bh % H;
+        double *scratch = (double *)malloc(sizeof(double) * ((size_t)L + 3 * (size_t)D));
+        double *Sloc = (double *)malloc(sizeof(double) * D * D);
+        double *kf = (double *)malloc(sizeof(double) * D);
+        double *vf = (double *)malloc(sizeof(double) * D);
+        memcpy(Sloc, S + (size_t)bh * D * D, sizeof(double) * D * D);
+        for (int i = 0; i < L; ++i) {
+            size_t off = (((size_t)b * L + i) * H + h) * D;
+            /* the row of the layer against the state as this token sees it */
+            step_row(b, h, i, H, L, D, 0, q, k, v, g, Sloc, wq, rope_cos, rope_sin, scale, eps,
+                     out + off, scratch);
+            /* then the token's own write */
+            phi(k + off, wk, h, D, kf);
+            rope(kf, D, rope_cos, rope_sin, i);
+            l2norm(kf, D, eps);
+            phi(v + off, wv, h, D, vf);
+            double alpha = alpha_logit ? sigmoid(alpha_logit[((size_t)b * L + i) * H + h]) : 1.0;
+            for (int d = 0; d < D; ++d)
+                for (int e = 0; e < D; ++e)
+                    Sloc[(size_t)d * D + e] = alpha * Sloc[(size_t)d * D + e] + kf[d] * vf[e];
+        }
+        free(vf); free(kf); free(Sloc); free(scratch);
     }
 }
 

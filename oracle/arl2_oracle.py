@@ -136,6 +136,26 @@ def step_rows(q, k, v, g, S, rows, wq=None, rope_cos=None, rope_sin=None, scale=
     return out
 
 
+def step_token_level(q, k, v, g, S, alpha_logit=None, wq=None, wk=None, wv=None, rope_cos=None, rope_sin=None,
+                     scale=None, eps=1e-6):
+    """Token-level state access (comparison mode): token i reads S advanced by the block's tokens before it
+    (gated-linear update with per-token forget gates alpha_logit [B, L, H], None = 1).  Returns O; S is only read."""
+    q, k, v, g, S = _f64(q), _f64(k), _f64(v), _f64(g), _f64(S)
+    wq, wk, wv, rope_cos, rope_sin = _f64(wq), _f64(wk), _f64(wv), _f64(rope_cos), _f64(rope_sin)
+    alpha_logit = _f64(alpha_logit)
+    B, L, H, D = q.shape
+    assert S.shape == (B, H, D, D) and g.shape == (B, L, H)
+    assert alpha_logit is None or alpha_logit.shape == (B, L, H)
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    out = np.empty_like(q)
+    _load().arl2_oracle_step_token_level(
+        B, H, L, D, _p(q), _p(k), _p(v), _p(g), _p(alpha_logit), _p(S), _p(wq), _p(wk), _p(wv),
+        _p(rope_cos), _p(rope_sin), ctypes.c_double(scale), ctypes.c_double(eps), _p(out),
+    )
+    return out
+
+
 def attend_cache(q, k_cache, v_cache, scale=None):
     """Eq. 1: softmax attention of q [B, L, H, D] over a cache [B, Lk, H, D]; scale None = 1/sqrt(D)."""
     q, k_cache, v_cache = _f64(q), _f64(k_cache), _f64(v_cache)

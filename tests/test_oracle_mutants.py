@@ -43,6 +43,13 @@ MUTANTS = [
      "    arl2_oracle_commit(B, H, L, D, kc, vc, a, NULL, wk, wv, rope_cos, rope_sin, eps, 0, 0, NULL, NULL, S);",
      "    arl2_oracle_commit(B, H, L, D, kc, vc, a, NULL, wk, wv, rope_cos, rope_sin, eps, 0, 0, NULL, NULL, S);\n"
      "    arl2_oracle_step(B, H, L, D, q, kc, vc, g, S, wq, rope_cos, rope_sin, scale, eps, out);"),
+    ("token-level access reads the state after the token's own write",
+     "            step_row(b, h, i, H, L, D, 0, q, k, v, g, Sloc, wq, rope_cos, rope_sin, scale, eps,\n"
+     "                     out + off, scratch);\n            /* then the token's own write */",
+     "            /* then the token's own write */"),
+    ("token-level access decays the new term",
+     "Sloc[(size_t)d * D + e] = alpha * Sloc[(size_t)d * D + e] + kf[d] * vf[e];",
+     "Sloc[(size_t)d * D + e] = alpha * (Sloc[(size_t)d * D + e] + kf[d] * vf[e]);"),
     ("reset clears the wrong stream", "else memset(S + per * stream, 0, sizeof(double) * per);",
      "else memset(S, 0, sizeof(double) * per);"),
 ]

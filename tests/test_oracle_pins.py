@@ -550,6 +550,56 @@ def test_clean_pass_reads_the_state_before_it_commits(oracle):
                                rtol=1e-11, atol=1e-13)
 
 
+def test_token_level_access_against_sequential_commits_and_library_ops(oracle):
+    """Token-level state access (Sec. 4.3): token i reads the state advanced by the tokens before it.
+    (a) brute force through functions pinned elsewhere: commit the tokens one at a time with the per-token
+    gated-linear commit and read row i with the frame-level layer; (b) the causal linear-attention closed
+    form with library ops: O_inter_i = (prod_{j<i} alpha_j) Q'_i S + sum_{j<i} (prod_{j<m<i} alpha_m) (Q'_i . K'_j) V'_j;
+    (c) token 0 and one-token blocks coincide with the frame-level layer."""
+    B, L, H, D = 2, 6, 2, 8
+    q, k, v, g = rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, L, H)
+    al, S0 = rnd(B, L, H) + 1.0, rnd(B, H, D, D)
+    wq, wk, wv = rnd(H, D, D), rnd(H, D, D), rnd(H, D, D)
+    cos, sin = tables(L, D)
+    got = oracle.step_token_level(q, k, v, g, S0, al, wq, wk, wv, cos, sin)
+    # (a)
+    ref = np.empty_like(got)
+    S = S0.copy()
+    for i in range(L):
+        rows = np.array([(b, h, i) for b in range(B) for h in range(H)])
+        ref[:, i] = oracle.step_rows(q, k, v, g, S, rows, wq, cos, sin).reshape(B, H, D)
+        S = oracle.commit_decay_tokens(k[:, i:i + 1], v[:, i:i + 1], S, al[:, i:i + 1], wk, wv,
+                                       cos[i:i + 1], sin[i:i + 1])
+    np.testing.assert_allclose(got, ref, rtol=1e-11, atol=1e-13)
+    # (b): subtract the frame-level layer with the gate closed (the softmax branch alone)
+    intra = oracle.step(q, k, v, np.full_like(g, -800.0), S0, wq, cos, sin)
+    qf = torch.from_numpy(oracle.feature(q, wq, cos, sin, 1e-6, 0))
+    kf = torch.from_numpy(oracle.feature(k, wk, cos, sin, 1e-6, 0))
+    vf = torch.from_numpy(oracle.feature(v, wv, None, None, 1e-6, 1))
+    alpha = torch.from_numpy(sig(al))
+    incl = torch.cumprod(alpha, dim=1)                               # prod_{m<=i} alpha_m
+    excl = incl / alpha                                              # prod_{m<i}
+    decay = (excl[:, :, None, :] / incl[:, None, :, :])              # [b, i, j, h] = prod_{j<m<i} for j < i
+    mask = torch.tril(torch.ones(L, L), diagonal=-1)[None, :, :, None]
+    scores = torch.einsum("bihd,bjhd->bijh", qf, kf) * decay * mask
+    inter = excl[..., None] * torch.einsum("bihd,bhde->bihe", qf, torch.from_numpy(S0)) \
+        + torch.einsum("bijh,bjhe->bihe", scores, vf)
+    ref_b = intra + sig(g)[..., None] * inter.numpy()
+    np.testing.assert_allclose(got, ref_b, rtol=1e-10, atol=1e-12)
+    # (c)
+    frame = oracle.step(q, k, v, g, S0, wq, cos, sin)
+    np.testing.assert_array_equal(got[:, 0], frame[:, 0])
+    assert not np.allclose(got[:, 1:], frame[:, 1:])
+    one = oracle.step_token_level(q[:, :1], k[:, :1], v[:, :1], g[:, :1], S0, al[:, :1], wq, wk, wv, cos[:1], sin[:1])
+    np.testing.assert_array_equal(one, oracle.step(q[:, :1], k[:, :1], v[:, :1], g[:, :1], S0, wq, cos[:1], sin[:1]))
+    # gates absent = all gates open; the caller's state is never written
+    S_keep = S0.copy()
+    np.testing.assert_allclose(oracle.step_token_level(q, k, v, g, S0, None, wq, wk, wv, cos, sin),
+                               oracle.step_token_level(q, k, v, g, S0, np.full((B, L, H), 800.0), wq, wk, wv, cos, sin),
+                               rtol=1e-13, atol=1e-15)
+    np.testing.assert_array_equal(S0, S_keep)
+
+
 def test_reset(oracle):
     S = rnd(3, 2, 4, 4)
     r = oracle.reset(S, 1)
