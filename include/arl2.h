@@ -130,6 +130,25 @@ int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const voi
                       const float* d_gate_logits, void* d_out, void* stream);
 
 /*
+ * Token-level state access, the comparison mode of the paper's "State access granularity" ablation
+ * (Sec. 4.3; the layer itself uses frame-level access, Eq. 8).  Token i reads the state advanced by the
+ * tokens of the block before it -- each token sees its own sequentially accumulated state -- the
+ * gated-linear update being applied token by token on a private copy:
+ *   S^(0) = S,  S^(i+1) = alpha_i S^(i) + K'_i^T V'_i,
+ *   d_out[b,i,h,:] = softmax_j(<RoPE(q_i), RoPE(k_j)> scale) v_j + sigmoid(g[b,i,h]) Q'_i S^(i),
+ * with K' = L2Norm(RoPE(k Wphi_k)), V' = v Wphi_v of the pass's own k, v and alpha_i =
+ * sigmoid(d_alpha_logits[b,i,h]) (NULL: 1).  Token 0 reads S itself; a one-token block equals
+ * arl2_denoise_step.  READS the state, never writes it.  Computed chunkwise (128 tokens per chunk: a
+ * causal score matrix inside the chunk, the chunk-entry state in tensor memory across chunks) after the
+ * ordinary attention kernel has written the softmax branch.  Forget gates that stay below about 0.5
+ * for a whole chunk leave the fp32 range of the chunk factors.  Contexts with bf16 I/O, D = 128 and the
+ * headwise gate only (ARL2_ERR_UNSUPPORTED otherwise).  Other arguments as arl2_denoise_step.
+ */
+int arl2_denoise_step_token_level(arl2_ctx* ctx, const void* d_q, const void* d_k, const void* d_v,
+                                  const float* d_gate_logits, const float* d_alpha_logits, void* d_out,
+                                  void* stream);
+
+/*
  * The teacher's layer for comparison (Eq. 1): plain softmax attention of the current block's L
  * queries over a key/value cache of `cache_tokens` tokens (the blocks generated so far plus the
  * current one), all visible to every query:

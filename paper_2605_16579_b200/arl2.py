@@ -29,7 +29,7 @@ EXPORTS = (
     "arl2_workspace_bytes", "arl2_create", "arl2_set_params", "arl2_denoise_step", "arl2_commit",
     "arl2_reset", "arl2_get_state", "arl2_set_state", "arl2_sync_status", "arl2_launch_count",
     "arl2_set_profile_events", "arl2_commit_static_scratch", "arl2_commit_delta", "arl2_commit_tokens", "arl2_teacher_step", "arl2_commit_decay_tokens",
-    "arl2_step_kernel_name", "arl2_destroy", "arl2_last_error", "arl2_version", "arl2_debug_set_wait_limit", "arl2_clean_pass",
+    "arl2_step_kernel_name", "arl2_destroy", "arl2_last_error", "arl2_version", "arl2_debug_set_wait_limit", "arl2_clean_pass", "arl2_denoise_step_token_level",
 )
 
 
@@ -78,6 +78,8 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     lib.arl2_commit.argtypes = [vp] * 5
     lib.arl2_clean_pass.restype = ctypes.c_int
     lib.arl2_clean_pass.argtypes = [vp] * 8
+    lib.arl2_denoise_step_token_level.restype = ctypes.c_int
+    lib.arl2_denoise_step_token_level.argtypes = [vp] * 8
     lib.arl2_teacher_step.restype = ctypes.c_int
     lib.arl2_teacher_step.argtypes = [vp, vp, vp, vp, ctypes.c_int32, vp, vp]
     lib.arl2_commit_delta.restype = ctypes.c_int
@@ -224,6 +226,24 @@ class Layer:
         with torch.cuda.device(self.device):
             _check(load().arl2_clean_pass(self._ctx, _ptr(q), _ptr(k_clean), _ptr(v_clean), _ptr(gate_logits),
                                           _ptr(decay_logits), _ptr(out), _stream()), "arl2_clean_pass")
+        return out
+
+    def denoise_step_token_level(self, q, k, v, gate_logits, alpha_logits=None, out=None):
+        """Comparison mode: token i reads the state advanced by the block's tokens before it."""
+        shape = (self.B, self.L, self.H, self.D)
+        for t in (q, k, v):
+            self._want(t, shape, self.dtype, "q/k/v")
+        self._want(gate_logits, (self.B, self.L, self.H), torch.float32, "gate_logits")
+        if alpha_logits is not None:
+            self._want(alpha_logits, (self.B, self.L, self.H), torch.float32, "alpha_logits")
+        if out is None:
+            out = torch.empty(shape, dtype=self.dtype, device=self.device)
+        else:
+            self._want(out, shape, self.dtype, "out")
+        with torch.cuda.device(self.device):
+            _check(load().arl2_denoise_step_token_level(self._ctx, _ptr(q), _ptr(k), _ptr(v), _ptr(gate_logits),
+                                                        _ptr(alpha_logits), _ptr(out), _stream()),
+                   "arl2_denoise_step_token_level")
         return out
 
     def teacher_step(self, q, k_cache, v_cache, out=None):

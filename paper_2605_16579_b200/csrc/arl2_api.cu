@@ -352,6 +352,38 @@ int arl2_denoise_step(arl2_ctx* ctx, const void* d_q, const void* d_k, const voi
     return launch_step(ctx, d_q, k_rot, d_v, d_gate_logits, d_out, st);
 }
 
+int arl2_denoise_step_token_level(arl2_ctx* ctx, const void* d_q, const void* d_k, const void* d_v,
+                                  const float* d_gate_logits, const float* d_alpha_logits, void* d_out,
+                                  void* stream)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    if (!check_step_args("denoise_step_token_level", d_q, d_k, d_v, d_gate_logits, d_out)) return ARL2_ERR_INVALID_ARG;
+    if (!ctx->use_tc || (ctx->cfg.flags & (ARL2_FLAG_GATE_SCALAR | ARL2_FLAG_GATE_ELEMENTWISE))) {
+        set_error("denoise_step_token_level: built for bf16 I/O with D = 128 and the headwise gate only");
+        return ARL2_ERR_UNSUPPORTED;
+    }
+    cudaStream_t st = as_stream(stream);
+    // 1. the intra-block softmax branch alone (closed gate) ...
+    const void* k_rot = nullptr;
+    if (int r = rotate_k(ctx, d_k, &k_rot, st)) return r;
+    if (int r = launch_step(ctx, d_q, k_rot, d_v, nullptr, d_out, st)) return r;
+    // 2. ... then the causal readout adds sigmoid(g_i) Q'_i S^(i) to it
+    StepArgs a;
+    a.s = ctx->shape;
+    a.q = d_q; a.k_rot = d_k; a.v = d_v; a.gate = d_gate_logits;
+    a.state = ctx->state; a.wq = ctx->wq;
+    a.rope_cos = ctx->rope_cos; a.rope_sin = ctx->rope_sin;
+    a.out = d_out;
+    a.wait_limit = ctx->wait_limit;
+    a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status);
+    a.launch_parity = 0;
+    a.rope_h = ctx->rope_cos != nullptr ? ctx->ws + ctx->lay.rope_h : nullptr;
+    return account(ctx, tc_token_readout(a, d_alpha_logits,
+                                         reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wq_op),
+                                         reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wk_op),
+                                         reinterpret_cast<const __nv_bfloat16*>(ctx->ws + ctx->lay.wv_op), st));
+}
+
 int arl2_teacher_step(arl2_ctx* ctx, const void* d_q, const void* d_k_cache, const void* d_v_cache,
                       int32_t cache_tokens, void* d_out, void* stream)
 {

@@ -129,6 +129,11 @@ int tc_commit_partials(CommitArgs& a, const __nv_bfloat16* wk_op, cudaStream_t s
 // ... then S <- alpha S + (sum of slots) W_phi_v [- (sum of G slots) S_old], mirror written to state_bf16_next
 int tc_commit_finish(const CommitArgs& a, cudaStream_t st);
 
+// out += sigmoid(g) Q' S^(i): token-level state access (a.k_rot holds the RAW K here; a.out already holds the
+// softmax branch); alpha_logits [B, L, H] or nullptr
+int tc_token_readout(const StepArgs& a, const float* alpha_logits, const __nv_bfloat16* wq_op,
+                     const __nv_bfloat16* wk_op, const __nv_bfloat16* wv_op, cudaStream_t st);
+
 int tc_commit_tokens(const TokenCommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat16* wv_op,
                      const void* rope_h, uint32_t* status, cudaStream_t st);   // prepare + ordered scan
 
