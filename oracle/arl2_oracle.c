@@ -508,6 +508,37 @@ void arl2_oracle_commit_decay_tokens(int B, int H, int L, int D,
     }
 }
 
+/*
+ * The projections around the core (Sec. 3.1: Q = x W_q, K = x W_k, V = x W_v; Eq. 6-7: the gate logits
+ * x W_g and the output projection y = O W_o).  x, o, y: [rows, d] with rows = B * L and d = H * D, so that
+ * Q, K, V and O are the [B, L, H, D] tensors of the core; weights are (in, out), row-major; g: [rows, H].
+ */
+static void matmul_rows(long rows, int K, int N, const double *x, const double *w, double *y)
+{
+#pragma omp parallel for schedule(static)
+    for (long r = 0; r < rows; ++r)
+        for (int n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int kk = 0; kk < K; ++kk) acc += x[(size_t)r * K + kk] * w[(size_t)kk * N + n];
+            y[(size_t)r * N + n] = acc;
+        }
+}
+
+void arl2_oracle_project_in(long rows, int d, int H, const double *x,
+                            const double *w_q, const double *w_k, const double *w_v, const double *w_g,
+                            double *q, double *k, double *v, double *g)
+{
+    matmul_rows(rows, d, d, x, w_q, q);
+    matmul_rows(rows, d, d, x, w_k, k);
+    matmul_rows(rows, d, d, x, w_v, v);
+    matmul_rows(rows, d, H, x, w_g, g);
+}
+
+void arl2_oracle_project_out(long rows, int d, const double *o, const double *w_o, double *y)
+{
+    matmul_rows(rows, d, d, o, w_o, y);
+}
+
 /* S <- 0 for stream `stream` (or all streams when stream < 0): Algorithm 1, first line. */
 void arl2_oracle_reset(int B, int H, int D, int stream, double *S)
 {

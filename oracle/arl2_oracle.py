@@ -260,6 +260,30 @@ def commit_decay_tokens(kc, vc, S, alpha_logit, wk=None, wv=None, rope_cos=None,
     return S
 
 
+def project_in(x, w_q, w_k, w_v, w_g, H):
+    """Sec. 3.1 / Eq. 6: Q, K, V = x W_q, x W_k, x W_v as [B, L, H, D] and the gate logits x W_g [B, L, H]."""
+    x, w_q, w_k, w_v, w_g = _f64(x), _f64(w_q), _f64(w_k), _f64(w_v), _f64(w_g)
+    B, L, d = x.shape
+    assert d % H == 0 and w_q.shape == (d, d) and w_k.shape == (d, d) and w_v.shape == (d, d) and w_g.shape == (d, H)
+    q, k, v = (np.empty((B, L, d)) for _ in range(3))
+    g = np.empty((B, L, H))
+    _load().arl2_oracle_project_in(ctypes.c_long(B * L), d, H, _p(x), _p(w_q), _p(w_k), _p(w_v), _p(w_g),
+                                   _p(q), _p(k), _p(v), _p(g))
+    D = d // H
+    return q.reshape(B, L, H, D), k.reshape(B, L, H, D), v.reshape(B, L, H, D), g
+
+
+def project_out(o, w_o):
+    """Eq. 7: y = O W_o with O [B, L, H, D] read as [B, L, d]."""
+    o, w_o = _f64(o), _f64(w_o)
+    B, L, H, D = o.shape
+    d = H * D
+    assert w_o.shape == (d, d)
+    y = np.empty((B, L, d))
+    _load().arl2_oracle_project_out(ctypes.c_long(B * L), d, _p(o), _p(w_o), _p(y))
+    return y
+
+
 def reset(S, stream: int = -1):
     """S <- 0 for one stream or all (stream < 0).  Returns a new array."""
     S = _f64(S).copy()

@@ -50,6 +50,8 @@ MUTANTS = [
     ("token-level access decays the new term",
      "Sloc[(size_t)d * D + e] = alpha * Sloc[(size_t)d * D + e] + kf[d] * vf[e];",
      "Sloc[(size_t)d * D + e] = alpha * (Sloc[(size_t)d * D + e] + kf[d] * vf[e]);"),
+    ("projection weight read transposed", "acc += x[(size_t)r * K + kk] * w[(size_t)kk * N + n];",
+     "acc += x[(size_t)r * K + kk] * w[(size_t)n * K + kk];"),
     ("reset clears the wrong stream", "else memset(S + per * stream, 0, sizeof(double) * per);",
      "else memset(S, 0, sizeof(double) * per);"),
 ]

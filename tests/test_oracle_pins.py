@@ -600,6 +600,29 @@ def test_token_level_access_against_sequential_commits_and_library_ops(oracle):
     np.testing.assert_array_equal(S0, S_keep)
 
 
+def test_projections_against_library_matmul(oracle):
+    """Sec. 3.1 and Eq. 6-7: the projections are plain matrix products in the [B, L, H, D] layout of the core."""
+    B, L, H, D = 2, 5, 3, 4
+    d = H * D
+    x = rnd(B, L, d)
+    w_q, w_k, w_v, w_o, w_g = rnd(d, d), rnd(d, d), rnd(d, d), rnd(d, d), rnd(d, H)
+    q, k, v, g = oracle.project_in(x, w_q, w_k, w_v, w_g, H)
+    np.testing.assert_allclose(q, (x @ w_q).reshape(B, L, H, D), rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(k, (x @ w_k).reshape(B, L, H, D), rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(v, (x @ w_v).reshape(B, L, H, D), rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(g, x @ w_g, rtol=1e-12, atol=1e-13)
+    # head h of a token is columns [h D, (h + 1) D) of the projected row
+    np.testing.assert_allclose(q[1, 2, 1], x[1, 2] @ w_q[:, D:2 * D], rtol=1e-12, atol=1e-13)
+    o = rnd(B, L, H, D)
+    np.testing.assert_allclose(oracle.project_out(o, w_o), o.reshape(B, L, d) @ w_o, rtol=1e-12, atol=1e-13)
+    # identity weights pass the tokens through; a weight with one non-zero entry moves one channel
+    eye = np.eye(d)
+    np.testing.assert_array_equal(oracle.project_out(o, eye), o.reshape(B, L, d))
+    one = np.zeros((d, d)); one[3, 7] = 2.0
+    y = oracle.project_out(o, one)
+    np.testing.assert_allclose(y[..., 7], 2.0 * o.reshape(B, L, d)[..., 3]); assert not y[..., :7].any()
+
+
 def test_reset(oracle):
     S = rnd(3, 2, 4, 4)
     r = oracle.reset(S, 1)
