@@ -229,6 +229,28 @@ int arl2_commit_decay_tokens(arl2_ctx* ctx, const void* d_k_clean, const void* d
 int arl2_commit_tokens(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_clean,
                        const float* d_alpha_logits, const float* d_beta_logits, void* stream);
 
+/*
+ * The projections around the core (Sec. 3.1: Q = x W_q, K = x W_k, V = x W_v; Eq. 6: gate logits x W_g;
+ * Eq. 7: y = O W_o), so that the context is a drop-in attention module: x, y are [B, L, d] with
+ * d = H * D, and Q, K, V, O are the same memory read as [B, L, H, D].  Tensor-core contexts (bf16 I/O,
+ * D = 128) only.  All weights are bf16, row-major, indexed (in, out): W_q, W_k, W_v, W_o [d, d],
+ * W_g [d, H].
+ *   arl2_projection_workspace_bytes  bytes of the caller-owned packing buffer (256-byte aligned)
+ *   arl2_set_projections             copies W_q | W_k | W_v | W_g side by side into the packing buffer
+ *                                    (one GEMM then yields all four results) and keeps the W_o pointer;
+ *                                    the buffers must stay valid until replaced or the context is destroyed
+ *   arl2_project_in                  d_q, d_k, d_v [B, L, H, D] bf16 and d_gate_logits [B, L, H] fp32 from
+ *                                    d_x [B, L, d] bf16 -- one launch of a tcgen05 GEMM kernel
+ *   arl2_project_out                 d_y [B, L, d] bf16 = d_o [B, L, H, D] W_o -- one launch
+ * fp32 accumulation in tensor memory; results are rounded to bf16 (the gate logits stay fp32).
+ */
+size_t arl2_projection_workspace_bytes(const arl2_config* cfg);
+int arl2_set_projections(arl2_ctx* ctx, const void* d_wq, const void* d_wk, const void* d_wv, const void* d_wg,
+                         const void* d_wo, void* d_pack, size_t pack_bytes, void* stream);
+int arl2_project_in(arl2_ctx* ctx, const void* d_x, void* d_q, void* d_k, void* d_v, float* d_gate_logits,
+                    void* stream);
+int arl2_project_out(arl2_ctx* ctx, const void* d_o, void* d_y, void* stream);
+
 /* S <- 0 for stream `stream_index` (0..B-1) or all streams (-1): Algorithm 1, first line. */
 int arl2_reset(arl2_ctx* ctx, int32_t stream_index, void* stream);
 

@@ -30,6 +30,7 @@ EXPORTS = (
     "arl2_reset", "arl2_get_state", "arl2_set_state", "arl2_sync_status", "arl2_launch_count",
     "arl2_set_profile_events", "arl2_commit_static_scratch", "arl2_commit_delta", "arl2_commit_tokens", "arl2_teacher_step", "arl2_commit_decay_tokens",
     "arl2_step_kernel_name", "arl2_destroy", "arl2_last_error", "arl2_version", "arl2_debug_set_wait_limit", "arl2_clean_pass", "arl2_denoise_step_token_level",
+    "arl2_projection_workspace_bytes", "arl2_set_projections", "arl2_project_in", "arl2_project_out",
 )
 
 
@@ -80,6 +81,14 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     lib.arl2_clean_pass.argtypes = [vp] * 8
     lib.arl2_denoise_step_token_level.restype = ctypes.c_int
     lib.arl2_denoise_step_token_level.argtypes = [vp] * 8
+    lib.arl2_projection_workspace_bytes.restype = ctypes.c_size_t
+    lib.arl2_projection_workspace_bytes.argtypes = [cp]
+    lib.arl2_set_projections.restype = ctypes.c_int
+    lib.arl2_set_projections.argtypes = [vp] * 7 + [ctypes.c_size_t, vp]
+    lib.arl2_project_in.restype = ctypes.c_int
+    lib.arl2_project_in.argtypes = [vp] * 7
+    lib.arl2_project_out.restype = ctypes.c_int
+    lib.arl2_project_out.argtypes = [vp] * 4
     lib.arl2_teacher_step.restype = ctypes.c_int
     lib.arl2_teacher_step.argtypes = [vp, vp, vp, vp, ctypes.c_int32, vp, vp]
     lib.arl2_commit_delta.restype = ctypes.c_int
@@ -245,6 +254,46 @@ class Layer:
                                                         _ptr(alpha_logits), _ptr(out), _stream()),
                    "arl2_denoise_step_token_level")
         return out
+
+    def set_projections(self, w_q, w_k, w_v, w_g, w_o):
+        """W_q, W_k, W_v, W_o [d, d] and W_g [d, H], bf16, (in, out): the module around the core."""
+        d = self.H * self.D
+        for w in (w_q, w_k, w_v, w_o):
+            self._want(w, (d, d), torch.bfloat16, "projection weight")
+        self._want(w_g, (d, self.H), torch.bfloat16, "gate weight")
+        n = load().arl2_projection_workspace_bytes(ctypes.byref(self.cfg))
+        with torch.cuda.device(self.device):
+            self._pack = torch.empty(n, dtype=torch.uint8, device=self.device)
+            self._proj = (w_q, w_k, w_v, w_g, w_o)
+            _check(load().arl2_set_projections(self._ctx, _ptr(w_q), _ptr(w_k), _ptr(w_v), _ptr(w_g), _ptr(w_o),
+                                               _ptr(self._pack), n, _stream()), "arl2_set_projections")
+
+    def project_in(self, x, q=None, k=None, v=None, gate_logits=None):
+        """x [B, L, d] bf16 -> q, k, v [B, L, H, D] bf16 and gate logits [B, L, H] fp32."""
+        d = self.H * self.D
+        self._want(x, (self.B, self.L, d), torch.bfloat16, "x")
+        shape = (self.B, self.L, self.H, self.D)
+        q, k, v = (torch.empty(shape, dtype=torch.bfloat16, device=self.device) if t is None else t for t in (q, k, v))
+        if gate_logits is None:
+            gate_logits = torch.empty(self.B, self.L, self.H, dtype=torch.float32, device=self.device)
+        for t in (q, k, v):
+            self._want(t, shape, torch.bfloat16, "q/k/v")
+        self._want(gate_logits, (self.B, self.L, self.H), torch.float32, "gate_logits")
+        with torch.cuda.device(self.device):
+            _check(load().arl2_project_in(self._ctx, _ptr(x), _ptr(q), _ptr(k), _ptr(v), _ptr(gate_logits), _stream()),
+                   "arl2_project_in")
+        return q, k, v, gate_logits
+
+    def project_out(self, o, y=None):
+        """o [B, L, H, D] bf16 -> y [B, L, d] bf16 = o W_o."""
+        d = self.H * self.D
+        self._want(o, (self.B, self.L, self.H, self.D), torch.bfloat16, "o")
+        if y is None:
+            y = torch.empty(self.B, self.L, d, dtype=torch.bfloat16, device=self.device)
+        self._want(y, (self.B, self.L, d), torch.bfloat16, "y")
+        with torch.cuda.device(self.device):
+            _check(load().arl2_project_out(self._ctx, _ptr(o), _ptr(y), _stream()), "arl2_project_out")
+        return y
 
     def teacher_step(self, q, k_cache, v_cache, out=None):
         """Eq. 1: softmax attention of q [B, L, H, D] over a cache [B, Lk, H, D] (no rotation, no state)."""

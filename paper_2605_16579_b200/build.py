@@ -12,7 +12,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libarl2.so")
-SOURCES = ["arl2_api.cu", "arl2_simt.cu", "arl2_tc.cu", "arl2_tc_commit.cu", "arl2_tc_token_readout.cu", "arl2_noalloc.cu"]
+SOURCES = ["arl2_api.cu", "arl2_simt.cu", "arl2_tc.cu", "arl2_tc_commit.cu", "arl2_tc_token_readout.cu", "arl2_tc_gemm.cu", "arl2_noalloc.cu"]
 HEADERS = [os.path.join(CSRC, "arl2_internal.h"), os.path.join(ROOT, "include", "arl2.h")]
 
 

@@ -137,6 +137,10 @@ struct arl2_ctx {
     int mirror;            // which of the two bf16 copies of S is current
     cudaEvent_t ev_before, ev_after;  // one-shot timing hook around the step kernel
     uint32_t wait_limit;   // 0: the kernels' default bound; n: waits give up after n - 1 polls (test hook)
+    // projections around the core (arl2_set_projections)
+    const void* w_pack;    // [d, 3 d + gate pad] bf16: W_q | W_k | W_v | W_g (zero padded)
+    const void* w_o;       // [d, d] bf16
+    int pack_cols;
 };
 
 namespace {
@@ -220,6 +224,8 @@ int arl2_create(const arl2_config* cfg, void* d_state, void* d_workspace, size_t
     ctx->launches = 0;
     ctx->step_calls = 0;
     ctx->mirror = 0;
+    ctx->w_pack = ctx->w_o = nullptr;
+    ctx->pack_cols = 0;
     ctx->wait_limit = cfg->flags >> ARL2_FLAG_DEBUG_WAIT_LIMIT_SHIFT;
     ctx->ev_before = ctx->ev_after = nullptr;
     int r = account(ctx, fill_zero(ctx->ws + lay.status, kStatusWords * sizeof(uint32_t),
@@ -609,6 +615,100 @@ int arl2_commit_decay_tokens(arl2_ctx* ctx, const void* d_k_clean, const void* d
     int r = account(ctx, decay_weights(ctx->shape, d_alpha_logits, w, total, as_stream(stream)));
     if (r != ARL2_OK) return r;
     return commit_impl(ctx, d_k_clean, d_v_clean, total, 2, w, true, stream);
+}
+
+namespace {
+// the gate logits ride in a last, zero-padded segment so that the packed width is a multiple of 256
+int gate_pad_cols(int d) { return (3 * d) % 256 == 0 ? 256 : 128; }
+}  // namespace
+
+size_t arl2_projection_workspace_bytes(const arl2_config* cfg)
+{
+    if (!valid_config(cfg)) return 0;
+    const size_t d = (size_t)cfg->H * cfg->D;
+    return align_up(d * (3 * d + gate_pad_cols((int)d)) * 2);
+}
+
+int arl2_set_projections(arl2_ctx* ctx, const void* d_wq, const void* d_wk, const void* d_wv, const void* d_wg,
+                         const void* d_wo, void* d_pack, size_t pack_bytes, void* stream)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    if (!ctx->use_tc) {
+        set_error("set_projections: built for bf16 I/O with D = 128 (the tensor-core context) only");
+        return ARL2_ERR_UNSUPPORTED;
+    }
+    if (!d_wq || !d_wk || !d_wv || !d_wg || !d_wo || !d_pack) {
+        set_error("set_projections: the five weights and the packing buffer must not be NULL");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    const size_t d = (size_t)ctx->cfg.H * ctx->cfg.D;
+    const int pad = gate_pad_cols((int)d);
+    const size_t cols = 3 * d + pad;
+    if (pack_bytes < d * cols * 2 || reinterpret_cast<uintptr_t>(d_pack) % 256 != 0 ||
+        reinterpret_cast<uintptr_t>(d_wo) % 16 != 0) {
+        set_error("set_projections: the packing buffer needs %zu bytes, 256-byte aligned; W_o 16-byte aligned", d * cols * 2);
+        return ARL2_ERR_WORKSPACE;
+    }
+    cudaStream_t st = as_stream(stream);
+    uint8_t* pack = static_cast<uint8_t*>(d_pack);
+    cudaError_t e = cudaMemsetAsync(pack, 0, d * cols * 2, st);
+    const void* src[3] = {d_wq, d_wk, d_wv};
+    for (int i = 0; i < 3 && e == cudaSuccess; ++i)
+        e = cudaMemcpy2DAsync(pack + i * d * 2, cols * 2, src[i], d * 2, d * 2, d, cudaMemcpyDeviceToDevice, st);
+    if (e == cudaSuccess)
+        e = cudaMemcpy2DAsync(pack + 3 * d * 2, cols * 2, d_wg, (size_t)ctx->cfg.H * 2, (size_t)ctx->cfg.H * 2, d,
+                              cudaMemcpyDeviceToDevice, st);
+    if (e != cudaSuccess) { set_error("set_projections: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
+    ctx->w_pack = d_pack;
+    ctx->w_o = d_wo;
+    ctx->pack_cols = (int)cols;
+    return ARL2_OK;
+}
+
+int arl2_project_in(arl2_ctx* ctx, const void* d_x, void* d_q, void* d_k, void* d_v, float* d_gate_logits,
+                    void* stream)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    if (ctx->w_pack == nullptr) { set_error("project_in: call arl2_set_projections first"); return ARL2_ERR_INVALID_ARG; }
+    if (!d_x || !d_q || !d_k || !d_v || !d_gate_logits) {
+        set_error("project_in: x, q, k, v and gate_logits must not be NULL");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    if ((reinterpret_cast<uintptr_t>(d_x) | reinterpret_cast<uintptr_t>(d_q) | reinterpret_cast<uintptr_t>(d_k) |
+         reinterpret_cast<uintptr_t>(d_v)) % 32 != 0) {
+        set_error("project_in: x, q, k and v must be 32-byte aligned");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    const int d = ctx->cfg.H * ctx->cfg.D;
+    GemmArgs a;
+    a.a = d_x; a.b = ctx->w_pack;
+    a.M = ctx->cfg.B * ctx->cfg.L; a.N = ctx->pack_cols; a.K = d;
+    a.out[0] = d_q; a.out[1] = d_k; a.out[2] = d_v;
+    a.seg_cols = d; a.ld_out = d; a.n_bf16_seg = 3;
+    a.out_f32 = d_gate_logits; a.f32_cols = ctx->cfg.H; a.ld_f32 = ctx->cfg.H;
+    a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status);
+    a.wait_limit = ctx->wait_limit;
+    return account(ctx, tc_gemm(a, as_stream(stream)));
+}
+
+int arl2_project_out(arl2_ctx* ctx, const void* d_o, void* d_y, void* stream)
+{
+    if (!check_ctx(ctx)) return ARL2_ERR_INVALID_ARG;
+    if (ctx->w_o == nullptr) { set_error("project_out: call arl2_set_projections first"); return ARL2_ERR_INVALID_ARG; }
+    if (!d_o || !d_y || d_o == d_y) { set_error("project_out: o and y must be two non-NULL buffers"); return ARL2_ERR_INVALID_ARG; }
+    if ((reinterpret_cast<uintptr_t>(d_o) | reinterpret_cast<uintptr_t>(d_y)) % 32 != 0) {
+        set_error("project_out: o and y must be 32-byte aligned");
+        return ARL2_ERR_INVALID_ARG;
+    }
+    const int d = ctx->cfg.H * ctx->cfg.D;
+    GemmArgs a;
+    a.a = d_o; a.b = ctx->w_o;
+    a.M = ctx->cfg.B * ctx->cfg.L; a.N = d; a.K = d;
+    a.out[0] = d_y;
+    a.seg_cols = d; a.ld_out = d; a.n_bf16_seg = 1;
+    a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status);
+    a.wait_limit = ctx->wait_limit;
+    return account(ctx, tc_gemm(a, as_stream(stream)));
 }
 
 int arl2_reset(arl2_ctx* ctx, int32_t stream_index, void* stream)

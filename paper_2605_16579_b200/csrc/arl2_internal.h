@@ -137,6 +137,21 @@ int tc_token_readout(const StepArgs& a, const float* alpha_logits, const __nv_bf
 int tc_commit_tokens(const TokenCommitArgs& a, const __nv_bfloat16* wk_op, const __nv_bfloat16* wv_op,
                      const void* rope_h, uint32_t* status, cudaStream_t st);   // prepare + ordered scan
 
+// C[M, N] = A[M, K] B[K, N] on tensor cores (bf16 operands, row-major); the columns of C are routed to up to
+// four bf16 tensors of seg_cols columns each (row stride ld_out) and, after them, one fp32 tensor.
+struct GemmArgs {
+    const void* a;        // [M, K] bf16
+    const void* b;        // [K, N] bf16
+    int M, N, K;
+    void* out[4] = {nullptr, nullptr, nullptr, nullptr};
+    int seg_cols = 0, ld_out = 0, n_bf16_seg = 0;
+    float* out_f32 = nullptr;
+    int f32_cols = 0, ld_f32 = 0;
+    uint32_t* status = nullptr;
+    uint32_t wait_limit = 0;
+};
+int tc_gemm(const GemmArgs& a, cudaStream_t st);
+
 void set_error(const char* fmt, ...);
 
 }  // namespace arl2
