@@ -335,6 +335,104 @@ def short_leg(name, dev, blocks=8):
             "l2": "two resident input sets of %d MiB" % (sum(t.numel() * t.element_size() for t in sets[0]) >> 20)}
 
 
+def stack_leg(dev, horizons=(1, 2, 4, 8, 16), n_layers=30, n_hybrid=23):
+    """The attention modules of a whole model, measured: 30 layers of (x -> W_q | W_k | W_v | W_g -> attention
+    core -> W_o) per denoise pass at the base model's geometry (d = 1536, H = 12, 4680 tokens per block), once
+    with every layer a softmax teacher over a key/value cache of n blocks (Eq. 1) and once with 23 of the 30
+    layers replaced by the hybrid layer (the paper's 75 % model).  Every layer has its own weights, state and
+    cache; the feed-forward blocks, norms and residuals between the attention modules are not part of this
+    path and are left out of both arms.  Returns ms per pass against the horizon and the GEMM rates."""
+    import torch
+
+    from paper_2605_16579_b200 import arl2, workload
+
+    cfg = workload.CONFIGS["chunked"]
+    pk = peaks()
+    B, H, L, D = cfg.B, cfg.H, cfg.L, cfg.D
+    d = H * D
+    gen = torch.Generator(device="cpu").manual_seed(4242)
+    rnd = lambda *s: (torch.randn(*s, generator=gen) * d ** -0.5).to(torch.bfloat16).to(dev)  # noqa: E731
+    wq, wk, wv = (w.to(dev) for w in workload.feature_weights(cfg))
+    cos, sin = (t.to(dev) for t in workload.rope_tables(L, D))
+    layers = []
+    for _ in range(n_layers):
+        layer = arl2.Layer(B, H, L, D, "bf16", device=dev)
+        layer.set_params(wq, wk, wv, cos, sin)
+        layer.set_projections(rnd(d, d), rnd(d, d), rnd(d, d), rnd(d, H), rnd(d, d))
+        kc, vc, a = (t.to(dev) for t in workload.commit_inputs(cfg, 0))
+        layer.commit(kc, vc, a)
+        layers.append(layer)
+    nmax = max(horizons)
+    caches = [(torch.randn(B, nmax * L, H, D, device=dev).to(torch.bfloat16),
+               torch.randn(B, nmax * L, H, D, device=dev).to(torch.bfloat16)) for _ in range(n_layers)]
+    xs = [torch.randn(B, L, d, device=dev).to(torch.bfloat16) for _ in range(2)]
+    q = torch.empty(B, L, H, D, dtype=torch.bfloat16, device=dev)
+    k, v, o = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+    g = torch.empty(B, L, H, device=dev)
+
+    def one_pass(hybrid_set, n):
+        x, y = xs
+        for i, layer in enumerate(layers):
+            if i in hybrid_set:
+                layer.project_in(x, q, k, v, g)
+                layer.denoise_step(q, k, v, g, out=o)
+            else:
+                # the block's keys and values land at the tail of this layer's cache
+                ck, cv = caches[i]
+                k_cur, v_cur = ck[:, (n - 1) * L:n * L], cv[:, (n - 1) * L:n * L]
+                layer.project_in(x, q, k_cur, v_cur, g)
+                layer.teacher_step(q, ck[:, :n * L], cv[:, :n * L], out=o)
+            layer.project_out(o, y)
+            x, y = y, x
+
+    def timed(hybrid_set, n, reps=4):
+        for _ in range(2):
+            one_pass(hybrid_set, n)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            one_pass(hybrid_set, n)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    # which layers stay softmax: spread over the depth (the paper selects them by sensitivity; the cost
+    # does not depend on which ones they are)
+    keep = {round(j * (n_layers - 1) / (n_layers - n_hybrid - 1)) for j in range(n_layers - n_hybrid)}
+    hybrid_set = set(range(n_layers)) - keep
+    res = {"geometry": f"B={B} H={H} D={D} d={d} L={L}, {n_layers} layers, {n_hybrid} hybrid + {n_layers - n_hybrid} softmax",
+           "cache_blocks": list(horizons), "all_softmax_ms": [], "hybrid75_ms": [], "speedup": []}
+    for n in horizons:
+        t_all = timed(set(), n)
+        t_hyb = timed(hybrid_set, n)
+        res["all_softmax_ms"].append(t_all)
+        res["hybrid75_ms"].append(t_hyb)
+        res["speedup"].append(t_all / t_hyb)
+    # the two GEMMs on their own
+    def gemm_ms(fn, reps=20):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(reps):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+    t_in = gemm_ms(lambda i=0: layers[i % n_layers].project_in(xs[0], q, k, v, g))
+    t_out = gemm_ms(lambda i=0: layers[i % n_layers].project_out(o, xs[1]))
+    f_in, f_out = 2.0 * B * L * d * (3 * d + H), 2.0 * B * L * d * d
+    res["project_in"] = {"ms": t_in, "tflops": f_in / t_in / 1e9, "frac_of_burst": f_in / t_in / 1e9 / pk["bf16_tflops"]}
+    res["project_out"] = {"ms": t_out, "tflops": f_out / t_out / 1e9, "frac_of_burst": f_out / t_out / 1e9 / pk["bf16_tflops"]}
+    res["kv_cache_bytes_per_block_per_layer"] = 2 * B * L * d * 2
+    res["state_bytes_per_layer"] = B * H * D * D * 4
+    for layer in layers:
+        layer.sync_status()
+    return res
+
+
 def launcher_command(n, argv, port=None):
     """The command that runs this file as n ranks of one node (what a caller would type)."""
     port = port or 29400 + os.getpid() % 500
@@ -554,6 +652,45 @@ def run_ours(args):
     tok.sync_status()
     del tok
 
+    # the clean pass of a block: the fused call against the two separate calls, alternating so that
+    # both see the same clocks; and the token-level state access mode beside the frame-level pass
+    clean_ms = None
+    if layer.step_kernel == "tcgen05":
+        q0, _, _, g0 = dev_sets[0]
+        kc0, vc0, a0 = dev_commit
+
+        def run_ms(fn, reps):
+            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c0.record()
+            for _ in range(reps):
+                fn()
+            c1.record()
+            torch.cuda.synchronize()
+            return c0.elapsed_time(c1) / reps
+
+        def two_calls():
+            layer.denoise_step(q0, kc0, vc0, g0, out=out)
+            layer.commit(kc0, vc0, a0)
+
+        def fused():
+            layer.clean_pass(q0, kc0, vc0, g0, a0, out=out)
+
+        layer.reset()
+        for fn in (two_calls, fused):
+            run_ms(fn, 3)
+        t_two, t_fused = [], []
+        for _ in range(4):
+            t_two.append(run_ms(two_calls, 8))
+            t_fused.append(run_ms(fused, 8))
+        alpha0 = workload.token_gate_logits(cfg, commit_block)[0].to(dev)
+        run_ms(lambda: layer.denoise_step_token_level(q0, kc0, vc0, g0, alpha0, out=out), 2)
+        t_tok = run_ms(lambda: layer.denoise_step_token_level(q0, kc0, vc0, g0, alpha0, out=out), 5)
+        t_frame = run_ms(lambda: layer.denoise_step(q0, kc0, vc0, g0, out=out), 5)
+        clean_ms = {"step_then_commit": statistics.median(t_two), "clean_pass": statistics.median(t_fused),
+                    "frame_level_pass": t_frame, "token_level_pass": t_tok}
+        layer.sync_status()
+        layer.reset()
+
     # the teacher's layer on the same kernels (Eq. 1 over a key/value cache that grows by one block
     # per generated block) against the horizon: its cost per denoise pass grows, the layer's does not
     teacher = None
@@ -574,16 +711,12 @@ def run_ours(args):
             teacher["ms_per_pass"].append(statistics.mean(ts))
             del kcache, vcache
         layer.sync_status()
-        # derived from the measured figures (no further kernel runs): attention time per denoise pass
-        # of a 30-layer stack, all teacher layers against 23 hybrid + 7 teacher layers (the paper's
-        # 75 %-replaced model); the hybrid layer's time does not depend on the horizon
-        hyb = statistics.mean(a.elapsed_time(b) for a, b in step_events)
-        teacher["stack30_teacher_ms"] = [30 * t for t in teacher["ms_per_pass"]]
-        teacher["stack30_hybrid75_ms"] = [23 * hyb + 7 * t for t in teacher["ms_per_pass"]]
-
     batched = None
     if rank == 0 and world == 1 and cfg.name == "long" and not args.no_batched_leg:
         batched = short_leg("batched", dev, blocks=8)
+    stack = None
+    if rank == 0 and world == 1 and layer.step_kernel == "tcgen05" and not args.no_stack:
+        stack = stack_leg(dev)
 
     ms_total, ms_e2e, kern_mean, pass_mean = max_over_ranks(
         [ms_total, ms_e2e, statistics.mean(kern_ms), statistics.mean(pass_ms)], world, dev)
@@ -643,6 +776,7 @@ def run_ours(args):
             "clocks": clocks,
             "horizon": horizon_report(block_ms, mem_marks, layer.workspace_bytes + layer.state.numel() * 4),
             "commit_ms": commit_ms,
+            "clean_pass_ms": clean_ms,
             # the commit is HBM-bound by its arithmetic intensity (about 175 flop/B); the same bytes
             # serve the delta and per-token-decay variants, whose extra work is on-chip
             "commit_roofline": {
@@ -653,6 +787,7 @@ def run_ours(args):
             },
             "teacher_horizon": teacher,
             "batched_leg": batched,
+            "module_stack": stack,
         }
         if world == 1 and not args.no_cpu_baseline:
             s = CpuSample(cfg)
@@ -685,6 +820,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-teacher", action="store_true", help="skip the teacher-attention horizon leg")
     ap.add_argument("--no-batched-leg", action="store_true", help="skip the short run of the batched workload")
+    ap.add_argument("--no-stack", action="store_true", help="skip the 30-layer module stack leg")
     ap.add_argument("--traffic-probe", action="store_true",
                     help="set up, run four denoise passes and a commit, exit (for a one-launch profiler capture)")
     args = ap.parse_args()

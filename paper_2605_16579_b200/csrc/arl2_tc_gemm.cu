@@ -52,6 +52,19 @@ struct GemmParams {
     uint32_t spin_limit;
 };
 
+// Tile order: bands of kGBand row tiles; inside a band the row tile varies fastest, then the column
+// tile, so the CTAs running at one time share a few B tiles and a band of A that stays in L2.
+constexpr int kGBand = 32;
+__device__ __forceinline__ void tile_origin(int t, const GemmParams& p, int& m0, int& n0)
+{
+    const int per_band = kGBand * p.n_tiles;
+    const int band = t / per_band, in_band = t - band * per_band;
+    const int rows = min(kGBand, p.m_tiles - band * kGBand);   // the last band may be shorter
+    const int nt = in_band / rows;
+    m0 = (band * kGBand + in_band - nt * rows) * kGBM;
+    n0 = nt * kGBN;
+}
+
 __global__ void __launch_bounds__(kGThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const GemmParams p)
 {
@@ -98,7 +111,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             bool ok = true;
             uint32_t n = 0;
             for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
-                const int m0 = (t % p.m_tiles) * kGBM, n0 = (t / p.m_tiles) * kGBN;
+                int m0, n0;
+                tile_origin(t, p, m0, n0);
                 for (int kb = 0; kb < n_kb && ok; ++kb, ++n) {
                     const uint32_t s = n % kGStages;
                     if (n >= (uint32_t)kGStages) ok = wait_bar(bars + 8 * (kGBarEmpty0 + s), ((n / kGStages) - 1) & 1u, ab, 120);
@@ -166,7 +180,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         uint32_t it = 0;
         for (int t = blockIdx.x; t < total && ok; t += gridDim.x, ++it) {
             const uint32_t buf = it & 1u;
-            const int m0 = (t % p.m_tiles) * kGBM, n0 = (t / p.m_tiles) * kGBN;
+            int m0, n0;
+            tile_origin(t, p, m0, n0);
             const int row = m0 + r;
             ok = wait_bar(bars + 8 * (kGBarAccFull0 + buf), (it >> 1) & 1u, ab, 123);
             if (!ok) break;
