@@ -2,7 +2,8 @@
 // x W_g and y = O W_o) as one persistent tcgen05 GEMM kernel: C[M, N] = A[M, K] B[K, N], bf16 operands,
 // fp32 accumulation in tensor memory, bf16 (or, for the gate logits, fp32) results.
 //
-// Tiles of 128 x 256 outputs, the contraction in blocks of 64; one CTA per SM walks its tiles.
+// Tiles of 128 x 256 outputs (128 x 128 when N <= 128), the contraction in blocks of 64; one CTA per
+// SM walks its tiles.
 //   warp 0     TMA producer: per k-block the A tile [128 x 64] (K-major) and the B tile [64 x 256]
 //              (rows = contraction index, as it lies in a row-major (in, out) weight) through a
 //              4-stage ring
@@ -19,10 +20,10 @@ namespace arl2 {
 
 namespace {
 
-constexpr int kGBM = 128, kGBN = 256, kGBK = 64;
+constexpr int kGBM = 128, kGBK = 64;   // the tile is kGBM x BN outputs, BN = 256 or 128 (template)
 constexpr int kGStages = 4;
 constexpr int kGABytes = kGBM * kGBK * 2;             // 16 KB
-constexpr int kGBBytes = kGBK * kGBN * 2;             // 32 KB: 4 groups of 64 columns x 64 rows
+constexpr int kGBBytes = kGBK * 256 * 2;              // up to 32 KB: groups of 64 columns x 64 rows
 constexpr int kGStageBytes = kGABytes + kGBBytes;
 constexpr int kGOffBars = kGStages * kGStageBytes;
 constexpr int kGemmSmemBytes = kGOffBars + 256 + 1024;
@@ -40,7 +41,7 @@ static_assert(kGNumBars * 8 + 16 <= 256, "barrier block");
 
 struct GemmParams {
     int M, N, K;
-    int m_tiles, n_tiles;
+    int m_tiles, n_tiles, bn;
     // output routing: column n of the product belongs to segment n / seg_cols; segments
     // 0 .. n_bf16_seg - 1 are bf16 tensors with row stride ld_out, the one after them (if any) is the
     // fp32 tensor out_f32 with f32_cols valid columns and row stride ld_f32
@@ -62,9 +63,10 @@ __device__ __forceinline__ void tile_origin(int t, const GemmParams& p, int& m0,
     const int rows = min(kGBand, p.m_tiles - band * kGBand);   // the last band may be shorter
     const int nt = in_band / rows;
     m0 = (band * kGBand + in_band - nt * rows) * kGBM;
-    n0 = nt * kGBN;
+    n0 = nt * p.bn;
 }
 
+template <int BN>
 __global__ void __launch_bounds__(kGThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const GemmParams p)
 {
@@ -119,10 +121,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     if (!ok) break;
                     const uint32_t bar = bars + 8 * (kGBarFull0 + s);
                     const uint32_t dst = smem_base + s * kGStageBytes;
-                    mbar_expect_tx(bar, kGStageBytes);
+                    mbar_expect_tx(bar, kGABytes + kGBK * BN * 2);
                     tma_load_2d(dst, &tm_a, bar, kb * kGBK, m0);
 #pragma unroll
-                    for (int g = 0; g < kGBN / 64; ++g)
+                    for (int g = 0; g < BN / 64; ++g)
                         tma_load_2d(dst + kGABytes + g * (kGBK * 128), &tm_b, bar, n0 + g * 64, kb * kGBK);
                 }
             }
@@ -142,7 +144,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(desc_hi));
                 return d;
             };
-            constexpr uint32_t idesc = idesc_bf16(kGBM, kGBN, 0, 1);   // A K-major, B rows = contraction index
+            constexpr uint32_t idesc = idesc_bf16(kGBM, BN, 0, 1);   // A K-major, B rows = contraction index
             bool ok = true;
             uint32_t n = 0, it = 0;
             for (int t = blockIdx.x; t < total && ok; t += gridDim.x, ++it) {
@@ -160,7 +162,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     const uint32_t b_lo = ((smem_base + s * kGStageBytes + kGABytes) >> 4) | kLboB;
 #pragma unroll
                     for (int ks = 0; ks < kGBK / 16; ++ks)
-                        mma_ss(tmem_base + buf * kGBN, desc64(a_lo + (uint32_t)((ks * 32) >> 4)),
+                        mma_ss(tmem_base + buf * 256, desc64(a_lo + (uint32_t)((ks * 32) >> 4)),
                                desc64(b_lo + (uint32_t)(ks * (2048 >> 4))), idesc, (kb > 0 || ks > 0) ? 1u : 0u);
                     mma_commit(bars + 8 * (kGBarEmpty0 + s));
                 }
@@ -187,9 +189,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             if (!ok) break;
             tc_fence_after();
 #pragma unroll 1
-            for (int c = 0; c < kGBN / 32; ++c) {
+            for (int c = 0; c < BN / 32; ++c) {
                 uint32_t o[32];
-                tmem_ld32(lane_base + buf * kGBN + c * 32, o);
+                tmem_ld32(lane_base + buf * 256 + c * 32, o);
                 tmem_wait_ld();
                 const int n = n0 + c * 32;                                  // 32 columns lie inside one segment
                 if (row >= p.M || n >= p.N) continue;
@@ -250,7 +252,11 @@ DeviceSetup g_setup[kMaxDevices];
 int tc_gemm(const GemmArgs& a, cudaStream_t st)
 {
     int num_sms = 0;
-    if (int r = device_setup_once(g_setup_mutex, g_setup, [] { return opt_in_smem(tc_gemm_kernel, kGemmSmemBytes); }, &num_sms))
+    if (int r = device_setup_once(g_setup_mutex, g_setup, [] {
+            cudaError_t e = opt_in_smem(tc_gemm_kernel<256>, kGemmSmemBytes);
+            if (e == cudaSuccess) e = opt_in_smem(tc_gemm_kernel<128>, kGemmSmemBytes);
+            return e;
+        }, &num_sms))
         return r;
     if (a.K % kGBK != 0 || a.N % 64 != 0 || a.seg_cols % 32 != 0 || a.M < 1) {
         set_error("tc_gemm: K must be a multiple of %d, N of 64 and the segment width of 32 (got M=%d N=%d K=%d)",
@@ -263,7 +269,11 @@ int tc_gemm(const GemmArgs& a, cudaStream_t st)
     GemmParams p;
     p.M = a.M; p.N = a.N; p.K = a.K;
     p.m_tiles = (a.M + kGBM - 1) / kGBM;
-    p.n_tiles = (a.N + kGBN - 1) / kGBN;   // columns past N are fetched as zeros and not stored
+    // 256 columns per tile: a 128 x 128 tile would read as many operand bytes from shared memory per MMA
+    // clock as shared memory delivers (measured: 673 against 871 TFLOP/s on the 1536-wide output
+    // projection, although its 444 tiles fill three waves exactly); the narrow tile serves N <= 128 only
+    p.bn = a.N <= 128 ? 128 : 256;
+    p.n_tiles = (a.N + p.bn - 1) / p.bn;   // columns past N are fetched as zeros and not stored
     for (int i = 0; i < 4; ++i) p.out[i] = static_cast<__nv_bfloat16*>(a.out[i]);
     p.seg_cols = a.seg_cols; p.ld_out = a.ld_out; p.n_bf16_seg = a.n_bf16_seg;
     p.out_f32 = a.out_f32; p.f32_cols = a.f32_cols; p.ld_f32 = a.ld_f32;
@@ -271,7 +281,10 @@ int tc_gemm(const GemmArgs& a, cudaStream_t st)
     p.spin_limit = a.wait_limit ? a.wait_limit - 1 : kSpinLimit;
     const int total = p.m_tiles * p.n_tiles;
     const int grid = total < num_sms ? total : num_sms;
-    tc_gemm_kernel<<<grid, kGThreads, kGemmSmemBytes, st>>>(tm_a, tm_b, p);
+    if (p.bn == 256)
+        tc_gemm_kernel<256><<<grid, kGThreads, kGemmSmemBytes, st>>>(tm_a, tm_b, p);
+    else
+        tc_gemm_kernel<128><<<grid, kGThreads, kGemmSmemBytes, st>>>(tm_a, tm_b, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_error("launch of tc_gemm_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
     return 1;
