@@ -58,6 +58,10 @@ typedef enum {
 #define ARL2_FLAG_GATE_ELEMENTWISE 8u /* d_gate_logits is [B, L, H, D]: one gate per output channel */
 #define ARL2_FLAG_TOKEN_GATES 2u /* reserve workspace for arl2_commit_tokens (3 fp32 copies of a
                                     [B, H, ceil(L/64)*64, D] tensor)                             */
+/* arl2_commit_tokens: each token's prediction is made against the state after its own forget gate,
+   S <- alpha_l S + beta_l K'_l^T (V'_l - K'_l (alpha_l S)) -- the Gated DeltaNet's form -- instead of Eq. 4
+   as printed (prediction against the undecayed state).                                                   */
+#define ARL2_FLAG_DELTA_DECAYED_PREDICTION 32u
 /* Test hook for the time-out path: every bounded wait inside the tensor-core kernels gives up
    after `polls` polls of its barrier (0 .. 65534) instead of 2^24.  With 0 the first wait of a
    launch expires at once: the kernel records ARL2_ERR_TIMEOUT and the wait's site in the status

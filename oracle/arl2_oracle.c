@@ -421,7 +421,10 @@ void arl2_oracle_clean_pass(int B, int H, int L, int D,
  *   for j = 0..L-1:   S <- alpha_j S + beta_j K'_j^T (V'_j - K'_j S)
  * where the S on the right is the state before token j (both uses), alpha_j =
  * sigmoid(alpha_logit[b,j,h]), beta_j = sigmoid(beta_logit[b,j,h]).  Eq. 4 is taken as
- * printed: the prediction K'_j S uses the undecayed previous state.
+ * printed: the prediction K'_j S uses the undecayed previous state.  With `decayed` non-zero the
+ * other reading is taken instead, the one of the Gated DeltaNet the paper builds on: the token's
+ * prediction is made against the state after its forget gate,
+ *   S <- alpha_j S + beta_j K'_j^T (V'_j - K'_j (alpha_j S)).
  *   alpha_logit, beta_logit  [B, L, H]; NULL = gate fixed at 1.
  */
 static void commit_head_tokens(int b, int h, int H, int L, int D,
@@ -429,7 +432,7 @@ static void commit_head_tokens(int b, int h, int H, int L, int D,
                                const double *alpha_logit, const double *beta_logit,
                                const double *wk, const double *wv,
                                const double *rope_cos, const double *rope_sin, double eps,
-                               double *S)
+                               int decayed, double *S)
 {
     double *Sh = S + ((size_t)b * H + h) * D * D;
     double *kf = (double *)malloc(sizeof(double) * D);
@@ -447,7 +450,7 @@ static void commit_head_tokens(int b, int h, int H, int L, int D,
         for (int e = 0; e < D; ++e) {   /* V'_j - K'_j S, with the state before this token */
             double acc = 0.0;
             for (int d = 0; d < D; ++d) acc += kf[d] * Sh[(size_t)d * D + e];
-            err[e] = vf[e] - acc;
+            err[e] = vf[e] - (decayed ? alpha * acc : acc);
         }
         for (int d = 0; d < D; ++d)
             for (int e = 0; e < D; ++e)
@@ -462,7 +465,7 @@ void arl2_oracle_commit_tokens(int B, int H, int L, int D,
                                const double *alpha_logit, const double *beta_logit,
                                const double *wk, const double *wv,
                                const double *rope_cos, const double *rope_sin, double eps,
-                               int n_heads, const int *bs, const int *hs, double *S)
+                               int n_heads, const int *bs, const int *hs, int decayed, double *S)
 {
     int total = bs ? n_heads : B * H;
 #pragma omp parallel for schedule(dynamic, 1)
@@ -470,7 +473,7 @@ void arl2_oracle_commit_tokens(int B, int H, int L, int D,
         int b = bs ? bs[t] : t / H;
         int h = bs ? hs[t] : t % H;
         commit_head_tokens(b, h, H, L, D, kc, vc, alpha_logit, beta_logit, wk, wv, rope_cos,
-                           rope_sin, eps, S);
+                           rope_sin, eps, decayed, S);
     }
 }
 

@@ -214,8 +214,9 @@ def clean_pass(q, kc, vc, g, a, S, wq=None, wk=None, wv=None, rope_cos=None, rop
 
 
 def commit_tokens(kc, vc, S, alpha_logit=None, beta_logit=None, wk=None, wv=None, rope_cos=None,
-                  rope_sin=None, eps=1e-6, heads=None):
-    """Eq. 4 token by token with per-token gates [B, L, H] (None = gate 1).  Returns the new S."""
+                  rope_sin=None, eps=1e-6, heads=None, decayed_prediction=False):
+    """Eq. 4 token by token with per-token gates [B, L, H] (None = gate 1).  Returns the new S.
+    decayed_prediction: each token predicts against alpha_j S instead of S (the other reading of Eq. 4)."""
     kc, vc = _f64(kc), _f64(vc)
     wk, wv, rope_cos, rope_sin = _f64(wk), _f64(wv), _f64(rope_cos), _f64(rope_sin)
     alpha_logit, beta_logit = _f64(alpha_logit), _f64(beta_logit)
@@ -233,7 +234,7 @@ def commit_tokens(kc, vc, S, alpha_logit=None, beta_logit=None, wk=None, wv=None
         hs = np.ascontiguousarray(heads[:, 1])
     _load().arl2_oracle_commit_tokens(
         B, H, L, D, _p(kc), _p(vc), _p(alpha_logit), _p(beta_logit), _p(wk), _p(wv), _p(rope_cos),
-        _p(rope_sin), ctypes.c_double(eps), n, _p(bs), _p(hs), _p(S),
+        _p(rope_sin), ctypes.c_double(eps), n, _p(bs), _p(hs), int(bool(decayed_prediction)), _p(S),
     )
     return S
 

@@ -20,6 +20,7 @@ ARL2_FLAG_FORCE_SIMT = 1
 ARL2_FLAG_TOKEN_GATES = 2
 ARL2_FLAG_GATE_SCALAR = 4
 ARL2_FLAG_GATE_ELEMENTWISE = 8
+ARL2_FLAG_DELTA_DECAYED_PREDICTION = 32
 
 
 def ARL2_FLAG_DEBUG_WAIT_LIMIT(polls: int) -> int:

@@ -582,6 +582,7 @@ int arl2_commit_tokens(arl2_ctx* ctx, const void* d_k_clean, const void* d_v_cle
     a.kh = reinterpret_cast<float*>(ctx->ws + ctx->lay.tok_kh);
     a.gc = reinterpret_cast<float*>(ctx->ws + ctx->lay.tok_gc);
     a.nchunk = ctx->lay.nchunk;
+    a.decayed = (ctx->cfg.flags & ARL2_FLAG_DELTA_DECAYED_PREDICTION) != 0;
     a.wait_limit = ctx->wait_limit;
     if ((reinterpret_cast<uintptr_t>(d_k_clean) | reinterpret_cast<uintptr_t>(d_v_clean)) % 16 != 0) {
         set_error("commit_tokens: k_clean and v_clean must be 16-byte aligned");

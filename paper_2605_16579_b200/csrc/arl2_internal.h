@@ -97,6 +97,7 @@ struct TokenCommitArgs {
     float* kh;              // same shape
     float* gc;              // [B, H, nchunk] decay of a whole chunk
     int nchunk;             // ceil(L / 64)
+    bool decayed = false;   // each token predicts against alpha_j S_{j-1} instead of S_{j-1}
     uint32_t wait_limit = 0;   // as in StepArgs
 };
 constexpr int kTokenChunk = 64;

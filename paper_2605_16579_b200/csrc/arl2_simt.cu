@@ -483,6 +483,7 @@ __global__ void __launch_bounds__(NT) token_prepare_kernel(TokenCommitArgs a)
     const T* wk = a.wk ? static_cast<const T*>(a.wk) + (size_t)h * D * D : nullptr;
     const T* wv = a.wv ? static_cast<const T*>(a.wv) + (size_t)h * D * D : nullptr;
 
+    const int dec = a.decayed ? 1 : 0;
     load_rows<T>(Ks, LD, kc, b, h, r0, 0, D, L, L, H, D, tid);
     load_rows<T>(Vs2, LD, vc, b, h, r0, 0, D, L, L, H, D, tid);
     if (tid < kTokChunk) {
@@ -537,7 +538,8 @@ __global__ void __launch_bounds__(NT) token_prepare_kernel(TokenCommitArgs a)
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int row = ty * 4 + i, col = tx * 4 + e;
-                As[row * LA + col] = col < row ? bet[row] * expf(cl[row] - cl[col + 1]) * g[i][e] : 0.0f;
+                // g_{j-1} / g_i as printed; g_j / g_i when the prediction is made against the decayed state
+                As[row * LA + col] = col < row ? bet[row] * expf(cl[row + dec] - cl[col + 1]) * g[i][e] : 0.0f;
             }
     }
     __syncthreads();
@@ -563,7 +565,7 @@ __global__ void __launch_bounds__(NT) token_prepare_kernel(TokenCommitArgs a)
         const float* src = pass == 0 ? Ks : Vs2;
         for (int idx = tid; idx < kTokChunk * D; idx += NT) {
             const int j = idx / D, d = idx % D;
-            const float sc = pass == 0 ? bet[j] * expf(cl[j]) : bet[j];
+            const float sc = pass == 0 ? bet[j] * expf(cl[j + dec]) : bet[j];
             Ws[idx] = src[j * LD + d] * sc;
         }
         __syncthreads();

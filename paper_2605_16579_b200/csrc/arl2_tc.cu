@@ -814,6 +814,7 @@ struct TcTokenParams {
     uint32_t spin_limit;
     int ntile;                 // 128-token tiles; rows_pad = 128 * ntile
     int nchunk;                // ceil(L / 64): chunks the scan walks
+    int decayed;               // prediction against alpha_j S_{j-1}
 };
 
 __global__ void __launch_bounds__(128, 1)
@@ -894,6 +895,9 @@ tc_token_prepare_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
     __syncthreads();
     const float cl_total = cl_s[chunk * kTokC + kTokC - 1];
     const float cl_excl = cl - la;
+    // log of the factor on K'_j S_0: g_{j-1} for Eq. 4 as printed, g_j when the token's prediction is made
+    // against the state after its own forget gate
+    const float cl_pred = p.decayed ? cl : cl_excl;
 
     constexpr uint32_t kLboK = 1u << 16;
     constexpr uint32_t kLboMN = (uint32_t)(kHalfBytes >> 4) << 16;
@@ -961,7 +965,7 @@ tc_token_prepare_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
         }
         const float f = rsqrtf((ss4[0] + ss4[1]) + (ss4[2] + ss4[3]) + p.s.eps);
         store_row_bf16_swizzled(smem + kTPOffK, tid, sreg, f);
-        store_row_bf16_swizzled(smem + kTPOffKs, tid, sreg, f * be * expf(cl_excl));
+        store_row_bf16_swizzled(smem + kTPOffKs, tid, sreg, f * be * expf(cl_pred));
         store_row_bf16_global(p.kh + grow * kTile, sreg, f * expf(cl_total - cl));
         // ---- diag(beta) V'
 #pragma unroll
@@ -999,7 +1003,7 @@ tc_token_prepare_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 const int i = i4 * 4 + k;
-                const float w = be * __expf(cl_excl - cl_s[chunk * kTokC + i]);
+                const float w = be * __expf(cl_pred - cl_s[chunk * kTokC + i]);
                 v[k] = i < jj ? w * __uint_as_float(g[i]) : 0.0f;
             }
             *reinterpret_cast<float4*>(arow + i4 * 4) = make_float4(v[0], v[1], v[2], v[3]);
@@ -1493,6 +1497,7 @@ int tc_commit_tokens(const TokenCommitArgs& a, const __nv_bfloat16* wk_op, const
     p.spin_limit = a.wait_limit ? a.wait_limit - 1 : kSpinLimit;
     p.ntile = (a.s.L + kTile - 1) / kTile;
     p.nchunk = (a.s.L + kTokC - 1) / kTokC;
+    p.decayed = a.decayed ? 1 : 0;
     const size_t rows = (size_t)a.s.B * a.s.H * p.ntile * kTile;
     if (rows >= ((size_t)1 << 31)) { set_error("tc_commit_tokens: too many rows"); return ARL2_ERR_UNSUPPORTED; }
     CUtensorMap tm_k, tm_v, tm_wk, tm_wv, tm_w, tm_kh, tm_u1, tm_s;

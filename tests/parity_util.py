@@ -212,7 +212,7 @@ class Pair:
                                                              eps=self.eps),
             heads)
 
-    def commit_tokens(self, kc, vc, alpha, beta, heads=None):
+    def commit_tokens(self, kc, vc, alpha, beta, heads=None, decayed_prediction=False):
         """Token-sequential commit with per-token gates on both sides; worst per-head error of S."""
         d = self.dev
         dv = lambda t: None if t is None else t.to(d)  # noqa: E731
@@ -220,7 +220,7 @@ class Pair:
         return self._after_commit(
             lambda vw, S, u: self.oracle.commit_tokens(vw(kc), vw(vc), S, vw(alpha), vw(beta),
                                                        self._wu(self.wk, u), self._wu(self.wv, u), self.cos,
-                                                       self.sin, eps=self.eps),
+                                                       self.sin, eps=self.eps, decayed_prediction=decayed_prediction),
             heads)
 
     def clean_pass(self, q, kc, vc, g, a, rows=None):

@@ -82,3 +82,22 @@ def test_token_commit_full_size_sampled_heads(oracle):
         alpha, beta = workload.token_gate_logits(cfg, blk)
         err = pair.commit_tokens(kc, vc, alpha, beta, heads=heads)
         assert err <= pair.tol, f"block {blk}: error {err:.3e}"
+
+
+@pytest.mark.parametrize("dtype,D,B,H,L", [("fp32", 64, 1, 2, 200), ("bf16", 128, 2, 3, 333), ("bf16", 128, 1, 2, 1100)])
+def test_token_commit_with_the_prediction_against_the_decayed_state(oracle, dtype, D, B, H, L):
+    """The other reading of Eq. 4 (each token predicts against alpha_j S_{j-1}), chosen by a context flag."""
+    from paper_2605_16579_b200 import arl2
+
+    cfg = workload.custom(B=B, H=H, D=D, L=L, dtype=dtype, cfg_id=46)
+    pair = Pair(oracle, cfg, flags=FLAG | arl2.ARL2_FLAG_DELTA_DECAYED_PREDICTION)
+    plain = Pair(oracle, cfg, flags=FLAG)
+    for blk in range(3):
+        kc, vc, _ = workload.commit_inputs(cfg, blk)
+        alpha, beta = workload.token_gate_logits(cfg, blk, alpha_mean=3.0)
+        err = pair.commit_tokens(kc, vc, alpha, beta, decayed_prediction=True)
+        assert err <= pair.tol, f"block {blk}: error {err:.3e} > {pair.tol}"
+        assert plain.commit_tokens(kc, vc, alpha, beta) <= plain.tol
+    # the two readings do differ on these inputs
+    a, b = pair.layer.get_state().numpy(), plain.layer.get_state().numpy()
+    assert np.abs(a - b).max() > 1e-3 * np.abs(b).max()

@@ -29,7 +29,10 @@ MUTANTS = [
     ("token-sequential rule without its decay", "Sh[t] *= alpha;", "Sh[t] *= 1.0;"),
     ("frame-level delta rule writes into the running state",
      "double *dst = (rule == 1) ? dS : Sh;", "double *dst = Sh;"),
-    ("per-token rule predicts from the decayed state", "err[e] = vf[e] - acc;", "err[e] = vf[e] - alpha * acc;"),
+    ("per-token rule predicts from the decayed state when asked for the printed form",
+     "err[e] = vf[e] - (decayed ? alpha * acc : acc);", "err[e] = vf[e] - alpha * acc;"),
+    ("per-token rule ignores the request for the decayed prediction",
+     "err[e] = vf[e] - (decayed ? alpha * acc : acc);", "err[e] = vf[e] - acc;"),
     ("per-token rule forgets the learning rate",
      "alpha * Sh[(size_t)d * D + e] + beta * kf[d] * err[e];", "alpha * Sh[(size_t)d * D + e] + kf[d] * err[e];"),
     ("per-token decay applied to the new term", "alpha * Sh[(size_t)d * D + e] + kf[d] * vf[e];",

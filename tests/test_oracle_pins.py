@@ -413,16 +413,18 @@ def test_cache_attention_against_library_and_the_layer(oracle):
     np.testing.assert_allclose(big, np.einsum("bhlj,bjhe->blhe", w, v2), rtol=1e-10, atol=1e-10)
 
 
-def test_token_gates_matrix_product_form(oracle):
+@pytest.mark.parametrize("decayed", [False, True])
+def test_token_gates_matrix_product_form(oracle, decayed):
     """Per-token Eq. 4 rewritten as S_j = (alpha_j I - beta_j k_j^T k_j) S_{j-1} + beta_j k_j^T v_j
     and evaluated with explicit D x D transition matrices (library matmul), with feature maps,
-    rotation and normalisation taken from the library-pinned feature routine."""
+    rotation and normalisation taken from the library-pinned feature routine.  The other reading
+    (prediction against the decayed state) has the transition alpha_j (I - beta_j k_j^T k_j)."""
     B, L, H, D = 2, 9, 2, 8
     k, v, S0 = rnd(B, L, H, D), rnd(B, L, H, D), rnd(B, H, D, D)
     al, bl = rnd(B, L, H) + 1.0, rnd(B, L, H)
     wk, wv = np.eye(D) + 0.1 * rnd(H, D, D), np.eye(D) + 0.1 * rnd(H, D, D)
     cos, sin = tables(L, D)
-    got = oracle.commit_tokens(k, v, S0, al, bl, wk, wv, cos, sin, eps=1e-6)
+    got = oracle.commit_tokens(k, v, S0, al, bl, wk, wv, cos, sin, eps=1e-6, decayed_prediction=decayed)
     kf = oracle.feature(k, wk, cos, sin, 1e-6, 0)
     vf = oracle.feature(v, wv, None, None, 1e-6, 1)
     ref = S0.copy()
@@ -432,7 +434,11 @@ def test_token_gates_matrix_product_form(oracle):
             for j in range(L):
                 kk = torch.from_numpy(kf[b, j, h])[None, :]          # 1 x D
                 vv = torch.from_numpy(vf[b, j, h])[None, :]
-                M = sig(al[b, j, h]) * torch.eye(D, dtype=torch.float64) - sig(bl[b, j, h]) * (kk.T @ kk)
+                eye = torch.eye(D, dtype=torch.float64)
+                if decayed:
+                    M = sig(al[b, j, h]) * (eye - sig(bl[b, j, h]) * (kk.T @ kk))
+                else:
+                    M = sig(al[b, j, h]) * eye - sig(bl[b, j, h]) * (kk.T @ kk)
                 S = M @ S + sig(bl[b, j, h]) * (kk.T @ vv)
             ref[b, h] = S.numpy()
     np.testing.assert_allclose(got, ref, rtol=1e-11, atol=1e-13)
