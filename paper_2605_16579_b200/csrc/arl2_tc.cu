@@ -76,45 +76,6 @@ struct TcStepParams {
     int n_items;               // + ceil(B * H / 2) items of ragged last tiles when n_q is odd
 };
 
-// 2^x for two values on the FMA pipe instead of the special-function unit: x = j + f with
-// j = round(x) and f in [-0.5, 0.5]; 2^f by a cubic fitted on that interval (relative error below
-// 1e-4, far under the bf16 rounding of the probabilities); 2^j by adding j to the exponent field
-// with one integer multiply-add.  x is clamped at -126 (the result is then a denormal-sized
-// 2^-126 instead of 0: it is rounded to bf16 and summed like any other term).
-#ifndef ARL2_POLY_COUNT
-#define ARL2_POLY_COUNT 0
-#endif
-#ifndef ARL2_POLY_PERIOD
-#define ARL2_POLY_PERIOD 2
-#endif
-#ifdef ARL2_NO_TOKEN
-constexpr bool kUseToken = false;
-#else
-constexpr bool kUseToken = true;
-#endif
-constexpr int kPolyCount = ARL2_POLY_COUNT;    // of every kPolyPeriod element pairs, this many take the
-constexpr int kPolyPeriod = ARL2_POLY_PERIOD;  // FMA-pipe exponential, the rest the special-function unit
-__device__ __forceinline__ void exp2_fma2(float x0, float x1, float& r0, float& r1)
-{
-    const float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
-    x0 = fmaxf(x0, -126.0f);
-    x1 = fmaxf(x1, -126.0f);
-    const uint64_t x2 = pack2(x0, x1);
-    const uint64_t t2 = add2(x2, pack2(kMagic, kMagic));
-    const uint64_t j2 = add2(t2, pack2(-kMagic, -kMagic));
-    const uint64_t f2 = fma2(j2, pack2(-1.0f, -1.0f), x2);
-    uint64_t p2 = fma2(pack2(0.05517132207751274f, 0.05517132207751274f), f2,
-                       pack2(0.24261054396629333f, 0.24261054396629333f));
-    p2 = fma2(p2, f2, pack2(0.6932609677314758f, 0.6932609677314758f));
-    p2 = fma2(p2, f2, pack2(0.9999281167984009f, 0.9999281167984009f));
-    float t0, t1, q0, q1;
-    unpack2(t2, t0, t1);
-    unpack2(p2, q0, q1);
-    // (bits of t) << 23 == j << 23 modulo 2^32: the magic constant's bits fall off the top
-    r0 = __int_as_float(__float_as_int(q0) + __float_as_int(t0) * 0x800000);
-    r1 = __int_as_float(__float_as_int(q1) + __float_as_int(t1) * 0x800000);
-}
-
 // A work item drives up to two 128-row query tiles.  A "pair" item holds two consecutive tiles of
 // one (stream, head): they share every K/V tile.  A "ragged" item holds the last, partial tiles
 // of two different (stream, head) units (or of one, when the number of units is odd): each tile
@@ -308,7 +269,7 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                     }
                 }
                 const uint64_t neg_m2 = pack2(-m_ref, -m_ref);
-                if (kUseToken && it.ntile == 2) {
+                if (it.ntile == 2) {
                     // the two groups alternate in the exponential phase, so that one group's
                     // exponentials overlap the other tile's MMAs instead of its exponentials
                     const uint32_t par = (t == 0) ? ((tok_cnt + 1) & 1) : (tok_cnt & 1);
@@ -320,16 +281,12 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                     float x0, x1, p0, p1;
                     unpack2(fma2(pack2(__uint_as_float(sreg[2 * c]), __uint_as_float(sreg[2 * c + 1])), c2x2, neg_m2),
                             x0, x1);
-                    if ((c % kPolyPeriod) < kPolyCount) {
-                        exp2_fma2(x0, x1, p0, p1);            // FMA pipe
-                    } else {
-                        p0 = ex2_approx(x0);                  // special-function unit
-                        p1 = ex2_approx(x1);
-                    }
+                    p0 = ex2_approx(x0);
+                    p1 = ex2_approx(x1);
                     l2 = add2(l2, pack2(p0, p1));
                     sreg[c] = pack_bf16(p0, p1);
                 }
-                if (kUseToken && it.ntile == 2) mbar_arrive(bars + 8 * (kBarTok0 + (t ^ 1)));
+                if (it.ntile == 2) mbar_arrive(bars + 8 * (kBarTok0 + (t ^ 1)));
                 tmem_st32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sreg[0]));
                 tmem_st32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[32]));
                 tmem_wait_st();
