@@ -89,8 +89,11 @@ typedef struct {
  * holds a status word, the rotated copy of K made once per step, two tensor-core operand
  * copies of S (a commit writes the one that is not current) and one of each feature map, the
  * packed rotation table, the partial sums of the commit reduction (two sets: the delta rule
- * has two accumulators), the per-token decay weights and, with ARL2_FLAG_TOKEN_GATES, the chunk
- * factors of arl2_commit_tokens.  Returns 0 for an invalid configuration.
+ * has two accumulators), the per-token decay weights, with bf16 I/O and D = 128 the partial rows
+ * of attention work items cut into key ranges (about 39 MB: when the last wave of a step launch
+ * would leave more than half of the SMs idle, its items are computed as 2 to 4 parts and a second
+ * small launch merges them) and, with ARL2_FLAG_TOKEN_GATES, the chunk factors of
+ * arl2_commit_tokens.  Returns 0 for an invalid configuration.
  */
 size_t arl2_workspace_bytes(const arl2_config* cfg);
 

@@ -27,7 +27,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, k_rot, partials, partials_g, state_bf16, state_bf16_b, wq_op, wk_op, wv_op, rope_h, dec_w, dec_total, tok_w, tok_u1, tok_kh, tok_gc, total;
+    size_t status, split_ml, split_o, k_rot, partials, partials_g, state_bf16, state_bf16_b, wq_op, wk_op, wv_op, rope_h, dec_w, dec_total, tok_w, tok_u1, tok_kh, tok_gc, total;
     int nsplit, nchunk, nslot;
 };
 
@@ -81,6 +81,13 @@ Layout make_layout(const arl2_config& c)
     l.nsplit = (c.L + kCommitChunk - 1) / kCommitChunk;
     size_t off = 0;
     l.status = off;     off += align_up(kStatusWords * sizeof(uint32_t));
+    // key-range split of the step kernel's last wave (tensor-core path): the parts' row statistics
+    // and unnormalised rows
+    l.split_ml = l.split_o = off;
+    if (tc_supported(c)) {
+        l.split_ml = off;      off += align_up((size_t)kSplitTileParts * 128 * 2 * sizeof(float));
+        l.split_o = off;       off += align_up((size_t)kSplitTileParts * 128 * 128 * sizeof(float));
+    }
     l.k_rot = off;      off += align_up(tensor);
     // partial-sum slots per (stream, head): the plain-FMA kernels use one per 512-token chunk; the
     // tensor-core kernel one per run of tiles a head falls into, runs sized for a 148-SM device
@@ -300,6 +307,15 @@ bool check_step_args(const char* who, const void* d_q, const void* d_k, const vo
 }
 
 // The fused attention kernel of one pass; k_rot is K after RoPE (or K itself without a rotation).
+// The buffers the step kernel needs to cut the items of its last wave into key ranges.
+void attach_split(const arl2_ctx* ctx, StepArgs& a)
+{
+    if (!ctx->use_tc) return;
+    a.split_o = reinterpret_cast<float*>(ctx->ws + ctx->lay.split_o);
+    a.split_ml = reinterpret_cast<float*>(ctx->ws + ctx->lay.split_ml);
+    a.split_tile_parts = kSplitTileParts;
+}
+
 int launch_step(arl2_ctx* ctx, const void* d_q, const void* k_rot, const void* d_v,
                 const float* d_gate_logits, void* d_out, cudaStream_t st)
 {
@@ -314,6 +330,7 @@ int launch_step(arl2_ctx* ctx, const void* d_q, const void* k_rot, const void* d
     a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lay.status);
     a.launch_parity = (int)(ctx->step_calls & 1u);
     a.rope_h = (ctx->use_tc && ctx->rope_cos != nullptr) ? ctx->ws + ctx->lay.rope_h : nullptr;
+    attach_split(ctx, a);
     cudaEvent_t e0 = ctx->ev_before, e1 = ctx->ev_after;
     ctx->ev_before = ctx->ev_after = nullptr;
     if (e0 != nullptr) cudaEventRecord(e0, st);
@@ -431,6 +448,7 @@ int arl2_teacher_step(arl2_ctx* ctx, const void* d_q, const void* d_k_cache, con
     a.launch_parity = (int)(ctx->step_calls & 1u);
     a.rope_h = nullptr;                    // the caller's Q and cache are already rotated
     a.Lk = cache_tokens;
+    attach_split(ctx, a);
     cudaStream_t st = as_stream(stream);
     cudaEvent_t e0 = ctx->ev_before, e1 = ctx->ev_after;
     ctx->ev_before = ctx->ev_after = nullptr;

@@ -19,6 +19,10 @@ enum StatusWord : int {
 };
 
 constexpr int kCommitChunk = 512;  // tokens per partial sum of the commit reduction
+// Key-range split of the step kernel's last wave: at most kMaxSplit parts per item, and room for
+// the partial rows of 2 x 148 parts of two query tiles each (more SMs: the launcher splits less)
+constexpr int kMaxSplit = 4;
+constexpr int kSplitTileParts = 4 * 148;
 
 struct Shape {
     int B, H, L, D;
@@ -44,6 +48,10 @@ struct StepArgs {
     int Lk = 0;             // > 0: K and V hold Lk tokens (a cache), [B, Lk, H, D]; 0: L
     int gate_mode = 0;      // 0: gate [B, L, H]; 1: [B, L]; 2: [B, L, H, D]
     uint32_t wait_limit = 0;  // 0: default; n > 0: bounded waits give up after n - 1 polls (test hook)
+    // key-range split of the last wave of work items (tensor-core path), or nullptr: never split
+    float* split_o = nullptr;            // [split_tile_parts][128][128] fp32
+    float* split_ml = nullptr;           // [split_tile_parts][128][2] fp32
+    int split_tile_parts = 0;
 };
 
 struct CommitArgs {

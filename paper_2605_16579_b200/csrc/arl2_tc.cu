@@ -74,6 +74,15 @@ struct TcStepParams {
     int n_kv;                  // key tiles per head
     int n_pair_items;          // B * H * (n_q / 2): items with two query tiles
     int n_items;               // + ceil(B * H / 2) items of ragged last tiles when n_q is odd
+    // Key-range split of the last wave: items [0, n_whole) run whole; item n_whole + s (s = "slot")
+    // runs as k_split parts over consecutive ranges of key tiles, scheduled as ids n_whole +
+    // s * k_split + part.  Every part leaves its unnormalised rows, reference maxima and row sums in
+    // the split buffers; tc_split_merge_kernel then combines the parts of a row in index order.
+    int n_whole;
+    int k_split;               // 1: nothing is split
+    int n_sched;               // ids the scheduler hands out: n_whole + (n_items - n_whole) * k_split
+    float* split_o;            // [slot][tile][part][128 rows][128] unnormalised output rows
+    float* split_ml;           // [slot][tile][part][128 rows][2] reference maximum (log2 units), row sum
 };
 
 // A work item drives up to two 128-row query tiles.  A "pair" item holds two consecutive tiles of
@@ -84,13 +93,29 @@ struct Item {
     int b[2], h[2], row0[2];
     int ntile;    // active tiles: 1 or 2
     bool shared;  // both tiles read the same K, V, W_phi_q and state
+    int j0, nj;   // key tiles [j0, j0 + nj) of the head
+    int part;     // -1: the whole key range; else index of this part
+    int slot;     // split items only: index among the split items
 };
 
 // Items [0, n_pair_items) are pairs of full tiles, (b, h)-major so that neighbours share K and V
 // in L2; the rest pack the ragged last tiles two by two.
+template <bool kSplit>
 __device__ __forceinline__ Item decode_item(int id, const TcStepParams& p)
 {
     Item it;
+    it.j0 = 0;
+    it.nj = p.n_kv;
+    it.part = -1;
+    it.slot = 0;
+    if (kSplit && id >= p.n_whole) {
+        const int x = id - p.n_whole;
+        it.slot = x / p.k_split;
+        it.part = x - it.slot * p.k_split;
+        id = p.n_whole + it.slot;
+        it.j0 = (it.part * p.n_kv) / p.k_split;
+        it.nj = ((it.part + 1) * p.n_kv) / p.k_split - it.j0;
+    }
     const int full_pairs = p.n_q >> 1;
     const int units = p.s.B * p.s.H;
     if (id < p.n_pair_items) {
@@ -160,7 +185,7 @@ __device__ __forceinline__ Entry item_entry(const Item& it, int n_kv, int e)
 
 // One softmax group thread: owns query row `r` of tile `t` of every item.  kElemGate compiles the
 // per-channel gate variant in (a separate kernel instantiation, so the default path is unchanged).
-template <bool kElemGate>
+template <bool kElemGate, bool kSplit>
 __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* smem, uint32_t bars,
                                              uint32_t tmem_base, const Abort& ab,
                                              const volatile int* item_slots, int t, int r,
@@ -184,7 +209,8 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
         if (!wait_bar(bars + 8 * kBarQFull, item & 1, ab, 10)) return;
         const int id = item_slots[item & 1];
         if (id < 0) return;
-        const Item it = decode_item(id, p);
+        const Item it = decode_item<kSplit>(id, p);
+        const int j0 = kSplit ? it.j0 : 0, nj = kSplit ? it.nj : n_kv;
         const int b = it.b[t], h = it.h[t];
         const int row = it.row0[t] + r;
         const bool valid_row = row < L;
@@ -222,7 +248,8 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
             float m_ref = -INFINITY;   // reference maximum (scaled, base 2) of the probabilities
             uint64_t l2 = pack2(0.0f, 0.0f);   // running row sum relative to m_ref, two lanes
 
-            for (int j = 0; j < n_kv; ++j) {
+            for (int jj = 0; jj < nj; ++jj) {
+                const int j = j0 + jj;
                 if (!wait_bar(bar_s, s_cnt & 1, ab, 20 + t)) return;
                 ++s_cnt;
                 tc_fence_after();
@@ -254,7 +281,7 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
                         m_ref = m_new;
                         l2 = fma2(l2, pack2(alpha, alpha), pack2(0.0f, 0.0f));
                     }
-                    if (j > 0) {
+                    if (jj > 0) {
                         // the MMA that last accumulated into O_t finished before S_t(j) was
                         // signalled, and the next one waits for this group's arrival below
 #pragma unroll 1
@@ -407,8 +434,34 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
             if (!wait_bar(bars + 8 * (kBarOFinal0 + t), of_cnt & 1, ab, 40 + t)) return;
             ++of_cnt;
             tc_fence_after();
-            const float inv_l = 1.0f / l_sum;
             __nv_bfloat16* orow = p.out + (((size_t)b * L + (valid_row ? row : 0)) * H + h) * kTile;
+            if (kSplit && it.part >= 0) {
+                // ---- one part of a split item: its rows of O_t, unnormalised (the readout in them
+                // is scaled by this part's row sum, so that the merged sum carries gate * Q' S times
+                // the total row sum), the reference maximum and the row sum go to the split buffers;
+                // tc_split_merge_kernel combines the parts
+                const size_t tp = ((size_t)it.slot * 2 + t) * p.k_split + it.part;
+                float* mine = p.split_o + (tp * kTile + r) * kTile;
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(o_addr + c * 32, o);
+                    tmem_wait_ld();
+                    if (valid_row) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(
+                                             mine + c * 32 + e * 8),
+                                         "r"(o[e * 8]), "r"(o[e * 8 + 1]), "r"(o[e * 8 + 2]), "r"(o[e * 8 + 3]),
+                                         "r"(o[e * 8 + 4]), "r"(o[e * 8 + 5]), "r"(o[e * 8 + 6]), "r"(o[e * 8 + 7])
+                                         : "memory");
+                    }
+                }
+                tc_fence_before();
+                if (valid_row) *reinterpret_cast<float2*>(p.split_ml + (tp * kTile + r) * 2) = make_float2(m_ref, l_sum);
+                continue;
+            }
+            const float inv_l = 1.0f / l_sum;
 #pragma unroll 1
             for (int c = 0; c < 4; ++c) {
                 uint32_t o[32];
@@ -435,7 +488,7 @@ __device__ __forceinline__ void softmax_role(const TcStepParams& p, uint8_t* sme
     }
 }
 
-template <bool kElemGate>
+template <bool kElemGate, bool kSplit>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_w,
@@ -489,7 +542,7 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
     if (warp < 8) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
-        softmax_role<kElemGate>(p, smem, bars, tmem_base, ab, item_slots, warp >> 2, (warp & 3) * 32 + lane, warp & 3);
+        softmax_role<kElemGate, kSplit>(p, smem, bars, tmem_base, ab, item_slots, warp >> 2, (warp & 3) * 32 + lane, warp & 3);
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
     }
@@ -509,13 +562,14 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             for (uint32_t item = 0; ok; ++item) {
                 if (item > 0) ok = wait_bar(bars + 8 * kBarQFree, (item - 1) & 1, ab, 50);
                 if (!ok) break;
-                if (id >= p.n_items) {
+                if (id >= p.n_sched) {
                     item_slots[item & 1] = -1;
                     mbar_arrive(bar_q);
                     break;
                 }
                 item_slots[item & 1] = id;
-                const Item it = decode_item(id, p);
+                const Item it = decode_item<kSplit>(id, p);
+                const int j0 = kSplit ? it.j0 : 0, nj = kSplit ? it.nj : n_kv;
                 const int ntile = it.ntile;
                 mbar_expect_tx(bar_q, ntile * kTileBytes);
                 q_item = (int)item;
@@ -524,7 +578,7 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     tma_load_4d(dst, &tm_q, bar_q, 0, it.h[t], it.row0[t], it.b[t]);
                     tma_load_4d(dst + kHalfBytes, &tm_q, bar_q, 64, it.h[t], it.row0[t], it.b[t]);
                 }
-                const int entries = item_entries(it, n_kv);
+                const int entries = item_entries(it, nj);
                 for (int e = 0; e < entries && ok; ++e, ++n) {
                     const uint32_t slot = n % kStages;
                     if (n >= (uint32_t)kStages)
@@ -533,12 +587,12 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     const uint32_t bar = bars + 8 * (kBarFull0 + slot);
                     const uint32_t dst = smem_base + kOffRing + slot * kTileBytes;
                     mbar_expect_tx(bar, kTileBytes);
-                    const Entry en = item_entry(it, n_kv, e);
+                    const Entry en = item_entry(it, nj, e);
                     const int tb = it.b[en.tile], th = it.h[en.tile];
                     if (en.kind == kEntK || en.kind == kEntV) {
                         const CUtensorMap* tm = en.kind == kEntV ? &tm_v : &tm_k;
-                        tma_load_4d(dst, tm, bar, 0, th, en.j * kTile, tb);
-                        tma_load_4d(dst + kHalfBytes, tm, bar, 64, th, en.j * kTile, tb);
+                        tma_load_4d(dst, tm, bar, 0, th, (j0 + en.j) * kTile, tb);
+                        tma_load_4d(dst + kHalfBytes, tm, bar, 64, th, (j0 + en.j) * kTile, tb);
                     } else if (en.kind == kEntW) {
                         tma_load_2d(dst, &tm_w, bar, 0, th * kTile);
                         tma_load_2d(dst + kHalfBytes, &tm_w, bar, 64, th * kTile);
@@ -619,7 +673,8 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (!ok) break;
                 const int id = item_slots[item & 1];
                 if (id < 0) break;
-                const Item it = decode_item(id, p);
+                const Item it = decode_item<kSplit>(id, p);
+                const int nj = kSplit ? it.nj : n_kv;   // key tiles of this item (a part walks its own range)
                 const int ntile = it.ntile;
                 const bool active = t < ntile;
                 const bool shared = it.shared;
@@ -646,12 +701,12 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     issue_qk(q_tile, slot_addr(e_k));
                     mma_commit(bar_s);
                     release_mine(e_k, !shared);
-                    if (n_kv == 1) q_free();
+                    if (nj == 1) q_free();
                 }
                 cons += shared ? 1 : ntile;
 
-                for (int j = 0; j < n_kv && ok; ++j) {
-                    const bool last = j + 1 == n_kv;     // then the next "S" is the inter branch's Q W
+                for (int j = 0; j < nj && ok; ++j) {
+                    const bool last = j + 1 == nj;       // then the next "S" is the inter branch's Q W
                     const int per_tile = last ? 3 : 2;   // ragged item: V, K or W, [Qraw] per tile
                     const int group = shared ? (last ? 2 + ntile : 2) : per_tile * ntile;
                     if (active) {
@@ -672,7 +727,7 @@ tc_step_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                         release_mine(e_v, !shared);
                         release_mine(e_b, !shared);
                         if (last) release_mine(e_q, true);
-                        if (j + 2 == n_kv) q_free();   // S_t(n_kv - 1) was the last use of Q~
+                        if (j + 2 == nj) q_free();   // the last score MMA was the last use of Q~
                     }
                     cons += group;
                 }
@@ -1338,14 +1393,63 @@ __global__ void transpose_map_kernel(const __nv_bfloat16* __restrict__ w, __nv_b
     out[t] = v;
 }
 
+// Combines the parts of the split items of a step launch: one warp per query row, a lane owns four
+// output channels.  With part q's reference maximum m_q, row sum l_q and unnormalised row O_q:
+//   out = sum_q 2^(m_q - m) O_q / sum_q 2^(m_q - m) l_q,   m = max_q m_q,   summed in part order.
+__global__ void __launch_bounds__(256)
+tc_split_merge_kernel(const TcStepParams p)
+{
+    const int warp = (int)((blockIdx.x * 256u + threadIdx.x) >> 5), lane = threadIdx.x & 31;
+    const int r = warp & (kTile - 1), t = (warp >> 7) & 1, slot = warp >> 8;
+    const bool in_range = slot < p.n_items - p.n_whole;
+    Item it;
+    if (in_range) it = decode_item<false>(p.n_whole + slot, p);
+    const int k = p.k_split;
+    const size_t tp0 = ((size_t)slot * 2 + t) * k;
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // the step kernel has finished, its writes are visible
+    if (!in_range || t >= it.ntile || p.status[kStatusError] != 0u) return;
+    const int row = it.row0[t] + r;
+    if (row >= p.s.L) return;
+    float w[kMaxSplit], l[kMaxSplit];
+    float4 x[kMaxSplit];
+    float m_all = -INFINITY;
+#pragma unroll
+    for (int q = 0; q < kMaxSplit; ++q) {
+        if (q < k) {   // all loads go out before the first use
+            const float2 ml = *reinterpret_cast<const float2*>(p.split_ml + ((tp0 + q) * kTile + r) * 2);
+            x[q] = *reinterpret_cast<const float4*>(p.split_o + ((tp0 + q) * kTile + r) * kTile + lane * 4);
+            w[q] = ml.x;
+            l[q] = ml.y;
+            m_all = fmaxf(m_all, ml.x);
+        }
+    }
+    float l_all = 0.0f;
+    float4 acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+#pragma unroll
+    for (int q = 0; q < kMaxSplit; ++q) {
+        if (q < k) {
+            const float wq = ex2_approx(w[q] - m_all);
+            l_all = fmaf(wq, l[q], l_all);
+            acc.x = fmaf(wq, x[q].x, acc.x);
+            acc.y = fmaf(wq, x[q].y, acc.y);
+            acc.z = fmaf(wq, x[q].z, acc.z);
+            acc.w = fmaf(wq, x[q].w, acc.w);
+        }
+    }
+    const float inv = 1.0f / l_all;
+    __nv_bfloat16* orow = p.out + (((size_t)it.b[t] * p.s.L + row) * p.s.H + it.h[t]) * kTile;
+    *reinterpret_cast<uint2*>(orow + lane * 4) = make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+}
+
 std::mutex g_setup_mutex;
 DeviceSetup g_setup[kMaxDevices];
 
 int device_setup(int* num_sms)
 {
     return device_setup_once(g_setup_mutex, g_setup, [] {
-        cudaError_t e = opt_in_smem(tc_step_kernel<false>, kSmemBytes);
-        if (e == cudaSuccess) e = opt_in_smem(tc_step_kernel<true>, kSmemBytes);
+        cudaError_t e = opt_in_smem(tc_step_kernel<false, false>, kSmemBytes);
+        if (e == cudaSuccess) e = opt_in_smem(tc_step_kernel<true, false>, kSmemBytes);
+        if (e == cudaSuccess) e = opt_in_smem(tc_step_kernel<false, true>, kSmemBytes);
         if (e == cudaSuccess) e = opt_in_smem(tc_token_prepare_kernel, kTPSmemBytes);
         if (e == cudaSuccess) e = opt_in_smem(tc_token_scan_kernel, kTSSmemBytes);
         return e;
@@ -1420,14 +1524,56 @@ int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* 
     // two item counters alternate between launches: a launch consumes one and clears the other
     p.sched_counter = a.status + kStatusSched + (a.launch_parity & 1);
     p.sched_next = a.status + kStatusSched + ((a.launch_parity + 1) & 1);
-    const int grid = p.n_items < num_sms ? p.n_items : num_sms;
-    if (p.gate_mode == 2 && p.gate != nullptr)
-        tc_step_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(tm_q, tm_k, tm_v, tm_w, tm_s, p);
+    const bool elem_gate = p.gate_mode == 2 && p.gate != nullptr;
+    // The last wave: `rem` items on num_sms SMs.  Cut into k key ranges, the wave takes
+    // ceil(rem k / SMs) rounds of one part each; a part costs its share of the key iterations plus
+    // what every item costs (the readout iteration, the hand-over between items) plus the exchange
+    // of the partial rows -- measured: 3.7 k clk per iteration, 10.8 k per item, about 6 k for the
+    // exchange.  Take the k that makes the wave shortest, if that is shorter than leaving it whole.
+    p.n_whole = p.n_items;
+    p.k_split = 1;
+    if (!elem_gate && a.split_o != nullptr) {
+        const int waves = (p.n_items + num_sms - 1) / num_sms;
+        const int rem = p.n_items - (waves - 1) * num_sms;
+        const float iter = 3.74f, fixed = 10.8f, exchange = 6.0f;
+        float best = (p.n_kv + 1) * iter + fixed;
+        for (int k = 2; k <= kMaxSplit; ++k) {
+            if (p.n_kv < 4 * k || (long)rem * k * 2 > a.split_tile_parts) break;
+            const float part = ((float)p.n_kv / k + 1.0f) * iter + fixed + exchange;
+            const float cost = (float)((rem * k + num_sms - 1) / num_sms) * part;
+            if (cost < 0.95f * best) { best = cost; p.k_split = k; }
+        }
+        if (p.k_split > 1) p.n_whole = p.n_items - rem;
+    }
+    p.n_sched = p.n_whole + (p.n_items - p.n_whole) * p.k_split;
+    p.split_o = a.split_o;
+    p.split_ml = a.split_ml;
+    const int grid = p.n_sched < num_sms ? p.n_sched : num_sms;
+    if (elem_gate)
+        tc_step_kernel<true, false><<<grid, kThreads, kSmemBytes, st>>>(tm_q, tm_k, tm_v, tm_w, tm_s, p);
+    else if (p.k_split > 1)
+        tc_step_kernel<false, true><<<grid, kThreads, kSmemBytes, st>>>(tm_q, tm_k, tm_v, tm_w, tm_s, p);
     else
-        tc_step_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(tm_q, tm_k, tm_v, tm_w, tm_s, p);
+        tc_step_kernel<false, false><<<grid, kThreads, kSmemBytes, st>>>(tm_q, tm_k, tm_v, tm_w, tm_s, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_error("launch of tc_step_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
-    return 1;
+    if (p.k_split == 1) return 1;
+    // the parts' rows are combined by a second, small kernel (one warp per row); it may start
+    // before the step kernel ends and waits for it at its griddepcontrol.wait
+    const long rows = (long)(p.n_items - p.n_whole) * 2 * kTile;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((rows + 7) / 8));
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, tc_split_merge_kernel, p);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) { set_error("launch of tc_split_merge_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
+    return 2;
 }
 
 // Eq. 4 token by token with per-token gates on the tensor-core path (bf16 I/O, D = 128).  The

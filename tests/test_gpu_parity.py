@@ -244,3 +244,24 @@ def test_odd_unit_counts_bf16(oracle, B, H, L):
     cfg = workload.custom(B=B, H=H, D=128, L=L, dtype="bf16", cfg_id=23)
     pair = Pair(oracle, cfg)
     run_schedule(pair, 2, 2, closed_gate_blocks=(1,))
+
+
+@pytest.mark.parametrize("B,H,L", [(1, 3, 1100), (1, 2, 1700), (2, 2, 2100), (1, 1, 2048)])
+def test_key_range_split_bf16(oracle, B, H, L):
+    """With fewer work items in its last wave than half the SMs, the tensor-core step kernel cuts
+    those items into 2 to 4 ranges of key tiles and merges the parts' rows: every element against
+    the oracle (pair items and ragged items, 9 to 17 key tiles), and the same call twice must give
+    the same bits (the merge runs in part order whoever finishes last)."""
+    cfg = workload.custom(B=B, H=H, D=128, L=L, dtype="bf16", cfg_id=29)
+    pair = Pair(oracle, cfg)
+    run_schedule(pair, 2, 2, closed_gate_blocks=(1,))
+    d = pair.dev
+    q, k, v, g = (t.to(d) for t in workload.step_inputs(cfg, 1, 0))
+    outs = []
+    for _ in range(3):
+        out = torch.full((cfg.B, cfg.L, cfg.H, cfg.D), float("nan"), dtype=cfg.torch_dtype, device=d)
+        pair.layer.denoise_step(q, k, v, g, out=out)
+        outs.append(out)
+    pair.layer.sync_status()
+    assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16))
+    assert torch.equal(outs[0].view(torch.int16), outs[2].view(torch.int16))
