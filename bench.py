@@ -462,6 +462,21 @@ def run_traffic_probe(args):
     for i in range(4):
         layer.denoise_step(*sets[i % RING], out=out)
     layer.commit(kc, vc, a)
+    if args.probe_all and cfg.dtype == "bf16" and cfg.D == 128:
+        # one call of every other entry point, so that one small command shows every kernel
+        q, k, v, g = sets[0]
+        layer.clean_pass(q, kc, vc, g, a, out=out)
+        layer.commit_delta(kc, vc, a, workload.beta_logits(cfg, 0).to(dev))
+        alpha, _ = (t.to(dev) for t in workload.token_gate_logits(cfg, 0))
+        layer.commit_decay_tokens(kc, vc, alpha)
+        layer.denoise_step_token_level(q, k, v, g, alpha, out=out)
+        d = cfg.H * cfg.D
+        gen = torch.Generator(device="cpu").manual_seed(4242)
+        rnd = lambda *s: (torch.randn(*s, generator=gen) * d ** -0.5).to(torch.bfloat16).to(dev)  # noqa: E731
+        layer.set_projections(rnd(d, d), rnd(d, d), rnd(d, d), rnd(d, cfg.H), rnd(d, d))
+        x = torch.randn(cfg.B, cfg.L, d, generator=gen).to(torch.bfloat16).to(dev)
+        pq, pk_, pv, pg = layer.project_in(x)
+        layer.project_out(pq)
     layer.sync_status()
     print(json.dumps({"traffic_probe": workload_text(cfg), "launches": layer.launch_count}))
 
@@ -823,6 +838,8 @@ def main():
     ap.add_argument("--no-stack", action="store_true", help="skip the 30-layer module stack leg")
     ap.add_argument("--traffic-probe", action="store_true",
                     help="set up, run four denoise passes and a commit, exit (for a one-launch profiler capture)")
+    ap.add_argument("--probe-all", action="store_true",
+                    help="with --traffic-probe: also call every other entry point once (bf16, D = 128)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

@@ -873,30 +873,34 @@ int launch_commit(const CommitArgs& a, cudaStream_t st)
 }  // namespace
 
 // Suffix products of the per-token forget gates of one (stream, head), in log space.  The block
-// walks the tokens from the end of the sequence in tiles of 256 x 8; inside a tile every thread owns
-// 8 consecutive tokens, the threads' sums are combined by a suffix scan (warp shuffles, then the 8
-// warp totals through shared memory), and `carry` holds the log-product of all later tiles.
-__global__ void __launch_bounds__(256) decay_weights_kernel(const float* __restrict__ alpha,
-                                                            float* __restrict__ w, float* __restrict__ total,
-                                                            int L, int H)
+// (1024 threads) walks the tokens from the end of the sequence in tiles of 1024 x seg, seg chosen
+// by the host so that a block of up to 8192 tokens is a single tile with every thread busy; inside
+// a tile every thread owns seg consecutive tokens, the threads' sums are combined by a suffix scan
+// (warp shuffles, then the 32 warp totals through shared memory), and `carry` holds the
+// log-product of all later tiles.
+__global__ void __launch_bounds__(1024) decay_weights_kernel(const float* __restrict__ alpha,
+                                                             float* __restrict__ w, float* __restrict__ total,
+                                                             int L, int H, int seg)
 {
-    constexpr int SEG = 8, TILE = 256 * SEG;
-    __shared__ float warp_tot[8];
+    constexpr int kMaxSeg = 8;
+    __shared__ float warp_tot[32];
     const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const size_t base = (size_t)b * L * H + h;
+    const int tile_tokens = 1024 * seg;
     float carry = 0.0f;
-    const int ntile = (L + TILE - 1) / TILE;
+    const int ntile = (L + tile_tokens - 1) / tile_tokens;
     for (int tile = ntile - 1; tile >= 0; --tile) {
-        const int l0 = tile * TILE + tid * SEG;
-        float la[SEG];
+        const int l0 = tile * tile_tokens + tid * seg;
+        float la[kMaxSeg];
         float mine = 0.0f;
+        // every load goes out before the first logarithm
 #pragma unroll
-        for (int i = 0; i < SEG; ++i) {
-            float v = 0.0f;   // tokens past L: alpha = 1
-            if (l0 + i < L) {
-                const float x = alpha[base + (size_t)(l0 + i) * H];
-                v = x >= 0.0f ? -log1pf(expf(-x)) : x - log1pf(expf(x));
-            }
+        for (int i = 0; i < kMaxSeg; ++i)
+            la[i] = (i < seg && l0 + i < L) ? alpha[base + (size_t)(l0 + i) * H] : INFINITY;   // past L: alpha = 1
+#pragma unroll
+        for (int i = 0; i < kMaxSeg; ++i) {
+            const float x = la[i];
+            const float v = x >= 0.0f ? -log1pf(expf(-x)) : x - log1pf(expf(x));   // log sigmoid(x)
             la[i] = v;
             mine += v;
         }
@@ -909,14 +913,15 @@ __global__ void __launch_bounds__(256) decay_weights_kernel(const float* __restr
         }
         if (lane == 0) warp_tot[wid] = incl;
         __syncthreads();
-        float later_warps = 0.0f;
-        for (int q = wid + 1; q < 8; ++q) later_warps += warp_tot[q];
-        float tile_total = 0.0f;
-        for (int q = 0; q < 8; ++q) tile_total += warp_tot[q];
+        float later_warps = 0.0f, tile_total = 0.0f;
+        for (int q = 31; q >= 0; --q) {
+            if (q == wid) later_warps = tile_total;
+            tile_total += warp_tot[q];
+        }
         float run = carry + later_warps + (incl - mine);   // log-product of every token after mine
 #pragma unroll
-        for (int i = SEG - 1; i >= 0; --i) {
-            if (l0 + i < L) w[base + (size_t)(l0 + i) * H] = expf(run);
+        for (int i = kMaxSeg - 1; i >= 0; --i) {
+            if (i < seg && l0 + i < L) w[base + (size_t)(l0 + i) * H] = expf(run);
             run += la[i];
         }
         carry += tile_total;
@@ -927,7 +932,9 @@ __global__ void __launch_bounds__(256) decay_weights_kernel(const float* __restr
 
 int decay_weights(const Shape& s, const float* alpha_logits, float* w, float* total, cudaStream_t st)
 {
-    decay_weights_kernel<<<dim3(s.H, s.B), 256, 0, st>>>(alpha_logits, w, total, s.L, s.H);
+    int seg = (s.L + 1023) / 1024;
+    seg = seg < 1 ? 1 : seg > 8 ? 8 : seg;
+    decay_weights_kernel<<<dim3(s.H, s.B), 1024, 0, st>>>(alpha_logits, w, total, s.L, s.H, seg);
     if (int r = check_launch("decay_weights_kernel")) return r;
     return 1;
 }

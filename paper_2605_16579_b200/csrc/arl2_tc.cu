@@ -1393,14 +1393,17 @@ __global__ void transpose_map_kernel(const __nv_bfloat16* __restrict__ w, __nv_b
     out[t] = v;
 }
 
-// Combines the parts of the split items of a step launch: one warp per query row, a lane owns four
-// output channels.  With part q's reference maximum m_q, row sum l_q and unnormalised row O_q:
+// Combines the parts of the split items of a step launch: a warp takes kMergeRows consecutive query
+// rows of one tile (the item is decoded once per warp), a lane four output channels of each.  With
+// part q's reference maximum m_q, row sum l_q and unnormalised row O_q:
 //   out = sum_q 2^(m_q - m) O_q / sum_q 2^(m_q - m) l_q,   m = max_q m_q,   summed in part order.
+constexpr int kMergeRows = 4;
 __global__ void __launch_bounds__(256)
 tc_split_merge_kernel(const TcStepParams p)
 {
     const int warp = (int)((blockIdx.x * 256u + threadIdx.x) >> 5), lane = threadIdx.x & 31;
-    const int r = warp & (kTile - 1), t = (warp >> 7) & 1, slot = warp >> 8;
+    constexpr int kWarpsPerTile = kTile / kMergeRows;
+    const int r0 = (warp % kWarpsPerTile) * kMergeRows, t = (warp / kWarpsPerTile) & 1, slot = warp / (2 * kWarpsPerTile);
     const bool in_range = slot < p.n_items - p.n_whole;
     Item it;
     if (in_range) it = decode_item<false>(p.n_whole + slot, p);
@@ -1408,37 +1411,46 @@ tc_split_merge_kernel(const TcStepParams p)
     const size_t tp0 = ((size_t)slot * 2 + t) * k;
     asm volatile("griddepcontrol.wait;" ::: "memory");   // the step kernel has finished, its writes are visible
     if (!in_range || t >= it.ntile || p.status[kStatusError] != 0u) return;
-    const int row = it.row0[t] + r;
-    if (row >= p.s.L) return;
-    float w[kMaxSplit], l[kMaxSplit];
-    float4 x[kMaxSplit];
-    float m_all = -INFINITY;
+    const int row0 = it.row0[t] + r0;
+    __nv_bfloat16* obase = p.out + (((size_t)it.b[t] * p.s.L + row0) * p.s.H + it.h[t]) * kTile + lane * 4;
+    // all loads of the warp's rows go out before the first use
+    float2 ml[kMergeRows][kMaxSplit];
+    float4 x[kMergeRows][kMaxSplit];
 #pragma unroll
-    for (int q = 0; q < kMaxSplit; ++q) {
-        if (q < k) {   // all loads go out before the first use
-            const float2 ml = *reinterpret_cast<const float2*>(p.split_ml + ((tp0 + q) * kTile + r) * 2);
-            x[q] = *reinterpret_cast<const float4*>(p.split_o + ((tp0 + q) * kTile + r) * kTile + lane * 4);
-            w[q] = ml.x;
-            l[q] = ml.y;
-            m_all = fmaxf(m_all, ml.x);
+    for (int i = 0; i < kMergeRows; ++i) {
+#pragma unroll
+        for (int q = 0; q < kMaxSplit; ++q) {
+            if (q < k && row0 + i < p.s.L) {
+                const size_t rr = (tp0 + q) * kTile + r0 + i;
+                ml[i][q] = *reinterpret_cast<const float2*>(p.split_ml + rr * 2);
+                x[i][q] = *reinterpret_cast<const float4*>(p.split_o + rr * kTile + lane * 4);
+            }
         }
     }
-    float l_all = 0.0f;
-    float4 acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
 #pragma unroll
-    for (int q = 0; q < kMaxSplit; ++q) {
-        if (q < k) {
-            const float wq = ex2_approx(w[q] - m_all);
-            l_all = fmaf(wq, l[q], l_all);
-            acc.x = fmaf(wq, x[q].x, acc.x);
-            acc.y = fmaf(wq, x[q].y, acc.y);
-            acc.z = fmaf(wq, x[q].z, acc.z);
-            acc.w = fmaf(wq, x[q].w, acc.w);
+    for (int i = 0; i < kMergeRows; ++i) {
+        if (row0 + i >= p.s.L) break;
+        float m_all = -INFINITY;
+#pragma unroll
+        for (int q = 0; q < kMaxSplit; ++q)
+            if (q < k) m_all = fmaxf(m_all, ml[i][q].x);
+        float l_all = 0.0f;
+        float4 acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+#pragma unroll
+        for (int q = 0; q < kMaxSplit; ++q) {
+            if (q < k) {
+                const float wq = ex2_approx(ml[i][q].x - m_all);
+                l_all = fmaf(wq, ml[i][q].y, l_all);
+                acc.x = fmaf(wq, x[i][q].x, acc.x);
+                acc.y = fmaf(wq, x[i][q].y, acc.y);
+                acc.z = fmaf(wq, x[i][q].z, acc.z);
+                acc.w = fmaf(wq, x[i][q].w, acc.w);
+            }
         }
+        const float inv = 1.0f / l_all;
+        *reinterpret_cast<uint2*>(obase + (size_t)i * p.s.H * kTile) =
+            make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
     }
-    const float inv = 1.0f / l_all;
-    __nv_bfloat16* orow = p.out + (((size_t)it.b[t] * p.s.L + row) * p.s.H + it.h[t]) * kTile;
-    *reinterpret_cast<uint2*>(orow + lane * 4) = make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
 }
 
 std::mutex g_setup_mutex;
@@ -1560,9 +1572,9 @@ int tc_step(const StepArgs& a, const __nv_bfloat16* wq_op, const __nv_bfloat16* 
     if (p.k_split == 1) return 1;
     // the parts' rows are combined by a second, small kernel (one warp per row); it may start
     // before the step kernel ends and waits for it at its griddepcontrol.wait
-    const long rows = (long)(p.n_items - p.n_whole) * 2 * kTile;
+    const long warps = (long)(p.n_items - p.n_whole) * 2 * (kTile / kMergeRows);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)((rows + 7) / 8));
+    cfg.gridDim = dim3((unsigned)((warps + 7) / 8));
     cfg.blockDim = dim3(256);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];

@@ -401,52 +401,88 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 }
 
 // S <- alpha S + (sum_s A_s) W_phi_v [- (sum_s G_s) S_old]; one CTA per 16 state rows of a head, 128
-// threads, each a 4 x 4 block of the 16 x 128 output.  The slots of a head are added in index order.
-// The right-hand matrices (the head's value map, then S_old) pass through shared memory as bf16.
-// Every global load the CTA needs is requested before the first result is used.
+// threads.  The slots of a head are added in index order (each thread a 4 x 4 block) into shared
+// memory; the products with the right-hand matrices (the head's value map, then S_old; both bf16)
+// run on the warp-level tensor-core instruction, one 16 x 32 block of the output per warp, with the
+// fp32 sums split into a bf16 head and a bf16 remainder (two MMAs, relative error 2^-17: far below
+// the bf16 rounding of the matrices themselves).  Every global load the CTA needs is requested
+// before the first result is used.
 constexpr int kFinRows = 16;
 constexpr int kFinThreads = 128;
 constexpr int kFinMaxParts = 6;     // slots of one head the unrolled loads cover; more fall back to a loop
-// shared memory: the right-hand matrix as bf16 [128][128], then A and G rows with every value stored
-// twice in a row (x, x): a 16-byte load then yields two packed-FMA operands
-constexpr int kFinSmemBytes = kTileBytes + 2 * kFinRows * kTile * 8;
+constexpr int kFinLdM = kTile + 8;  // bf16 row stride of a right-hand matrix: 272 bytes, conflict-free 8 x 8 loads
+constexpr int kFinLdA = kTile + 8;  // fp32 row stride of the summed rows: a fragment's 8-byte reads spread over the banks
+constexpr int kFinMatBytes = kTile * kFinLdM * 2;
+// shared memory: value map | A rows | delta rule only: S_old | G rows
+constexpr int kFinRowBytes = kFinRows * kFinLdA * 4;
+constexpr int fin_smem_bytes(int mode) { return (mode == 1 ? 2 : 1) * (kFinMatBytes + kFinRowBytes); }
 
+// a [128][128] bf16 matrix from global memory into padded rows of shared memory
 __device__ __forceinline__ void fin_load_matrix(__nv_bfloat16* dst, const __nv_bfloat16* __restrict__ src, int tid)
 {
     const uint4* s4 = reinterpret_cast<const uint4*>(src);
-    uint4* d4 = reinterpret_cast<uint4*>(dst);
-    constexpr int kPer = kTileBytes / 16 / kFinThreads;
+    constexpr int kPer = kTile * kTile / 8 / kFinThreads;   // 16-byte pieces per thread
     uint4 v[kPer];
 #pragma unroll
     for (int i = 0; i < kPer; ++i) v[i] = __ldg(s4 + tid + i * kFinThreads);
 #pragma unroll
-    for (int i = 0; i < kPer; ++i) d4[tid + i * kFinThreads] = v[i];
+    for (int i = 0; i < kPer; ++i) {
+        const int c = tid + i * kFinThreads;
+        *reinterpret_cast<uint4*>(dst + (c >> 4) * kFinLdM + (c & 15) * 8) = v[i];
+    }
 }
 
-// acc[i][j] (+/-)= sum_m X[i][m] * M[m][4 cg + j]   (X: this thread's 4 rows, each value doubled, row
-// stride 256 floats; two columns per packed FMA; bf16 -> fp32 by shifts, off the FMA pipe)
-template <bool kSubtract>
-__device__ __forceinline__ void fin_multiply(uint64_t (&acc)[4][2], const float* __restrict__ X,
-                                             const __nv_bfloat16* __restrict__ M, int cg)
+// x = head + remainder, both bf16 (two values at a time)
+__device__ __forceinline__ void fin_split(float x0, float x1, uint32_t& head, uint32_t& rem)
 {
-    constexpr uint32_t kSign = kSubtract ? 0x80000000u : 0u;
-#pragma unroll 4
-    for (int m = 0; m < kTile; m += 2) {
-        ulonglong2 xr[4];      // (x_m, x_m), (x_m+1, x_m+1) of each row
+    head = pack_bf16(x0, x1);
+    rem = pack_bf16(x0 - __uint_as_float(head << 16), x1 - __uint_as_float(head & 0xFFFF0000u));
+}
+
+__device__ __forceinline__ void fin_mma(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+                 "{%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// acc[j] (+/-)= X[16 x 128] * M[128 x 8 columns of block j], j = 0..3: this warp's 32 columns.
+// X: fp32 rows in shared memory (stride kFinLdA); M: bf16 [m][e] in shared memory (stride kFinLdM).
+// Fragment layout of the instruction (g = lane / 4, t = lane % 4): A rows g, g + 8, columns 2t, 2t + 1
+// (+ 8); B rows 2t, 2t + 1 (+ 8), column g -- the 8 x 8 blocks of M come transposed from ldmatrix.
+template <bool kSubtract>
+__device__ __forceinline__ void fin_multiply(float (&acc)[4][4], const float* __restrict__ X,
+                                             const __nv_bfloat16* __restrict__ M, int warp, int lane)
+{
+    constexpr uint32_t kSign = kSubtract ? 0x80008000u : 0u;
+    const int g = lane >> 2, t = lane & 3;
+    const int mat = lane >> 3;
+    const uint32_t m_base = smem_u32(M + ((lane & 7) + (mat & 1) * 8) * kFinLdM + warp * 32 + (mat >> 1) * 8);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) xr[i] = *reinterpret_cast<const ulonglong2*>(X + i * 2 * kTile + 2 * m);
+    for (int ks = 0; ks < kTile / 16; ++ks) {
+        const float2 x0 = *reinterpret_cast<const float2*>(X + g * kFinLdA + ks * 16 + 2 * t);
+        const float2 x1 = *reinterpret_cast<const float2*>(X + (g + 8) * kFinLdA + ks * 16 + 2 * t);
+        const float2 x2 = *reinterpret_cast<const float2*>(X + g * kFinLdA + ks * 16 + 2 * t + 8);
+        const float2 x3 = *reinterpret_cast<const float2*>(X + (g + 8) * kFinLdA + ks * 16 + 2 * t + 8);
+        uint32_t ah[4], al[4];
+        fin_split(x0.x, x0.y, ah[0], al[0]);
+        fin_split(x1.x, x1.y, ah[1], al[1]);
+        fin_split(x2.x, x2.y, ah[2], al[2]);
+        fin_split(x3.x, x3.y, ah[3], al[3]);
 #pragma unroll
-        for (int mm = 0; mm < 2; ++mm) {
-            const uint2 wb = *reinterpret_cast<const uint2*>(M + (m + mm) * kTile + 4 * cg);   // 4 columns
-            uint64_t w01, w23;
-            asm("mov.b64 %0, {%1, %2};" : "=l"(w01) : "r"((wb.x << 16) ^ kSign), "r"((wb.x & 0xFFFF0000u) ^ kSign));
-            asm("mov.b64 %0, {%1, %2};" : "=l"(w23) : "r"((wb.y << 16) ^ kSign), "r"((wb.y & 0xFFFF0000u) ^ kSign));
+        for (int i = 0; i < 4; ++i) { ah[i] ^= kSign; al[i] ^= kSign; }
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint64_t xx = mm == 0 ? xr[i].x : xr[i].y;
-                acc[i][0] = fma2(xx, w01, acc[i][0]);
-                acc[i][1] = fma2(xx, w23, acc[i][1]);
-            }
+        for (int jj = 0; jj < 2; ++jj) {
+            uint32_t b[4];   // blocks j = 2 jj (b[0], b[1]) and 2 jj + 1 (b[2], b[3])
+            const uint32_t addr = m_base + (uint32_t)((ks * 16 * kFinLdM + jj * 16) * 2);
+            asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(b[0]), "=r"(b[1]), "=r"(b[2]), "=r"(b[3])
+                         : "r"(addr));
+            fin_mma(acc[2 * jj], al, b[0], b[1]);
+            fin_mma(acc[2 * jj], ah, b[0], b[1]);
+            fin_mma(acc[2 * jj + 1], al, b[2], b[3]);
+            fin_mma(acc[2 * jj + 1], ah, b[2], b[3]);
         }
     }
 }
@@ -460,25 +496,29 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
                         int H, int share, int ntile, int nslot, const uint32_t* __restrict__ status)
 {
     extern __shared__ __align__(16) uint8_t fin_smem[];
-    __nv_bfloat16* Ms = reinterpret_cast<__nv_bfloat16*>(fin_smem);                 // [128][128] right-hand matrix
-    float* As = reinterpret_cast<float*>(fin_smem + kTileBytes);                    // [16][128] x 2 (doubled)
-    float* Gs = As + kFinRows * kTile * 2;                                          // same (delta rule)
-    const int tid = threadIdx.x, cg = tid & 31, rg = tid >> 5;
+    __nv_bfloat16* Ws = reinterpret_cast<__nv_bfloat16*>(fin_smem);                  // value map [m][e]
+    float* As = reinterpret_cast<float*>(fin_smem + kFinMatBytes);                   // [16][128] summed rows
+    __nv_bfloat16* Ss = reinterpret_cast<__nv_bfloat16*>(fin_smem + kFinMatBytes + kFinRowBytes);   // S_old [m][e] (delta rule)
+    float* Gs = reinterpret_cast<float*>(fin_smem + 2 * kFinMatBytes + kFinRowBytes);               // its rows
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int cg = lane, rg = warp;                       // the 4 x 4 block this thread sums: rows 4 rg .., columns 4 cg ..
     const int bh = (int)(blockIdx.x / (kTile / kFinRows)), h = bh % H;
-    const int row0 = (int)(blockIdx.x % (kTile / kFinRows)) * kFinRows + rg * 4;   // this thread's 4 rows
+    const int cta_row0 = (int)(blockIdx.x % (kTile / kFinRows)) * kFinRows;
     const size_t head = (size_t)bh * kTile * kTile;
-    const size_t mine = head + (size_t)row0 * kTile + 4 * cg;                      // rows 128 apart
     // Launched with programmatic stream serialisation: the CTA may start while the partial-sum kernel
-    // is still draining.  What does not depend on that kernel (the value map) is fetched first; the
-    // wait below returns once the whole preceding kernel has finished and its writes are visible.
-    if (wv != nullptr) fin_load_matrix(Ms, wv + (size_t)h * kTile * kTile, tid);   // [in = m][out = e]
+    // is still draining.  What does not depend on that kernel (the value map, the current mirror) is
+    // fetched first; the wait below returns once the whole preceding kernel has finished and its
+    // writes are visible.
+    if (wv != nullptr) fin_load_matrix(Ws, wv + (size_t)h * kTile * kTile, tid);
+    if (kMode == 1) fin_load_matrix(Ss, mirror_cur + head, tid);
     const float decay_v = decay[bh];
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t err = status != nullptr ? status[kStatusError] : 0u;
     const int first = (bh * ntile) / share, last = (bh * ntile + ntile - 1) / share;
     const int nparts = last - first + 1;
-    const size_t slot0 = ((size_t)bh * nslot * kTile + row0) * kTile + 4 * cg;
-    // ---- all loads first: the slots, the old state rows, the value map
+    const int sum_row0 = cta_row0 + rg * 4;
+    const size_t slot0 = ((size_t)bh * nslot * kTile + sum_row0) * kTile + 4 * cg;
+    // ---- all loads first: the slots, the old state at the positions of this thread's output fragment
     float4 pa[kFinMaxParts][4];
 #pragma unroll
     for (int s = 0; s < kFinMaxParts; ++s) {
@@ -488,23 +528,26 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
                 pa[s][i] = *reinterpret_cast<const float4*>(partials + slot0 + ((size_t)s * kTile + i) * kTile);
         }
     }
-    float4 old[4];
+    const int g = lane >> 2, t = lane & 3;
+    // output fragment: rows g and g + 8 of the CTA's 16, columns warp * 32 + 8 j + 2 t (+ 1), j = 0..3
+    const size_t out0 = head + (size_t)(cta_row0 + g) * kTile + warp * 32 + 2 * t;
+    float2 old[4][2];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) old[i] = *reinterpret_cast<const float4*>(state + mine + (size_t)i * kTile);
+    for (int j = 0; j < 4; ++j) {
+        old[j][0] = *reinterpret_cast<const float2*>(state + out0 + j * 8);
+        old[j][1] = *reinterpret_cast<const float2*>(state + out0 + j * 8 + 8 * kTile);
+    }
     if (err != 0u) {
         // a partial-sum CTA gave up on a bounded wait: S stays as it was, and so does its mirror
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-            *reinterpret_cast<uint2*>(mirror_next + mine + (size_t)i * kTile) =
-                *reinterpret_cast<const uint2*>(mirror_cur + mine + (size_t)i * kTile);
+        for (int j = 0; j < 4; ++j) {
+            *reinterpret_cast<uint32_t*>(mirror_next + out0 + j * 8) = *reinterpret_cast<const uint32_t*>(mirror_cur + out0 + j * 8);
+            *reinterpret_cast<uint32_t*>(mirror_next + out0 + j * 8 + 8 * kTile) =
+                *reinterpret_cast<const uint32_t*>(mirror_cur + out0 + j * 8 + 8 * kTile);
+        }
         return;
     }
     auto add4 = [](float4& d, const float4& v) { d.x += v.x; d.y += v.y; d.z += v.z; d.w += v.w; };
-    auto store_doubled = [&](float* dst, int i, const float4& v) {     // row rg * 4 + i, columns 4 cg .. + 3
-        float4* d = reinterpret_cast<float4*>(dst + (size_t)(rg * 4 + i) * 2 * kTile + 8 * cg);
-        d[0] = make_float4(v.x, v.x, v.y, v.y);
-        d[1] = make_float4(v.z, v.z, v.w, v.w);
-    };
     float4 a[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) a[i] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -521,7 +564,7 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
             add4(a[i], *reinterpret_cast<const float4*>(partials + slot0 + ((size_t)s * kTile + i) * kTile));
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i) store_doubled(As, i, a[i]);
+    for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(As + (rg * 4 + i) * kFinLdA + 4 * cg) = a[i];
     if (kMode == 1) {
         float4 gs[4];
 #pragma unroll
@@ -532,34 +575,33 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
                 add4(gs[i], *reinterpret_cast<const float4*>(partials_g + slot0 + ((size_t)s * kTile + i) * kTile));
         }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) store_doubled(Gs, i, gs[i]);
+        for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(Gs + (rg * 4 + i) * kFinLdA + 4 * cg) = gs[i];
     }
     __syncthreads();
-    uint64_t out[4][2];
+    float out[4][4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const bool id = wv == nullptr;
-        out[i][0] = pack2(id ? a[i].x : 0.0f, id ? a[i].y : 0.0f);
-        out[i][1] = pack2(id ? a[i].z : 0.0f, id ? a[i].w : 0.0f);
+    for (int j = 0; j < 4; ++j) {
+        if (wv == nullptr) {   // identity value map: the sums themselves
+            const float2 lo = *reinterpret_cast<const float2*>(As + g * kFinLdA + warp * 32 + j * 8 + 2 * t);
+            const float2 hi = *reinterpret_cast<const float2*>(As + (g + 8) * kFinLdA + warp * 32 + j * 8 + 2 * t);
+            out[j][0] = lo.x; out[j][1] = lo.y; out[j][2] = hi.x; out[j][3] = hi.y;
+        } else {
+            out[j][0] = out[j][1] = out[j][2] = out[j][3] = 0.0f;
+        }
     }
-    if (wv != nullptr) fin_multiply<false>(out, As + (size_t)rg * 4 * 2 * kTile, Ms, cg);
-    if (kMode == 1) {
-        __syncthreads();                                   // every thread is done with the value map
-        fin_load_matrix(Ms, mirror_cur + head, tid);       // S_old [m][e]
-        __syncthreads();
-        fin_multiply<true>(out, Gs + (size_t)rg * 4 * 2 * kTile, Ms, cg);
-    }
+    if (wv != nullptr) fin_multiply<false>(out, As, Ws, warp, lane);
+    if (kMode == 1) fin_multiply<true>(out, Gs, Ss, warp, lane);
     const float alpha = decay_direct ? decay_v : 1.0f / (1.0f + __expf(-decay_v));
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        float o0, o1, o2, o3;
-        unpack2(out[i][0], o0, o1);
-        unpack2(out[i][1], o2, o3);
-        const float4 nw = make_float4(alpha * old[i].x + o0, alpha * old[i].y + o1,
-                                      alpha * old[i].z + o2, alpha * old[i].w + o3);
-        *reinterpret_cast<float4*>(state + mine + (size_t)i * kTile) = nw;
-        *reinterpret_cast<uint2*>(mirror_next + mine + (size_t)i * kTile) =
-            make_uint2(pack_bf16(nw.x, nw.y), pack_bf16(nw.z, nw.w));
+    for (int j = 0; j < 4; ++j) {
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const float2 o = old[j][half];
+            const float2 nw = make_float2(alpha * o.x + out[j][2 * half], alpha * o.y + out[j][2 * half + 1]);
+            const size_t at = out0 + j * 8 + (size_t)half * 8 * kTile;
+            *reinterpret_cast<float2*>(state + at) = nw;
+            *reinterpret_cast<uint32_t*>(mirror_next + at) = pack_bf16(nw.x, nw.y);
+        }
     }
 }
 
@@ -572,8 +614,8 @@ int device_setup(int* num_sms)
         cudaError_t e = opt_in_smem(tc_commit_kernel<0>, kCommitSmemBytes);
         if (e == cudaSuccess) e = opt_in_smem(tc_commit_kernel<1>, kCommitSmemBytes);
         if (e == cudaSuccess) e = opt_in_smem(tc_commit_kernel<2>, kCommitSmemBytes);
-        if (e == cudaSuccess) e = opt_in_smem(tc_commit_finish_kernel<0>, kFinSmemBytes);
-        if (e == cudaSuccess) e = opt_in_smem(tc_commit_finish_kernel<1>, kFinSmemBytes);
+        if (e == cudaSuccess) e = opt_in_smem(tc_commit_finish_kernel<0>, fin_smem_bytes(0));
+        if (e == cudaSuccess) e = opt_in_smem(tc_commit_finish_kernel<1>, fin_smem_bytes(1));
         return e;
     }, num_sms);
 }
@@ -634,7 +676,7 @@ int tc_commit_finish(const CommitArgs& a, cudaStream_t st)
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(a.s.B * a.s.H) * (kTile / kFinRows));
     cfg.blockDim = dim3(kFinThreads);
-    cfg.dynamicSmemBytes = kFinSmemBytes;
+    cfg.dynamicSmemBytes = (size_t)fin_smem_bytes(a.mode == 1 ? 1 : 0);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
