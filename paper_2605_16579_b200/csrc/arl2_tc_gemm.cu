@@ -20,7 +20,7 @@ namespace arl2 {
 
 namespace {
 
-constexpr int kGBM = 128, kGBK = 64;   // the tile is kGBM x BN outputs, BN = 256 or 128 (template)
+constexpr int kGBM = 128, kGBK = 64;   // the tile is kGBM x BN outputs, BN = 256, 192 or 128 (template)
 constexpr int kGStages = 4;
 constexpr int kGABytes = kGBM * kGBK * 2;             // 16 KB
 constexpr int kGBBytes = kGBK * 256 * 2;              // up to 32 KB: groups of 64 columns x 64 rows
@@ -254,6 +254,7 @@ int tc_gemm(const GemmArgs& a, cudaStream_t st)
     int num_sms = 0;
     if (int r = device_setup_once(g_setup_mutex, g_setup, [] {
             cudaError_t e = opt_in_smem(tc_gemm_kernel<256>, kGemmSmemBytes);
+            if (e == cudaSuccess) e = opt_in_smem(tc_gemm_kernel<192>, kGemmSmemBytes);
             if (e == cudaSuccess) e = opt_in_smem(tc_gemm_kernel<128>, kGemmSmemBytes);
             return e;
         }, &num_sms))
@@ -273,6 +274,16 @@ int tc_gemm(const GemmArgs& a, cudaStream_t st)
     // clock as shared memory delivers (measured: 673 against 871 TFLOP/s on the 1536-wide output
     // projection, although its 444 tiles fill three waves exactly); the narrow tile serves N <= 128 only
     p.bn = a.N <= 128 ? 128 : 256;
+    if (p.bn == 256) {
+        // 192 columns instead when that fills the rounds of the persistent grid better: the time is
+        // (rounds of tiles) x (tile width), e.g. the 1536-wide output projection of 4680 tokens is 222
+        // tiles of 256 = two rounds on 148 SMs, the second half empty, but 296 tiles of 192 = two full ones
+        auto cost = [&](int bn) {
+            const long tiles = (long)p.m_tiles * ((a.N + bn - 1) / bn);
+            return ((tiles + num_sms - 1) / num_sms) * bn;
+        };
+        if (cost(192) < cost(256)) p.bn = 192;
+    }
     p.n_tiles = (a.N + p.bn - 1) / p.bn;   // columns past N are fetched as zeros and not stored
     for (int i = 0; i < 4; ++i) p.out[i] = static_cast<__nv_bfloat16*>(a.out[i]);
     p.seg_cols = a.seg_cols; p.ld_out = a.ld_out; p.n_bf16_seg = a.n_bf16_seg;
@@ -283,6 +294,8 @@ int tc_gemm(const GemmArgs& a, cudaStream_t st)
     const int grid = total < num_sms ? total : num_sms;
     if (p.bn == 256)
         tc_gemm_kernel<256><<<grid, kGThreads, kGemmSmemBytes, st>>>(tm_a, tm_b, p);
+    else if (p.bn == 192)
+        tc_gemm_kernel<192><<<grid, kGThreads, kGemmSmemBytes, st>>>(tm_a, tm_b, p);
     else
         tc_gemm_kernel<128><<<grid, kGThreads, kGemmSmemBytes, st>>>(tm_a, tm_b, p);
     cudaError_t e = cudaGetLastError();
