@@ -290,7 +290,8 @@ def step_traffic(cfg, kernel_name):
 
 def short_leg(name, dev, blocks=8):
     """A short run of another workload beside the main one: tokens/s per block and the step kernel's
-    rate.  Three warm-up blocks, then `blocks` timed ones; inputs rotate through two resident sets."""
+    rate.  Three warm-up blocks, then `blocks` timed ones; inputs rotate through resident sets that
+    together exceed the L2 cache (two at least)."""
     import torch
 
     from paper_2605_16579_b200 import arl2, workload
@@ -301,10 +302,13 @@ def short_leg(name, dev, blocks=8):
     wq, wk, wv = (w.to(dev) for w in workload.feature_weights(cfg))
     cos, sin = (t.to(dev) for t in workload.rope_tables(cfg.L, cfg.D))
     layer.set_params(wq, wk, wv, cos, sin)
-    sets = [tuple(t.to(dev) for t in workload.step_inputs(cfg, 0, s)) for s in range(2)]
+    set_bytes = (3 * cfg.D * 2 + 4) * cfg.B * cfg.L * cfg.H
+    nsets = max(2, -(-(160 << 20) // set_bytes))
+    sets = [tuple(t.to(dev) for t in workload.step_inputs(cfg, 0, s)) for s in range(nsets)]
     kc, vc, a = (t.to(dev) for t in workload.commit_inputs(cfg, 0))
     out = torch.empty(cfg.B, cfg.L, cfg.H, cfg.D, dtype=cfg.torch_dtype, device=dev)
     events = []
+    calls = [0]
 
     def block(timed):
         for s in range(cfg.steps):
@@ -312,7 +316,8 @@ def short_leg(name, dev, blocks=8):
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 layer.set_profile_events(e0, e1)
                 events.append((e0, e1))
-            layer.denoise_step(*sets[s % 2], out=out)
+            layer.denoise_step(*sets[calls[0] % nsets], out=out)
+            calls[0] += 1
         layer.commit(kc, vc, a)
 
     for _ in range(3):
@@ -332,7 +337,7 @@ def short_leg(name, dev, blocks=8):
             "tokens_per_s": cfg.B * cfg.L * cfg.steps / (ms_block * 1e-3), "step_kernel_ms": kern,
             "step_kernel_tflops": tf, "frac_of_burst": tf / pk["bf16_tflops"],
             "frac_of_sustained": tf / pk["bf16_tflops_sustained"],
-            "l2": "two resident input sets of %d MiB" % (sum(t.numel() * t.element_size() for t in sets[0]) >> 20)}
+            "l2": "%d resident input sets of %d MiB" % (nsets, sum(t.numel() * t.element_size() for t in sets[0]) >> 20)}
 
 
 def stack_leg(dev, horizons=(1, 2, 4, 8, 16), n_layers=30, n_hybrid=23):
@@ -726,9 +731,10 @@ def run_ours(args):
             teacher["ms_per_pass"].append(statistics.mean(ts))
             del kcache, vcache
         layer.sync_status()
-    batched = None
+    batched, chunked = None, None
     if rank == 0 and world == 1 and cfg.name == "long" and not args.no_batched_leg:
         batched = short_leg("batched", dev, blocks=8)
+        chunked = short_leg("chunked", dev, blocks=16)
     stack = None
     if rank == 0 and world == 1 and layer.step_kernel == "tcgen05" and not args.no_stack:
         stack = stack_leg(dev)
@@ -802,6 +808,7 @@ def run_ours(args):
             },
             "teacher_horizon": teacher,
             "batched_leg": batched,
+            "chunked_leg": chunked,
             "module_stack": stack,
         }
         if world == 1 and not args.no_cpu_baseline:
@@ -834,7 +841,7 @@ def main():
     ap.add_argument("--workload", default="long", choices=["tiny", "small", "chunked", "batched", "long"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-teacher", action="store_true", help="skip the teacher-attention horizon leg")
-    ap.add_argument("--no-batched-leg", action="store_true", help="skip the short run of the batched workload")
+    ap.add_argument("--no-batched-leg", action="store_true", help="skip the short runs of the batched and chunked workloads")
     ap.add_argument("--no-stack", action="store_true", help="skip the 30-layer module stack leg")
     ap.add_argument("--traffic-probe", action="store_true",
                     help="set up, run four denoise passes and a commit, exit (for a one-launch profiler capture)")
