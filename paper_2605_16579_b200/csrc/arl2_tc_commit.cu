@@ -417,20 +417,21 @@ constexpr int kFinMatBytes = kTile * kFinLdM * 2;
 constexpr int kFinRowBytes = kFinRows * kFinLdA * 4;
 constexpr int fin_smem_bytes(int mode) { return (mode == 1 ? 2 : 1) * (kFinMatBytes + kFinRowBytes); }
 
-// a [128][128] bf16 matrix from global memory into padded rows of shared memory
+// a [128][128] bf16 matrix from global memory into padded rows of shared memory, as asynchronous
+// 16-byte copies (no registers, and the thread goes on to request its other loads at once);
+// fin_matrices_landed() before the matrix is read
 __device__ __forceinline__ void fin_load_matrix(__nv_bfloat16* dst, const __nv_bfloat16* __restrict__ src, int tid)
 {
-    const uint4* s4 = reinterpret_cast<const uint4*>(src);
     constexpr int kPer = kTile * kTile / 8 / kFinThreads;   // 16-byte pieces per thread
-    uint4 v[kPer];
-#pragma unroll
-    for (int i = 0; i < kPer; ++i) v[i] = __ldg(s4 + tid + i * kFinThreads);
 #pragma unroll
     for (int i = 0; i < kPer; ++i) {
         const int c = tid + i * kFinThreads;
-        *reinterpret_cast<uint4*>(dst + (c >> 4) * kFinLdM + (c & 15) * 8) = v[i];
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst + (c >> 4) * kFinLdM + (c & 15) * 8)),
+                     "l"(src + (size_t)c * 8)
+                     : "memory");
     }
 }
+__device__ __forceinline__ void fin_matrices_landed() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
 // x = head + remainder, both bf16 (two values at a time)
 __device__ __forceinline__ void fin_split(float x0, float x1, uint32_t& head, uint32_t& rem)
@@ -479,9 +480,10 @@ __device__ __forceinline__ void fin_multiply(float (&acc)[4][4], const float* __
             asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
                          : "=r"(b[0]), "=r"(b[1]), "=r"(b[2]), "=r"(b[3])
                          : "r"(addr));
+            // the two accumulators alternate, so that no instruction waits for the one before it
             fin_mma(acc[2 * jj], al, b[0], b[1]);
-            fin_mma(acc[2 * jj], ah, b[0], b[1]);
             fin_mma(acc[2 * jj + 1], al, b[2], b[3]);
+            fin_mma(acc[2 * jj], ah, b[0], b[1]);
             fin_mma(acc[2 * jj + 1], ah, b[2], b[3]);
         }
     }
@@ -545,6 +547,7 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
             *reinterpret_cast<uint32_t*>(mirror_next + out0 + j * 8 + 8 * kTile) =
                 *reinterpret_cast<const uint32_t*>(mirror_cur + out0 + j * 8 + 8 * kTile);
         }
+        fin_matrices_landed();   // no copy into this CTA's shared memory outlives it
         return;
     }
     auto add4 = [](float4& d, const float4& v) { d.x += v.x; d.y += v.y; d.z += v.z; d.w += v.w; };
@@ -577,6 +580,7 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
 #pragma unroll
         for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(Gs + (rg * 4 + i) * kFinLdA + 4 * cg) = gs[i];
     }
+    fin_matrices_landed();
     __syncthreads();
     float out[4][4];
 #pragma unroll
