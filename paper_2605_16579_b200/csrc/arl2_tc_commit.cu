@@ -368,7 +368,10 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 if (!ok) break;
                 tc_fence_after();
                 const int part = (int)blockIdx.x - (bh * p.ntile) / p.share;
-                const size_t at = (((size_t)bh * p.nslot + part) * kTile + r) * kTile + hf * 64;
+                // inside a slot the 128 x 128 sums are stored in groups of 8 columns, rows running fastest
+                // (element (row, col) at ((col / 8) * 128 + row) * 8 + col % 8): the 32 rows of a warp
+                // then write 1 KB in one piece with every store instruction
+                const size_t at = ((size_t)bh * p.nslot + part) * kTile * kTile + ((size_t)(hf * 8) * kTile + r) * 8;
 #pragma unroll 1
                 for (int acc = 0; acc < (kMode == 1 ? 2 : 1); ++acc) {
                     float* dst = (acc == 0 ? p.partials : p.partials_g) + at;
@@ -378,8 +381,8 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                         tmem_ld32(lane_base + kColDS + acc * kTile + hf * 64 + c * 32, o);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int e = 0; e < 4; ++e)   // 32-byte stores: whole sectors
-                            asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + c * 32 + e * 8),
+                        for (int e = 0; e < 4; ++e)   // 32-byte stores: whole sectors, the warp's 32 side by side
+                            asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + (size_t)(c * 4 + e) * kTile * 8),
                                          "r"(o[e * 8]), "r"(o[e * 8 + 1]), "r"(o[e * 8 + 2]), "r"(o[e * 8 + 3]), "r"(o[e * 8 + 4]),
                                          "r"(o[e * 8 + 5]), "r"(o[e * 8 + 6]), "r"(o[e * 8 + 7])
                                          : "memory");
@@ -519,7 +522,8 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
     const int first = (bh * ntile) / share, last = (bh * ntile + ntile - 1) / share;
     const int nparts = last - first + 1;
     const int sum_row0 = cta_row0 + rg * 4;
-    const size_t slot0 = ((size_t)bh * nslot * kTile + sum_row0) * kTile + 4 * cg;
+    // slots hold their sums in groups of 8 columns, rows running fastest (see the write-out)
+    const size_t slot0 = (size_t)bh * nslot * kTile * kTile + ((size_t)(cg >> 1) * kTile + sum_row0) * 8 + (cg & 1) * 4;
     // ---- all loads first: the slots, the old state at the positions of this thread's output fragment
     float4 pa[kFinMaxParts][4];
 #pragma unroll
@@ -527,7 +531,7 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
         if (s < nparts) {
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-                pa[s][i] = *reinterpret_cast<const float4*>(partials + slot0 + ((size_t)s * kTile + i) * kTile);
+                pa[s][i] = *reinterpret_cast<const float4*>(partials + slot0 + (size_t)s * kTile * kTile + i * 8);
         }
     }
     const int g = lane >> 2, t = lane & 3;
@@ -564,7 +568,7 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
     for (int s = kFinMaxParts; s < nparts; ++s) {
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-            add4(a[i], *reinterpret_cast<const float4*>(partials + slot0 + ((size_t)s * kTile + i) * kTile));
+            add4(a[i], *reinterpret_cast<const float4*>(partials + slot0 + (size_t)s * kTile * kTile + i * 8));
     }
 #pragma unroll
     for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(As + (rg * 4 + i) * kFinLdA + 4 * cg) = a[i];
@@ -575,7 +579,7 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
         for (int s = 0; s < nparts; ++s) {
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-                add4(gs[i], *reinterpret_cast<const float4*>(partials_g + slot0 + ((size_t)s * kTile + i) * kTile));
+                add4(gs[i], *reinterpret_cast<const float4*>(partials_g + slot0 + (size_t)s * kTile * kTile + i * 8));
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(Gs + (rg * 4 + i) * kFinLdA + 4 * cg) = gs[i];
