@@ -121,6 +121,23 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async_smem();
+        // this thread is the TMA producer: the run's first map and first tile are requested now, while
+        // tensor memory is still being allocated (nothing else can start before they land)
+        if (n_my > 0) {
+            int bh, tl;
+            tile_of(0, bh, tl);
+            const int hb = bh / H, hh = bh - hb * H;
+            mbar_expect_tx(bars + 8 * kCBarWFull, kTileBytes);
+            tma_load_2d(smem_base + kCOffWk, &tm_wk, bars + 8 * kCBarWFull, 0, hh * kTile);
+            tma_load_2d(smem_base + kCOffWk + kHalfBytes, &tm_wk, bars + 8 * kCBarWFull, 64, hh * kTile);
+            const uint32_t bar = bars + 8 * (kCBarStageFull0 + 0);
+            const uint32_t dst = smem_base + stage_k(0);
+            mbar_expect_tx(bar, 2 * kTileBytes);
+            tma_load_4d(dst, &tm_k, bar, 0, hh, tl * kTile, hb);
+            tma_load_4d(dst + kHalfBytes, &tm_k, bar, 64, hh, tl * kTile, hb);
+            tma_load_4d(dst + kTileBytes, &tm_v, bar, 0, hh, tl * kTile, hb);
+            tma_load_4d(dst + kTileBytes + kHalfBytes, &tm_v, bar, 64, hh, tl * kTile, hb);
+        }
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(tmem_slot), 512);
@@ -136,11 +153,8 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0 && n_my > 0) {
-            prefetch_tensormap(&tm_k);
-            prefetch_tensormap(&tm_v);
-            prefetch_tensormap(&tm_wk);
             bool ok = true;
-            int n_w = 0, issued = 0;
+            int n_w = 1, issued = 1;   // tile 0 and its map went out in the prologue
             for (int k = 0; k < n_my && ok; ++k) {
                 int bh, tl;
                 tile_of(k, bh, tl);
@@ -148,15 +162,17 @@ tc_commit_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 const int s = k % kS;
                 if (k >= kS) ok = wait_bar(bars + 8 * (kCBarStageFree0 + s), (uint32_t)((k / kS) - 1) & 1u, ab, 80);
                 if (!ok) break;
-                const uint32_t bar = bars + 8 * (kCBarStageFull0 + s);
-                const uint32_t dst = smem_base + stage_k(s);
-                mbar_expect_tx(bar, 2 * kTileBytes);
-                tma_load_4d(dst, &tm_k, bar, 0, hh, tl * kTile, hb);
-                tma_load_4d(dst + kHalfBytes, &tm_k, bar, 64, hh, tl * kTile, hb);
-                tma_load_4d(dst + kTileBytes, &tm_v, bar, 0, hh, tl * kTile, hb);
-                tma_load_4d(dst + kTileBytes + kHalfBytes, &tm_v, bar, 64, hh, tl * kTile, hb);
-                ++issued;
-                if (seg_first(k)) {
+                if (k > 0) {
+                    const uint32_t bar = bars + 8 * (kCBarStageFull0 + s);
+                    const uint32_t dst = smem_base + stage_k(s);
+                    mbar_expect_tx(bar, 2 * kTileBytes);
+                    tma_load_4d(dst, &tm_k, bar, 0, hh, tl * kTile, hb);
+                    tma_load_4d(dst + kHalfBytes, &tm_k, bar, 64, hh, tl * kTile, hb);
+                    tma_load_4d(dst + kTileBytes, &tm_v, bar, 0, hh, tl * kTile, hb);
+                    tma_load_4d(dst + kTileBytes + kHalfBytes, &tm_v, bar, 64, hh, tl * kTile, hb);
+                    ++issued;
+                }
+                if (k > 0 && seg_first(k)) {
                     // the map of this head: once the MMAs that read the previous head's are done
                     if (n_w > 0) ok = wait_bar(bars + 8 * kCBarWFree, (uint32_t)(n_w - 1) & 1u, ab, 81);
                     if (!ok) break;
