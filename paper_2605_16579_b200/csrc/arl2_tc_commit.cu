@@ -522,7 +522,9 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
     __nv_bfloat16* Ss = reinterpret_cast<__nv_bfloat16*>(fin_smem + kFinMatBytes + kFinRowBytes);   // S_old [m][e] (delta rule)
     float* Gs = reinterpret_cast<float*>(fin_smem + 2 * kFinMatBytes + kFinRowBytes);               // its rows
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int cg = lane, rg = warp;                       // the 4 x 4 block this thread sums: rows 4 rg .., columns 4 cg ..
+    // what this thread sums: row lane / 2 of the CTA's 16, four columns (lane % 2) * 4 .. of each of
+    // the column groups 4 warp .. 4 warp + 3 -- a warp then reads 512 contiguous bytes of a slot at a time
+    const int srow = lane >> 1, shalf = lane & 1;
     const int bh = (int)(blockIdx.x / (kTile / kFinRows)), h = bh % H;
     const int cta_row0 = (int)(blockIdx.x % (kTile / kFinRows)) * kFinRows;
     const size_t head = (size_t)bh * kTile * kTile;
@@ -537,9 +539,9 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
     const uint32_t err = status != nullptr ? status[kStatusError] : 0u;
     const int first = (bh * ntile) / share, last = (bh * ntile + ntile - 1) / share;
     const int nparts = last - first + 1;
-    const int sum_row0 = cta_row0 + rg * 4;
-    // slots hold their sums in groups of 8 columns, rows running fastest (see the write-out)
-    const size_t slot0 = (size_t)bh * nslot * kTile * kTile + ((size_t)(cg >> 1) * kTile + sum_row0) * 8 + (cg & 1) * 4;
+    // slots hold their sums in groups of 8 columns, rows running fastest (see the write-out); from one
+    // of this thread's column groups to the next: 128 rows x 8
+    const size_t slot0 = (size_t)bh * nslot * kTile * kTile + ((size_t)(warp * 4) * kTile + cta_row0 + srow) * 8 + shalf * 4;
     // ---- all loads first: the slots, the old state at the positions of this thread's output fragment
     float4 pa[kFinMaxParts][4];
 #pragma unroll
@@ -547,7 +549,7 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
         if (s < nparts) {
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-                pa[s][i] = *reinterpret_cast<const float4*>(partials + slot0 + (size_t)s * kTile * kTile + i * 8);
+                pa[s][i] = *reinterpret_cast<const float4*>(partials + slot0 + (size_t)s * kTile * kTile + (size_t)i * kTile * 8);
         }
     }
     const int g = lane >> 2, t = lane & 3;
@@ -584,10 +586,10 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
     for (int s = kFinMaxParts; s < nparts; ++s) {
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-            add4(a[i], *reinterpret_cast<const float4*>(partials + slot0 + (size_t)s * kTile * kTile + i * 8));
+            add4(a[i], *reinterpret_cast<const float4*>(partials + slot0 + (size_t)s * kTile * kTile + (size_t)i * kTile * 8));
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(As + (rg * 4 + i) * kFinLdA + 4 * cg) = a[i];
+    for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(As + srow * kFinLdA + (warp * 4 + i) * 8 + shalf * 4) = a[i];
     if (kMode == 1) {
         float4 gs[4];
 #pragma unroll
@@ -595,10 +597,10 @@ tc_commit_finish_kernel(float* __restrict__ state, const float* __restrict__ par
         for (int s = 0; s < nparts; ++s) {
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-                add4(gs[i], *reinterpret_cast<const float4*>(partials_g + slot0 + (size_t)s * kTile * kTile + i * 8));
+                add4(gs[i], *reinterpret_cast<const float4*>(partials_g + slot0 + (size_t)s * kTile * kTile + (size_t)i * kTile * 8));
         }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(Gs + (rg * 4 + i) * kFinLdA + 4 * cg) = gs[i];
+        for (int i = 0; i < 4; ++i) *reinterpret_cast<float4*>(Gs + srow * kFinLdA + (warp * 4 + i) * 8 + shalf * 4) = gs[i];
     }
     fin_matrices_landed();
     __syncthreads();
