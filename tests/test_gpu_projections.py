@@ -47,6 +47,42 @@ def test_projections_match_oracle(oracle, B, H, L):
     layer.sync_status()
 
 
+@pytest.mark.parametrize("B,H", [(1, 12), (2, 20)])
+def test_projections_full_size_sampled_rows(oracle, B, H):
+    """The base model's geometry (4680 tokens, d = 1536) and a wider, two-stream one: 37 and 74 row
+    tiles walk more than one band of the persistent tile order, the output projection takes the
+    192-column tile.  A GEMM's rows are independent, so the oracle computes sampled rows (first and
+    last rows of tiles, band boundaries, the ragged tail tile in full) as a shorter sequence."""
+    L, d = 4680, H * 128
+    layer = arl2.Layer(B, H, L, 128, "bf16", device=DEV)
+    w_q, w_k, w_v, w_g, w_o = weights(d, H, 27)
+    layer.set_projections(*(w.to(DEV) for w in (w_q, w_k, w_v, w_g, w_o)))
+    gen = torch.Generator().manual_seed(28)
+    x = torch.randn(B, L, d, generator=gen).to(torch.bfloat16)
+    o = torch.randn(B, L, H, 128, generator=gen).to(torch.bfloat16)
+    rows = sorted(set([0, 1, 127, 128, 255, 256, 4095, 4096, 4097, 4223, 4224]
+                      + list(range(4608, 4680))
+                      + torch.randint(0, L, (48,), generator=gen).tolist()))
+    nan = float("nan")
+    q, k, v = (torch.full((B, L, H, 128), nan, dtype=torch.bfloat16, device=DEV) for _ in range(3))
+    g = torch.full((B, L, H), nan, device=DEV)
+    y = torch.full((B, L, d), nan, dtype=torch.bfloat16, device=DEV)
+    layer.project_in(x.to(DEV), q, k, v, g)
+    layer.project_out(o.to(DEV), y)
+    layer.sync_status()
+    for t in (q, k, v, g, y):
+        assert torch.isfinite(t.float()).all()          # every element was written
+    rq, rk, rv, rg = oracle.project_in(x[:, rows].contiguous(), w_q, w_k, w_v, w_g, H)
+    ry = oracle.project_out(o[:, rows].contiguous(), w_o)
+    idx = torch.tensor(rows, device=DEV)
+    worst = 0.0
+    for name, got, ref in (("q", q, rq), ("k", k, rk), ("v", v, rv), ("g", g, rg), ("y", y, ry)):
+        e = norm_err(got.index_select(1, idx).float().cpu().numpy(), ref)
+        worst = max(worst, e)
+        assert e <= TOL["bf16"], (name, e)
+    print(f"projections B={B} H={H} L={L}: worst normalised error {worst:.2e} on {len(rows)} rows per stream")
+
+
 def test_whole_module_against_the_oracle_composition(oracle):
     """x -> (W_q, W_k, W_v, W_g) -> hybrid core -> W_o, Eq. 7: y' = (O_intra + G . O_inter) W_o."""
     cfg = workload.custom(B=2, H=3, D=128, L=333, dtype="bf16", cfg_id=91)
