@@ -48,6 +48,28 @@ def test_teacher_step_matches_oracle(oracle, B, H, L, Lk):
     assert torch.isfinite(out.float()).all()
 
 
+def test_teacher_step_full_size_sampled_rows(oracle):
+    """The base geometry over a cache of two blocks: 222 work items on 148 SMs, the last 74 cut into
+    two ranges of 37 key tiles each.  Query rows are independent, so the oracle takes sampled rows
+    (tile edges, the ragged tail tile in full) as a shorter block over the whole cache."""
+    cfg = workload.CONFIGS["chunked"]
+    layer = arl2.Layer(cfg.B, cfg.H, cfg.L, cfg.D, cfg.dtype, device=DEV)
+    lk = 2 * cfg.L
+    q, k, v = _inputs(cfg, lk, 4321)
+    out = torch.full((cfg.B, cfg.L, cfg.H, cfg.D), float("nan"), dtype=torch.bfloat16, device=DEV)
+    layer.teacher_step(q.to(DEV), k.to(DEV), v.to(DEV), out=out)
+    layer.sync_status()
+    assert torch.isfinite(out.float()).all()
+    gen = torch.Generator().manual_seed(99)
+    rows = sorted(set([0, 127, 128, 255, 256, 4479, 4480, 4607] + list(range(4608, cfg.L))
+                      + torch.randint(0, cfg.L, (40,), generator=gen).tolist()))
+    ref = oracle.attend_cache(q[:, rows].contiguous(), k, v)
+    got = out.index_select(1, torch.tensor(rows, device=DEV)).float().cpu().numpy()
+    err = float(head_errors(got, ref).max())
+    print(f"teacher step, chunked geometry, cache of 2 blocks: error {err:.2e} on {len(rows)} rows per head")
+    assert err <= TOL["bf16"], f"error {err:.3e}"
+
+
 def test_teacher_step_rejects_other_contexts(oracle):
     cfg = workload.custom(B=1, H=2, D=64, L=64, dtype="fp32", cfg_id=52)
     layer = arl2.Layer(cfg.B, cfg.H, cfg.L, cfg.D, cfg.dtype, device=DEV)
