@@ -55,6 +55,8 @@ MUTANTS = [
      "Sloc[(size_t)d * D + e] = alpha * (Sloc[(size_t)d * D + e] + kf[d] * vf[e]);"),
     ("projection weight read transposed", "acc += x[(size_t)r * K + kk] * w[(size_t)kk * N + n];",
      "acc += x[(size_t)r * K + kk] * w[(size_t)n * K + kk];"),
+    ("keys projected with the query weights", "matmul_rows(rows, d, d, x, w_k, k);", "matmul_rows(rows, d, d, x, w_q, k);"),
+    ("gate logits projected from the wrong weights", "matmul_rows(rows, d, H, x, w_g, g);", "matmul_rows(rows, d, H, x, w_v, g);"),
     ("reset clears the wrong stream", "else memset(S + per * stream, 0, sizeof(double) * per);",
      "else memset(S, 0, sizeof(double) * per);"),
 ]
