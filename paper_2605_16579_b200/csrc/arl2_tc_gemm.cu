@@ -2,14 +2,18 @@
 // x W_g and y = O W_o) as one persistent tcgen05 GEMM kernel: C[M, N] = A[M, K] B[K, N], bf16 operands,
 // fp32 accumulation in tensor memory, bf16 (or, for the gate logits, fp32) results.
 //
-// Tiles of 128 x 256 outputs (128 x 128 when N <= 128), the contraction in blocks of 64; one CTA per
-// SM walks its tiles.
-//   warp 0     TMA producer: per k-block the A tile [128 x 64] (K-major) and the B tile [64 x 256]
-//              (rows = contraction index, as it lies in a row-major (in, out) weight) through a
-//              4-stage ring
-//   warp 1     MMA issuer: 4 MMAs of 128 x 256 x 16 per k-block into one of two TMEM accumulators
-//   warps 2-5  epilogue, one thread per output row: TMEM -> registers -> bf16 -> global, 32-byte
-//              stores; while it drains one accumulator the issuer fills the other
+// Tiles of (128 MH) x BN outputs, MH = 1 or 2 row halves of 128, BN = 256, 192 or 128 columns; the
+// contraction in blocks of 64; one CTA per SM walks its tiles.
+//   warp 0     TMA producer: per k-block the A tile [128 MH x 64] (K-major) and the B tile [64 x BN]
+//              (rows = contraction index, as it lies in a row-major (in, out) weight) through a ring
+//              of 4 (MH = 1) or 3 (MH = 2) stages
+//   warp 1     MMA issuer: per k-block 4 MMAs of 128 x BN x 16 per row half into TMEM accumulators
+//   warps 2-5  epilogue, one thread per output row of a half: TMEM -> registers -> bf16 -> global,
+//              32-byte stores
+// MH = 1 keeps two accumulators (while the epilogue drains one the issuer fills the other).  MH = 2
+// uses the whole of tensor memory for one 256 x 256 tile: both halves share every B block, which
+// cuts the bytes fetched from L2 per flop by a third -- with 128-row tiles the operand fetch
+// (48 KB per 512 MMA clocks) is what the tensor pipe waits for.
 // The N axis is a concatenation of column segments (Q | K | V | gate logits): a tile's columns go to
 // the segment's own tensor, so the three [B, L, H, D] tensors and the [B, L, H] logits come out of one
 // launch in the layouts the attention kernels read.
@@ -20,19 +24,20 @@ namespace arl2 {
 
 namespace {
 
-constexpr int kGBM = 128, kGBK = 64;   // the tile is kGBM x BN outputs, BN = 256, 192 or 128 (template)
-constexpr int kGStages = 4;
-constexpr int kGABytes = kGBM * kGBK * 2;             // 16 KB
+constexpr int kGBM = 128, kGBK = 64;   // an MMA covers kGBM x BN outputs; a tile is MH of them on top of each other
+constexpr int kGMaxStages = 4;
+constexpr int kGABytes = kGBM * kGBK * 2;             // 16 KB per row half
 constexpr int kGBBytes = kGBK * 256 * 2;              // up to 32 KB: groups of 64 columns x 64 rows
-constexpr int kGStageBytes = kGABytes + kGBBytes;
-constexpr int kGOffBars = kGStages * kGStageBytes;
+// 4 stages of one A half + B, or 3 stages of two A halves + B: 192 KB either way
+constexpr int kGOffBars = 4 * (kGABytes + kGBBytes);
+static_assert(3 * (2 * kGABytes + kGBBytes) == kGOffBars, "ring size");
 constexpr int kGemmSmemBytes = kGOffBars + 256 + 1024;
 constexpr int kGThreads = 192;
 
 enum GBar : int {
     kGBarFull0 = 0,
-    kGBarEmpty0 = kGBarFull0 + kGStages,
-    kGBarAccFull0 = kGBarEmpty0 + kGStages, kGBarAccFull1,
+    kGBarEmpty0 = kGBarFull0 + kGMaxStages,
+    kGBarAccFull0 = kGBarEmpty0 + kGMaxStages, kGBarAccFull1,
     kGBarAccFree0, kGBarAccFree1,
     kGBarDrain,
     kGNumBars
@@ -41,7 +46,7 @@ static_assert(kGNumBars * 8 + 16 <= 256, "barrier block");
 
 struct GemmParams {
     int M, N, K;
-    int m_tiles, n_tiles, bn;
+    int m_tiles, n_tiles, bn, tile_rows;   // tile_rows = 128 or 256
     // output routing: column n of the product belongs to segment n / seg_cols; segments
     // 0 .. n_bf16_seg - 1 are bf16 tensors with row stride ld_out, the one after them (if any) is the
     // fp32 tensor out_f32 with f32_cols valid columns and row stride ld_f32
@@ -62,11 +67,11 @@ __device__ __forceinline__ void tile_origin(int t, const GemmParams& p, int& m0,
     const int band = t / per_band, in_band = t - band * per_band;
     const int rows = min(kGBand, p.m_tiles - band * kGBand);   // the last band may be shorter
     const int nt = in_band / rows;
-    m0 = (band * kGBand + in_band - nt * rows) * kGBM;
+    m0 = (band * kGBand + in_band - nt * rows) * p.tile_rows;
     n0 = nt * p.bn;
 }
 
-template <int BN>
+template <int BN, int MH>
 __global__ void __launch_bounds__(kGThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const GemmParams p)
 {
@@ -81,9 +86,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int total = p.m_tiles * p.n_tiles;
     const int n_kb = p.K / kGBK;
+    constexpr int kGStages = MH == 2 ? 3 : 4;
+    constexpr int kGStageBytes = MH * kGABytes + kGBBytes;
 
     if (tid == 0) {
-        for (int s = 0; s < kGStages; ++s) {
+        for (int s = 0; s < kGMaxStages; ++s) {
             mbar_init(bars + 8 * (kGBarFull0 + s), 1);
             mbar_init(bars + 8 * (kGBarEmpty0 + s), 1);
         }
@@ -121,11 +128,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     if (!ok) break;
                     const uint32_t bar = bars + 8 * (kGBarFull0 + s);
                     const uint32_t dst = smem_base + s * kGStageBytes;
-                    mbar_expect_tx(bar, kGABytes + kGBK * BN * 2);
-                    tma_load_2d(dst, &tm_a, bar, kb * kGBK, m0);
+                    mbar_expect_tx(bar, MH * kGABytes + kGBK * BN * 2);
+#pragma unroll
+                    for (int hlf = 0; hlf < MH; ++hlf)   // rows past M are fetched as zeros
+                        tma_load_2d(dst + hlf * kGABytes, &tm_a, bar, kb * kGBK, m0 + hlf * kGBM);
 #pragma unroll
                     for (int g = 0; g < BN / 64; ++g)
-                        tma_load_2d(dst + kGABytes + g * (kGBK * 128), &tm_b, bar, n0 + g * 64, kb * kGBK);
+                        tma_load_2d(dst + MH * kGABytes + g * (kGBK * 128), &tm_b, bar, n0 + g * 64, kb * kGBK);
                 }
             }
             if (!ok || *abort_flag) {
@@ -148,8 +157,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             bool ok = true;
             uint32_t n = 0, it = 0;
             for (int t = blockIdx.x; t < total && ok; t += gridDim.x, ++it) {
-                const uint32_t buf = it & 1u;
-                if (it >= 2) ok = wait_bar(bars + 8 * (kGBarAccFree0 + buf), ((it >> 1) - 1) & 1u, ab, 121);
+                // MH = 1: two accumulators take turns; MH = 2: the one tile fills tensor memory, and its
+                // epilogue must be through before the next tile's first MMA
+                const uint32_t buf = MH == 1 ? (it & 1u) : 0u;
+                if (MH == 1) {
+                    if (it >= 2) ok = wait_bar(bars + 8 * (kGBarAccFree0 + buf), ((it >> 1) - 1) & 1u, ab, 121);
+                } else {
+                    if (it >= 1) ok = wait_bar(bars + 8 * kGBarAccFree0, (it - 1) & 1u, ab, 121);
+                }
                 // ordered after the epilogue's reads of this accumulator; inside the k loop the operands
                 // come from TMA (an mbarrier wait is all they need), and a tcgen05 fence there would hold
                 // the thread until the MMAs already in flight are done
@@ -159,11 +174,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     ok = wait_bar(bars + 8 * (kGBarFull0 + s), (n / kGStages) & 1u, ab, 122);
                     if (!ok) break;
                     const uint32_t a_lo = ((smem_base + s * kGStageBytes) >> 4) | kLboK;
-                    const uint32_t b_lo = ((smem_base + s * kGStageBytes + kGABytes) >> 4) | kLboB;
+                    const uint32_t b_lo = ((smem_base + s * kGStageBytes + MH * kGABytes) >> 4) | kLboB;
 #pragma unroll
-                    for (int ks = 0; ks < kGBK / 16; ++ks)
-                        mma_ss(tmem_base + buf * 256, desc64(a_lo + (uint32_t)((ks * 32) >> 4)),
-                               desc64(b_lo + (uint32_t)(ks * (2048 >> 4))), idesc, (kb > 0 || ks > 0) ? 1u : 0u);
+                    for (int ks = 0; ks < kGBK / 16; ++ks) {
+#pragma unroll
+                        for (int hlf = 0; hlf < MH; ++hlf)
+                            mma_ss(tmem_base + (MH == 1 ? buf : (uint32_t)hlf) * 256,
+                                   desc64(a_lo + (uint32_t)((hlf * kGABytes + ks * 32) >> 4)),
+                                   desc64(b_lo + (uint32_t)(ks * (2048 >> 4))), idesc, (kb > 0 || ks > 0) ? 1u : 0u);
+                    }
                     mma_commit(bars + 8 * (kGBarEmpty0 + s));
                 }
                 if (ok) mma_commit(bars + 8 * (kGBarAccFull0 + buf));
@@ -181,19 +200,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         bool ok = true;
         uint32_t it = 0;
         for (int t = blockIdx.x; t < total && ok; t += gridDim.x, ++it) {
-            const uint32_t buf = it & 1u;
+            const uint32_t buf = MH == 1 ? (it & 1u) : 0u;
             int m0, n0;
             tile_origin(t, p, m0, n0);
-            const int row = m0 + r;
-            ok = wait_bar(bars + 8 * (kGBarAccFull0 + buf), (it >> 1) & 1u, ab, 123);
+            ok = wait_bar(bars + 8 * (kGBarAccFull0 + buf), (MH == 1 ? (it >> 1) : it) & 1u, ab, 123);
             if (!ok) break;
             tc_fence_after();
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
+            for (int c = 0; c < MH * (BN / 32); ++c) {
+                // (MH = 2: the second half's chunks follow the first's; its rows lie 128 further down)
+                const int hlf = c / (BN / 32), cc = c - hlf * (BN / 32);
+                const int row = m0 + hlf * kGBM + r;
                 uint32_t o[32];
-                tmem_ld32(lane_base + buf * 256 + c * 32, o);
+                tmem_ld32(lane_base + (MH == 1 ? buf : (uint32_t)hlf) * 256 + cc * 32, o);
                 tmem_wait_ld();
-                const int n = n0 + c * 32;                                  // 32 columns lie inside one segment
+                const int n = n0 + cc * 32;                                 // 32 columns lie inside one segment
                 if (row >= p.M || n >= p.N) continue;
                 const int seg = n / p.seg_cols, col = n - seg * p.seg_cols;
                 if (seg < p.n_bf16_seg) {
@@ -253,9 +274,11 @@ int tc_gemm(const GemmArgs& a, cudaStream_t st)
 {
     int num_sms = 0;
     if (int r = device_setup_once(g_setup_mutex, g_setup, [] {
-            cudaError_t e = opt_in_smem(tc_gemm_kernel<256>, kGemmSmemBytes);
-            if (e == cudaSuccess) e = opt_in_smem(tc_gemm_kernel<192>, kGemmSmemBytes);
-            if (e == cudaSuccess) e = opt_in_smem(tc_gemm_kernel<128>, kGemmSmemBytes);
+            cudaError_t e = opt_in_smem(tc_gemm_kernel<256, 1>, kGemmSmemBytes);
+            if (e == cudaSuccess) e = opt_in_smem(tc_gemm_kernel<192, 1>, kGemmSmemBytes);
+            if (e == cudaSuccess) e = opt_in_smem(tc_gemm_kernel<128, 1>, kGemmSmemBytes);
+            if (e == cudaSuccess) e = opt_in_smem(tc_gemm_kernel<256, 2>, kGemmSmemBytes);
+            if (e == cudaSuccess) e = opt_in_smem(tc_gemm_kernel<192, 2>, kGemmSmemBytes);
             return e;
         }, &num_sms))
         return r;
@@ -269,21 +292,33 @@ int tc_gemm(const GemmArgs& a, cudaStream_t st)
     if (int r = make_map_2d(&tm_b, a.b, (size_t)a.K, (size_t)a.N, kGBK)) return r;
     GemmParams p;
     p.M = a.M; p.N = a.N; p.K = a.K;
-    p.m_tiles = (a.M + kGBM - 1) / kGBM;
-    // 256 columns per tile: a 128 x 128 tile would read as many operand bytes from shared memory per MMA
-    // clock as shared memory delivers (measured: 673 against 871 TFLOP/s on the 1536-wide output
-    // projection, although its 444 tiles fill three waves exactly); the narrow tile serves N <= 128 only
+    // Tile shape, by a cost in MMA clocks per CTA: (rounds of tiles over the persistent grid) x (time of
+    // a tile).  Measured: a 128-row tile's k-block of 512 MMA clocks takes about 740 (its 48 KB of
+    // operands come from L2 at about 53 B/clk per SM) with the epilogue hidden behind the next tile; a
+    // 256-row tile shares every B block between its halves -- a k-block of 1024 MMA clocks takes about
+    // 1200 -- but fills tensor memory, so its epilogue (about 4000 clocks) is not hidden: it pays for long
+    // contractions (K = 5120: 1430 against 1230 TFLOP/s) and not for K = 1536.  192 columns instead of 256
+    // where that fills the rounds better (the 1536-wide output projection of 4680 tokens: 222 tiles of
+    // 128 x 256 are two rounds on 148 SMs, the second half empty; 296 of 128 x 192 are two full ones).
+    // The 128-column tile serves N <= 128 only: at 128 x 128 both operands of an MMA come from shared
+    // memory at its full rate, measured slower even where it fills the rounds.
+    int mh = 1;
     p.bn = a.N <= 128 ? 128 : 256;
     if (p.bn == 256) {
-        // 192 columns instead when that fills the rounds of the persistent grid better: the time is
-        // (rounds of tiles) x (tile width), e.g. the 1536-wide output projection of 4680 tokens is 222
-        // tiles of 256 = two rounds on 148 SMs, the second half empty, but 296 tiles of 192 = two full ones
-        auto cost = [&](int bn) {
-            const long tiles = (long)p.m_tiles * ((a.N + bn - 1) / bn);
-            return ((tiles + num_sms - 1) / num_sms) * bn;
-        };
-        if (cost(192) < cost(256)) p.bn = 192;
+        const int n_kb = a.K / kGBK;
+        float best = 0.0f;
+        for (int cand_mh = 1; cand_mh <= 2; ++cand_mh) {
+            if (cand_mh == 2 && a.M <= kGBM) break;
+            for (int cand_bn = 256; cand_bn >= 192; cand_bn -= 64) {
+                const long tiles = (long)((a.M + cand_mh * kGBM - 1) / (cand_mh * kGBM)) * ((a.N + cand_bn - 1) / cand_bn);
+                const float tile = (cand_mh == 1 ? n_kb * 740.0f : n_kb * 1200.0f + 4000.0f) * cand_bn / 256.0f;
+                const float cost = (float)((tiles + num_sms - 1) / num_sms) * tile;
+                if (best == 0.0f || cost < best) { best = cost; mh = cand_mh; p.bn = cand_bn; }
+            }
+        }
     }
+    p.tile_rows = mh * kGBM;
+    p.m_tiles = (a.M + p.tile_rows - 1) / p.tile_rows;
     p.n_tiles = (a.N + p.bn - 1) / p.bn;   // columns past N are fetched as zeros and not stored
     for (int i = 0; i < 4; ++i) p.out[i] = static_cast<__nv_bfloat16*>(a.out[i]);
     p.seg_cols = a.seg_cols; p.ld_out = a.ld_out; p.n_bf16_seg = a.n_bf16_seg;
@@ -292,12 +327,16 @@ int tc_gemm(const GemmArgs& a, cudaStream_t st)
     p.spin_limit = a.wait_limit ? a.wait_limit - 1 : kSpinLimit;
     const int total = p.m_tiles * p.n_tiles;
     const int grid = total < num_sms ? total : num_sms;
-    if (p.bn == 256)
-        tc_gemm_kernel<256><<<grid, kGThreads, kGemmSmemBytes, st>>>(tm_a, tm_b, p);
+    if (mh == 2 && p.bn == 256)
+        tc_gemm_kernel<256, 2><<<grid, kGThreads, kGemmSmemBytes, st>>>(tm_a, tm_b, p);
+    else if (mh == 2)
+        tc_gemm_kernel<192, 2><<<grid, kGThreads, kGemmSmemBytes, st>>>(tm_a, tm_b, p);
+    else if (p.bn == 256)
+        tc_gemm_kernel<256, 1><<<grid, kGThreads, kGemmSmemBytes, st>>>(tm_a, tm_b, p);
     else if (p.bn == 192)
-        tc_gemm_kernel<192><<<grid, kGThreads, kGemmSmemBytes, st>>>(tm_a, tm_b, p);
+        tc_gemm_kernel<192, 1><<<grid, kGThreads, kGemmSmemBytes, st>>>(tm_a, tm_b, p);
     else
-        tc_gemm_kernel<128><<<grid, kGThreads, kGemmSmemBytes, st>>>(tm_a, tm_b, p);
+        tc_gemm_kernel<128, 1><<<grid, kGThreads, kGemmSmemBytes, st>>>(tm_a, tm_b, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_error("launch of tc_gemm_kernel failed: %s", cudaGetErrorString(e)); return ARL2_ERR_CUDA; }
     return 1;
